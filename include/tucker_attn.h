@@ -1,0 +1,163 @@
+/*
+ * tucker_attn.h -- C ABI of the B200 (sm_100a) Tucker-attention forward library.
+ *
+ * One Tucker-factorised attention layer ("Tucker Attention", Definition 1 of the paper):
+ * the pre-softmax tensor  W  = C  x_1 U1  x_2 U2  x_3 U3   (n_H x d x d, ranks r1,r2,r3) and
+ * the post-softmax tensor Wt = Ct x_1 Ut1 x_2 Ut2 x_3 Ut3  (ranks t1,t2,t3; mode 2 = output,
+ * mode 3 = value because the transposed per-head matrices are stacked, Eq. 3) are never
+ * formed.  The library evaluates Eq. 6 ("full-rank MHA" on these tensors) in the order of
+ * Sec. 3 of the paper:
+ *
+ *   Qt = X U2,  K = X U3,  V = X Ut3                 latent projections; K, V are the KV cache (Sec. 3.1)
+ *   G_h  = sum_a U1[h,a]  C[a,:,:]                   head-mode core contraction C x_1 U1 (Def. 2, Sec. 3.3)
+ *   Gt_h = sum_a Ut1[h,a] Ct[a,:,:]
+ *   Qhat_h = Qt G_h                                  per-head latent queries (Def. 2)
+ *   latent RoPE: Qhat_{h,m} R(m,r3),  K_n R(n,r3)    rotation in the latent key dimension (Eq. 9, App. C.2)
+ *   S_h = Qhat_h K^T * scale, causal mask, row softmax (online, never materialised; Sec. 3.3)
+ *   O_h = P_h V
+ *   Z   = sum_h O_h Gt_h^T ;  Y = Z Ut2^T            value/output-side factors (Eqs. 5-6)
+ *
+ * and the cached decode step of Eq. 8 for one new token per sequence.
+ *
+ * General conventions
+ *   - Every data pointer is CALLER-OWNED DEVICE memory unless stated otherwise; row-major,
+ *     contiguous, 16-byte aligned.  The library never allocates, frees or keeps a pointer
+ *     after the call returns.  Scratch space is passed in as `workspace`.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t cast to void*; NULL = default
+ *     stream).  No host synchronisation happens inside a call.
+ *   - Storage type (`dtype`): TA_DTYPE_F32 = float everywhere (plain FMA arithmetic, no
+ *     tensor cores); TA_DTYPE_BF16 = __nv_bfloat16 for X, weights, caches and Y with fp32
+ *     accumulation.
+ *   - Return value: TA_OK (0) or a negative tucker_attn_status.  Nothing throws, aborts or
+ *     traps.  Argument errors are detected on the host before anything is launched.
+ *   - RoPE convention: interleaved coordinate pairs (2i, 2i+1) of the r3 latent key
+ *     coordinates, angle pos * rope_base^(-2i/r3); x'[2i] = x[2i] cos - x[2i+1] sin,
+ *     x'[2i+1] = x[2i] sin + x[2i+1] cos; the same rotation for Qhat rows and K rows.
+ *     The K cache holds ROTATED keys.
+ */
+#ifndef TUCKER_ATTN_H_
+#define TUCKER_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TA_API __attribute__((visibility("default")))
+#else
+#define TA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TA_OK = 0,
+  TA_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, rank/shape inconsistency, odd r3 with rope */
+  TA_ERR_UNSUPPORTED_SHAPE = -2,   /* a rank or size outside what the kernels were built for */
+  TA_ERR_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < tucker_attn_*_workspace_bytes(...) */
+  TA_ERR_CUDA = -4,                /* a CUDA runtime / driver call failed (launch, tensor map) */
+  TA_ERR_DEVICE_TIMEOUT = -5       /* a bounded device-side wait gave up (see tucker_attn_last_device_error) */
+} tucker_attn_status;
+
+enum { TA_DTYPE_F32 = 0, TA_DTYPE_BF16 = 1 };
+
+/* Problem descriptor (host memory, read during the call only). */
+typedef struct {
+  int32_t B;          /* independent sequences (no cross-sequence terms) */
+  int32_t N;          /* tokens per sequence (prefill); ignored by decode */
+  int32_t d_model;    /* embedding width d */
+  int32_t n_H;        /* heads; d_model % n_H == 0; d_H = d_model / n_H */
+  int32_t r1, r2, r3; /* pre-softmax tensor: head, query, key ranks   (Definition 1) */
+  int32_t t1, t2, t3; /* post-softmax tensor: head, output, value ranks (Definition 1) */
+  int32_t causal;     /* 1: key n visible to query m iff n <= m */
+  int32_t rope;       /* 1: latent RoPE in r3 (Definition 2); needs r3 even */
+  float   rope_base;  /* e.g. 10000, 500000 */
+  int32_t pos0;       /* absolute position of token 0 of every sequence (prefill) */
+  float   scale;      /* softmax scale; <= 0 selects 1/sqrt(d_model/n_H) (Eq. 4) */
+  int32_t dtype;      /* TA_DTYPE_F32 or TA_DTYPE_BF16 */
+  int32_t flags;      /* TA_FLAG_* bits, 0 = let the library choose */
+} tucker_attn_desc;
+
+enum {
+  TA_FLAG_FORCE_GENERIC = 1   /* run the shape-generic FMA kernels even where a tensor-core path exists */
+};
+
+/* Bytes of scratch the corresponding call needs for this descriptor (0 on invalid descriptor). */
+TA_API size_t tucker_attn_fwd_workspace_bytes(const tucker_attn_desc* desc);
+TA_API size_t tucker_attn_decode_workspace_bytes(const tucker_attn_desc* desc, int32_t Lmax);
+
+/*
+ * Prefill forward of one layer (Definition 1 evaluated through Eq. 6; Sec. 3.1-3.3).
+ *   X    [B, N, d_model]                       in
+ *   C    [r1, r2, r3]   U1  [n_H, r1]   U2  [d_model, r2]   U3  [d_model, r3]      in
+ *   Ct   [t1, t2, t3]   Ut1 [n_H, t1]   Ut2 [d_model, t2]   Ut3 [d_model, t3]      in
+ *   Y    [B, N, d_model]                       out
+ *   Kcache_out [B, Lmax, r3], Vcache_out [B, Lmax, t3]   optional out (both NULL or both set,
+ *        Lmax >= N): rows 0..N-1 of every sequence receive the rotated latent keys and the
+ *        latent values (the KV cache of Sec. 3.1); other rows are left untouched.
+ *   workspace: >= tucker_attn_fwd_workspace_bytes(desc) bytes, 256-byte aligned.
+ * All steps, including the weight-only core contraction, run inside the call.
+ */
+TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
+                    const void* C, const void* U1, const void* U2, const void* U3,
+                    const void* Ct, const void* Ut1, const void* Ut2, const void* Ut3,
+                    void* Y, void* Kcache_out, void* Vcache_out, int32_t Lmax,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * One cached decode step (Eq. 8, "KV Caching"): for every sequence b the new token x[b] at
+ * position L = cache_len[b] attends to cache slots 0..L-1 and to itself.
+ *   x         [B, d_model]                     in
+ *   Kcache    [B, Lmax, r3] rotated latent keys, Vcache [B, Lmax, t3]   in (and out if append)
+ *   cache_len [B] int32, DEVICE memory; 0 <= cache_len[b] < Lmax (checked on the device: an
+ *             out-of-range entry is clamped and flagged in the device error word)
+ *   append    1: the new rotated key / value are also written to slot cache_len[b]
+ *             (the caller increments its lengths); 0: the caches are not modified
+ *   y         [B, d_model]                     out
+ *   desc->N, desc->pos0, desc->causal are ignored.
+ */
+TA_API int tucker_attn_decode(const tucker_attn_desc* desc, const void* x,
+                       const void* C, const void* U1, const void* U2, const void* U3,
+                       const void* Ct, const void* Ut1, const void* Ut2, const void* Ut3,
+                       void* Kcache, void* Vcache, int32_t Lmax,
+                       const int32_t* cache_len, int32_t append,
+                       void* y, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Human-readable name of a status code (static storage). */
+TA_API const char* tucker_attn_status_string(int status);
+
+/*
+ * Device error word.  Kernels never trap: a bounded wait that ran out or an index that
+ * failed a bounds check sets a bit in a per-device word and the kernel returns.  This call
+ * synchronises `cuda_stream`, reads and clears the word of the current device and returns
+ * it (0 = clean; otherwise a bit set of TA_DEVERR_*), or a negative status on CUDA errors.
+ */
+enum {
+  TA_DEVERR_WAIT_TIMEOUT = 1,   /* an mbarrier / flag wait hit its iteration limit */
+  TA_DEVERR_BAD_CACHE_LEN = 2,  /* cache_len[b] outside [0, Lmax) */
+  TA_DEVERR_BAD_INDEX = 4       /* an internal bounds check failed */
+};
+TA_API int tucker_attn_last_device_error(void* cuda_stream);
+
+/* Which path the last tucker_attn_fwd / tucker_attn_decode call on this thread took:
+ * 0 = none yet, 1 = generic FMA kernels, 2 = tensor-core kernels.  Number of kernels that
+ * call launched. */
+TA_API int tucker_attn_last_path(void);
+TA_API int tucker_attn_last_launch_count(void);
+
+/*
+ * Profiling hook (no counterpart in the paper; measurement plumbing).  Registers two
+ * caller-owned cudaEvent_t handles (created with timing enabled) for the calling thread.
+ * While registered, every tucker_attn_fwd / tucker_attn_decode call records `ev_start`
+ * immediately before and `ev_stop` immediately after its dominant kernel (the attention
+ * kernel: scores + online softmax + PV) on the call's stream, so that the caller can read
+ * that kernel's duration with cudaEventElapsedTime after synchronising.  Pass NULL, NULL to
+ * unregister.  Returns TA_OK, or TA_ERR_INVALID_ARG if exactly one handle is NULL.
+ */
+TA_API int tucker_attn_set_profile_events(void* ev_start, void* ev_stop);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TUCKER_ATTN_H_ */

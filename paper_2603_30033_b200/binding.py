@@ -1,0 +1,257 @@
+"""Thin ctypes binding of libtucker_attn.so (the C ABI declared in include/tucker_attn.h).
+
+Only argument marshalling happens here: tensors are checked for device / dtype / contiguity,
+their pointers and the current CUDA stream are handed to the library, and every step of the
+computation runs in the library's kernels.  torch is used for device memory and streams
+only.  If the library has not been built, loading raises; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtucker_attn.so")
+
+TA_OK = 0
+TA_DTYPE_F32, TA_DTYPE_BF16 = 0, 1
+TA_FLAG_FORCE_GENERIC = 1
+TA_DEVERR_WAIT_TIMEOUT, TA_DEVERR_BAD_CACHE_LEN, TA_DEVERR_BAD_INDEX = 1, 2, 4
+
+EXPORTS = (
+    "tucker_attn_fwd_workspace_bytes", "tucker_attn_decode_workspace_bytes", "tucker_attn_fwd",
+    "tucker_attn_decode", "tucker_attn_status_string", "tucker_attn_last_device_error",
+    "tucker_attn_last_path", "tucker_attn_last_launch_count", "tucker_attn_set_profile_events",
+)
+
+
+class TuckerAttnDesc(ctypes.Structure):
+    """Mirror of `tucker_attn_desc`."""
+    _fields_ = [
+        ("B", ctypes.c_int32), ("N", ctypes.c_int32), ("d_model", ctypes.c_int32), ("n_H", ctypes.c_int32),
+        ("r1", ctypes.c_int32), ("r2", ctypes.c_int32), ("r3", ctypes.c_int32),
+        ("t1", ctypes.c_int32), ("t2", ctypes.c_int32), ("t3", ctypes.c_int32),
+        ("causal", ctypes.c_int32), ("rope", ctypes.c_int32), ("rope_base", ctypes.c_float),
+        ("pos0", ctypes.c_int32), ("scale", ctypes.c_float), ("dtype", ctypes.c_int32),
+        ("flags", ctypes.c_int32),
+    ]
+
+
+class TuckerAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where} failed: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2603_30033_b200.build` "
+            "(needs nvcc); this package has no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    dp = ctypes.POINTER(TuckerAttnDesc)
+    lib.tucker_attn_fwd_workspace_bytes.restype = sz
+    lib.tucker_attn_fwd_workspace_bytes.argtypes = [dp]
+    lib.tucker_attn_decode_workspace_bytes.restype = sz
+    lib.tucker_attn_decode_workspace_bytes.argtypes = [dp, i32]
+    lib.tucker_attn_fwd.restype = ctypes.c_int
+    lib.tucker_attn_fwd.argtypes = [dp] + [vp] * 12 + [i32, vp, sz, vp]
+    lib.tucker_attn_decode.restype = ctypes.c_int
+    lib.tucker_attn_decode.argtypes = [dp] + [vp] * 11 + [i32, vp, i32, vp, vp, sz, vp]
+    lib.tucker_attn_status_string.restype = ctypes.c_char_p
+    lib.tucker_attn_status_string.argtypes = [ctypes.c_int]
+    lib.tucker_attn_last_device_error.restype = ctypes.c_int
+    lib.tucker_attn_last_device_error.argtypes = [vp]
+    lib.tucker_attn_last_path.restype = ctypes.c_int
+    lib.tucker_attn_last_launch_count.restype = ctypes.c_int
+    lib.tucker_attn_set_profile_events.restype = ctypes.c_int
+    lib.tucker_attn_set_profile_events.argtypes = [vp, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().tucker_attn_status_string(int(status)).decode()
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _dtype_code(t) -> int:
+    torch = _torch()
+    if t.dtype == torch.float32:
+        return TA_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return TA_DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}; use float32 or bfloat16")
+
+
+def _check(t, name, shape, dtype, device):
+    if t.device != device or not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor on {device}")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} has dtype {t.dtype}, expected {dtype}")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+
+
+def make_desc(*, B, N, d_model, n_H, r, t, causal, rope, rope_base=10000.0, pos0=0, scale=0.0,
+              dtype=TA_DTYPE_BF16, flags=0) -> TuckerAttnDesc:
+    return TuckerAttnDesc(int(B), int(N), int(d_model), int(n_H), int(r[0]), int(r[1]), int(r[2]),
+                          int(t[0]), int(t[1]), int(t[2]), int(bool(causal)), int(bool(rope)),
+                          float(rope_base), int(pos0), float(scale), int(dtype), int(flags))
+
+
+def fwd_workspace_bytes(desc: TuckerAttnDesc) -> int:
+    return int(load_library().tucker_attn_fwd_workspace_bytes(ctypes.byref(desc)))
+
+
+def decode_workspace_bytes(desc: TuckerAttnDesc, Lmax: int) -> int:
+    return int(load_library().tucker_attn_decode_workspace_bytes(ctypes.byref(desc), int(Lmax)))
+
+
+def alloc_workspace(nbytes: int, device):
+    """Device scratch buffer (256-byte aligned by the torch allocator)."""
+    torch = _torch()
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def _stream_ptr(device) -> int:
+    return int(_torch().cuda.current_stream(device).cuda_stream)
+
+
+def _weights_check(w, d_model, n_H, dtype, device):
+    C, U1, U2, U3, Ct, Ut1, Ut2, Ut3 = w
+    if C.dim() != 3 or Ct.dim() != 3:
+        raise ValueError("cores must be 3-way tensors")
+    r = tuple(C.shape)
+    t = tuple(Ct.shape)
+    _check(C, "C", r, dtype, device)
+    _check(U1, "U1", (n_H, r[0]), dtype, device)
+    _check(U2, "U2", (d_model, r[1]), dtype, device)
+    _check(U3, "U3", (d_model, r[2]), dtype, device)
+    _check(Ct, "Ct", t, dtype, device)
+    _check(Ut1, "Ut1", (n_H, t[0]), dtype, device)
+    _check(Ut2, "Ut2", (d_model, t[1]), dtype, device)
+    _check(Ut3, "Ut3", (d_model, t[2]), dtype, device)
+    return r, t
+
+
+def tucker_attn_fwd(X, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, *, n_H: int, causal: bool, rope: bool,
+                    rope_base: float = 10000.0, pos0: int = 0, scale: float = 0.0, out=None,
+                    Kcache=None, Vcache=None, workspace=None, flags: int = 0):
+    """Prefill forward (same name and argument meaning as the C entry point).  X [B, N, d];
+    returns Y [B, N, d].  Kcache [B, Lmax, r3] / Vcache [B, Lmax, t3], when given, receive the
+    rotated latent keys and the latent values in rows 0..N-1."""
+    torch = _torch()
+    lib = load_library()
+    if X.dim() != 3:
+        raise ValueError("X must be [B, N, d_model]")
+    B, N, d = X.shape
+    dev, dt = X.device, X.dtype
+    _check(X, "X", (B, N, d), dt, dev)
+    r, t = _weights_check((C, U1, U2, U3, Ct, Ut1, Ut2, Ut3), d, n_H, dt, dev)
+    desc = make_desc(B=B, N=N, d_model=d, n_H=n_H, r=r, t=t, causal=causal, rope=rope, rope_base=rope_base,
+                     pos0=pos0, scale=scale, dtype=_dtype_code(X), flags=flags)
+    if out is None:
+        out = torch.empty_like(X)
+    _check(out, "out", (B, N, d), dt, dev)
+    Lmax = 0
+    kp = vp = None
+    if (Kcache is None) != (Vcache is None):
+        raise ValueError("pass both caches or neither")
+    if Kcache is not None:
+        Lmax = Kcache.shape[1]
+        _check(Kcache, "Kcache", (B, Lmax, r[2]), dt, dev)
+        _check(Vcache, "Vcache", (B, Lmax, t[2]), dt, dev)
+        kp, vp = Kcache.data_ptr(), Vcache.data_ptr()
+    need = lib.tucker_attn_fwd_workspace_bytes(ctypes.byref(desc))
+    if workspace is None:
+        workspace = alloc_workspace(need, dev)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_attn_fwd(ctypes.byref(desc), X.data_ptr(), C.data_ptr(), U1.data_ptr(), U2.data_ptr(),
+                                 U3.data_ptr(), Ct.data_ptr(), Ut1.data_ptr(), Ut2.data_ptr(), Ut3.data_ptr(),
+                                 out.data_ptr(), kp, vp, int(Lmax), workspace.data_ptr(), workspace.numel(),
+                                 _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_attn_fwd")
+    return out
+
+
+def tucker_attn_decode(x, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, Kcache, Vcache, cache_len, *, n_H: int,
+                       rope: bool, rope_base: float = 10000.0, scale: float = 0.0, append: bool = True,
+                       out=None, workspace=None, flags: int = 0):
+    """One cached decode step (same name and argument meaning as the C entry point).
+    x [B, d]; Kcache [B, Lmax, r3] (rotated keys); Vcache [B, Lmax, t3]; cache_len int32 [B] on
+    the device.  Returns y [B, d]."""
+    torch = _torch()
+    lib = load_library()
+    if x.dim() != 2:
+        raise ValueError("x must be [B, d_model]")
+    B, d = x.shape
+    dev, dt = x.device, x.dtype
+    _check(x, "x", (B, d), dt, dev)
+    r, t = _weights_check((C, U1, U2, U3, Ct, Ut1, Ut2, Ut3), d, n_H, dt, dev)
+    Lmax = Kcache.shape[1]
+    _check(Kcache, "Kcache", (B, Lmax, r[2]), dt, dev)
+    _check(Vcache, "Vcache", (B, Lmax, t[2]), dt, dev)
+    _check(cache_len, "cache_len", (B,), torch.int32, dev)
+    desc = make_desc(B=B, N=1, d_model=d, n_H=n_H, r=r, t=t, causal=True, rope=rope, rope_base=rope_base,
+                     pos0=0, scale=scale, dtype=_dtype_code(x), flags=flags)
+    if out is None:
+        out = torch.empty_like(x)
+    _check(out, "out", (B, d), dt, dev)
+    need = lib.tucker_attn_decode_workspace_bytes(ctypes.byref(desc), int(Lmax))
+    if workspace is None:
+        workspace = alloc_workspace(need, dev)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_attn_decode(ctypes.byref(desc), x.data_ptr(), C.data_ptr(), U1.data_ptr(), U2.data_ptr(),
+                                    U3.data_ptr(), Ct.data_ptr(), Ut1.data_ptr(), Ut2.data_ptr(), Ut3.data_ptr(),
+                                    Kcache.data_ptr(), Vcache.data_ptr(), int(Lmax), cache_len.data_ptr(),
+                                    int(bool(append)), out.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                    _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_attn_decode")
+    return out
+
+
+def last_device_error(device=None) -> int:
+    """Synchronises the current stream and returns-and-clears the device error word."""
+    torch = _torch()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    with torch.cuda.device(dev):
+        return int(load_library().tucker_attn_last_device_error(_stream_ptr(dev)))
+
+
+def last_path() -> int:
+    return int(load_library().tucker_attn_last_path())
+
+
+def last_launch_count() -> int:
+    return int(load_library().tucker_attn_last_launch_count())
+
+
+def set_profile_events(start=None, stop=None) -> None:
+    """Registers two torch.cuda.Event(enable_timing=True) objects (already recorded once, so
+    that their handles exist) to be recorded around the dominant kernel of later calls;
+    call with no arguments to unregister."""
+    lib = load_library()
+    if start is None and stop is None:
+        rc = lib.tucker_attn_set_profile_events(None, None)
+    else:
+        rc = lib.tucker_attn_set_profile_events(start.cuda_event, stop.cuda_event)
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_attn_set_profile_events")

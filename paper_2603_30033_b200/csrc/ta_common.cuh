@@ -1,0 +1,84 @@
+// Shared declarations of the Tucker-attention CUDA library (internal; the public ABI is
+// include/tucker_attn.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "tucker_attn.h"
+
+namespace ta {
+
+typedef __nv_bfloat16 bf16;
+
+// Everything a path needs to run one call; filled by the API layer after validation.
+struct Problem {
+  tucker_attn_desc d;
+  float scale;              // resolved softmax scale
+  const void *X, *C, *U1, *U2, *U3, *Ct, *Ut1, *Ut2, *Ut3;
+  void* Y;
+  void *Kc, *Vc;            // prefill: optional cache outputs; decode: caches
+  int32_t Lmax;
+  const int32_t* cache_len; // decode only (device)
+  int32_t append;           // decode only
+  char* ws;                 // workspace base (256-byte aligned)
+  size_t ws_bytes;
+  cudaStream_t stream;
+  unsigned int* dev_err;    // device error word of the current device
+  int launches;             // kernels launched so far by this call
+  cudaEvent_t prof_start, prof_stop;  // optional: recorded around the dominant kernel
+};
+
+// Records the caller's profiling events (if registered) around the dominant kernel.
+static inline void prof_begin(const Problem& p) { if (p.prof_start) (void)cudaEventRecord(p.prof_start, p.stream); }
+static inline void prof_end(const Problem& p) { if (p.prof_stop) (void)cudaEventRecord(p.prof_stop, p.stream); }
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carves consecutive 256-byte aligned regions out of the workspace; with base == nullptr it
+// only measures.
+struct Carver {
+  char* base;
+  size_t off;
+  explicit Carver(char* b) : base(b), off(0) {}
+  template <typename T>
+  T* take(size_t count) {
+    size_t o = off;
+    off = align_up(off + count * sizeof(T), 256);
+    return base ? reinterpret_cast<T*>(base + o) : nullptr;
+  }
+};
+
+// shape-generic FMA path (ta_generic.cu)
+size_t generic_fwd_workspace(const tucker_attn_desc& d);
+size_t generic_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
+int generic_fwd(Problem& p);
+int generic_decode(Problem& p);
+
+// tensor-core path (bf16 storage): returns false from *_supported when the shape is outside
+// what the kernels were built for, in which case the generic path runs.
+bool fast_fwd_supported(const tucker_attn_desc& d);
+size_t fast_fwd_workspace(const tucker_attn_desc& d);
+int fast_fwd(Problem& p);
+bool fast_decode_supported(const tucker_attn_desc& d, int32_t Lmax);
+size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
+int fast_decode(Problem& p);
+
+#define TA_CUDA_TRY(expr)                          \
+  do {                                             \
+    cudaError_t _e = (expr);                       \
+    if (_e != cudaSuccess) return TA_ERR_CUDA;     \
+  } while (0)
+
+#define TA_LAUNCH_CHECK(p)                                   \
+  do {                                                       \
+    (p).launches++;                                          \
+    if (cudaPeekAtLastError() != cudaSuccess) {              \
+      (void)cudaGetLastError();                              \
+      return TA_ERR_CUDA;                                    \
+    }                                                        \
+  } while (0)
+
+}  // namespace ta

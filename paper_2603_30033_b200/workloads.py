@@ -23,7 +23,7 @@ import numpy as np
 
 __all__ = [
     "Workload", "WORKLOADS", "get_workload", "orthonormal_factor", "make_weights",
-    "make_X", "make_decode_state", "round_to_storage", "prefill_flops", "decode_bytes",
+    "make_X", "make_decode_state", "decode_cache_rows", "make_decode_x", "round_to_storage", "prefill_flops", "decode_bytes",
     "decode_flops",
 ]
 
@@ -73,9 +73,9 @@ def get_workload(name: str) -> Workload:
     raise KeyError(f"unknown workload {name!r}; have {sorted(WORKLOADS)}")
 
 
-def _rng(seed: int, stream: int) -> np.random.Generator:
-    """Independent PCG64 stream per tensor: (seed, stream) -> generator."""
-    return np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, stream])))
+def _rng(seed: int, *stream: int) -> np.random.Generator:
+    """Independent PCG64 stream per tensor: (seed, stream...) -> generator."""
+    return np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, *stream])))
 
 
 def orthonormal_factor(rng: np.random.Generator, rows: int, rank: int) -> np.ndarray:
@@ -142,12 +142,24 @@ def make_decode_state(w: Workload, B: int | None = None, L: int | None = None,
     x = _rng(w.seed, 10).standard_normal((B, w.d_model), dtype=np.float32)
     Kc = np.zeros((B, Lmax, w.r[2]), dtype=np.float32)
     Vc = np.zeros((B, Lmax, w.t[2]), dtype=np.float32)
-    gk, gv = _rng(w.seed, 11), _rng(w.seed, 12)
     for b in range(B):
         n = int(cache_len[b])
-        Kc[b, :n] = gk.standard_normal((n, w.r[2]), dtype=np.float32)
-        Vc[b, :n] = gv.standard_normal((n, w.t[2]), dtype=np.float32)
+        Kc[b, :n], Vc[b, :n] = decode_cache_rows(w, b, n)
     return x, Kc, Vc, cache_len
+
+
+def decode_cache_rows(w: Workload, b: int, n: int):
+    """The first n cached latent key / value rows of sequence b (float32, ~N(0,1)); every
+    sequence has its own stream, so a large cache can be produced one sequence at a time."""
+    k = _rng(w.seed, 11, b).standard_normal((n, w.r[2]), dtype=np.float32)
+    v = _rng(w.seed, 12, b).standard_normal((n, w.t[2]), dtype=np.float32)
+    return k, v
+
+
+def make_decode_x(w: Workload, B: int | None = None) -> np.ndarray:
+    """New-token embeddings x [B, d_model] ~ N(0,1) (same draw as make_decode_state)."""
+    B = w.B if B is None else B
+    return _rng(w.seed, 10).standard_normal((B, w.d_model), dtype=np.float32)
 
 
 def round_to_storage(a: np.ndarray, dtype: str) -> np.ndarray:

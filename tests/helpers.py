@@ -1,0 +1,51 @@
+"""Shared test plumbing: build seeded inputs once, hand bit-identical values to the oracle
+(as float64) and to the CUDA library (as torch tensors of the storage dtype)."""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+
+from paper_2603_30033_b200 import workloads as W
+
+WEIGHT_KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
+
+
+def custom_workload(name="custom", **kw) -> W.Workload:
+    base = dict(name=name, kind="prefill", B=1, N=16, d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), causal=True,
+                rope=False, rope_base=10000.0, dtype="fp32", seed=7)
+    base.update(kw)
+    return W.Workload(**base)
+
+
+def host_inputs(w: W.Workload, B=None, N=None, core_gain=1.0, core_std=None):
+    """Weights and X rounded to the storage dtype, as float64 numpy arrays."""
+    wt = W.make_weights(w, core_std=core_std, core_gain=core_gain)
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in wt.items()}
+    X = W.round_to_storage(W.make_X(w, B=B, N=N), w.dtype)
+    return X, wt
+
+
+def to_device(a: np.ndarray, dtype: str, device="cuda"):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+    t = t.to(torch.bfloat16) if dtype == "bf16" else t
+    return t.to(device).contiguous()
+
+
+def weights_to_device(wt: dict, dtype: str, device="cuda"):
+    return [to_device(wt[k], dtype, device) for k in WEIGHT_KEYS]
+
+
+def err_stats(got, ref):
+    d = np.abs(np.asarray(got, np.float64) - np.asarray(ref, np.float64))
+    return float(d.max()), float(d.mean())
+
+
+def tolerances(dtype: str):
+    """(max-abs, mean-abs) bounds: bf16 storage with fp32 accumulation 2e-2 / 2e-3; fp32 1e-4."""
+    return (2e-2, 2e-3) if dtype == "bf16" else (1e-4, 1e-4)
+
+
+def with_(w: W.Workload, **kw) -> W.Workload:
+    return dataclasses.replace(w, **kw)

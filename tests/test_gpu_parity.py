@@ -1,0 +1,241 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle on the same
+seeded inputs, element by element on small cases and on sampled query rows / sequences at
+the full benchmark sizes.  Bounds: bf16 storage max-abs <= 2e-2 and mean-abs <= 2e-3; fp32
+max-abs <= 1e-4."""
+import numpy as np
+import pytest
+
+from oracle import tucker_oracle as O
+from paper_2603_30033_b200 import binding as Bd
+from paper_2603_30033_b200 import workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_fwd(X, wt, w, rows=None, pos0=0, scale=None):
+    return O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=w.causal, rope=w.rope,
+                             rope_base=w.rope_base, pos0=pos0, rows=rows, scale=scale)
+
+
+def gpu_fwd(X, wt, w, flags=0, pos0=0, caches=None, scale=0.0):
+    dw = H.weights_to_device(wt, w.dtype)
+    Xd = H.to_device(X, w.dtype)
+    kw = {}
+    if caches is not None:
+        kw = dict(Kcache=caches[0], Vcache=caches[1])
+    Y = Bd.tucker_attn_fwd(Xd, *dw, n_H=w.n_H, causal=w.causal, rope=w.rope, rope_base=w.rope_base, pos0=pos0,
+                           flags=flags, scale=scale, **kw)
+    assert Bd.last_device_error() == 0
+    return Y.float().cpu().numpy().astype(np.float64)
+
+
+def check(got, ref, dtype, what=""):
+    mx, mean = H.err_stats(got, ref)
+    tmax, tmean = H.tolerances(dtype)
+    assert np.isfinite(got).all(), what
+    assert mx <= tmax and mean <= tmean, f"{what}: max-abs {mx:.3e} (<= {tmax}), mean-abs {mean:.3e} (<= {tmean})"
+    return mx, mean
+
+
+# --------------------------------------------------------------------------------------
+# config 1: tiny fp32 layer, plus weights that make Tucker attention equal MHA / GQA exactly
+# --------------------------------------------------------------------------------------
+
+def test_c1_tiny_fp32():
+    w = W.get_workload("c1")
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w)
+    check(got, oracle_fwd(X, wt, w), "fp32", "c1")
+    assert Bd.last_path() == 1
+
+
+@pytest.mark.parametrize("n_G", [4, 2, 1])
+def test_c1_mha_gqa_exact_weights(n_G):
+    # ranks (4,128,128) reproduce MHA, (4,128,n_G*32) reproduce GQA / MQA
+    w = W.get_workload("c1")
+    rng = np.random.default_rng(100 + n_G)
+    d, n_H, d_H = w.d_model, w.n_H, w.d_model // w.n_H
+    f32 = lambda a: a.astype(np.float32).astype(np.float64)
+    WQ, WO = (f32(rng.standard_normal((d, d)) / np.sqrt(d)) for _ in range(2))
+    WKg, WVg = (f32(rng.standard_normal((d, n_G * d_H)) / np.sqrt(d)) for _ in range(2))
+    X = f32(rng.standard_normal((1, w.N, d)))
+    wt = O.tucker_from_gqa(WQ, WKg, WVg, WO, n_H, n_G)
+    ref = O.gqa_reference(X[0], WQ, WKg, WVg, WO, n_H, n_G, causal=True)
+    got = gpu_fwd(X, wt, w)[0]
+    check(got, ref, "fp32", f"gqa n_G={n_G}")
+
+
+# --------------------------------------------------------------------------------------
+# small shapes, both storage types, ragged sizes, flags
+# --------------------------------------------------------------------------------------
+
+SMALL = [
+    dict(B=2, N=37, d_model=48, n_H=3, r=(2, 10, 12), t=(3, 9, 7), causal=True, rope=True),
+    dict(B=1, N=130, d_model=64, n_H=4, r=(4, 16, 32), t=(2, 24, 16), causal=False, rope=False),
+    dict(B=3, N=1, d_model=32, n_H=2, r=(1, 4, 6), t=(1, 5, 3), causal=True, rope=True),
+    dict(B=2, N=65, d_model=96, n_H=6, r=(3, 20, 18), t=(6, 33, 40), causal=True, rope=False),
+]
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("shape", SMALL)
+def test_small_shapes_generic(shape, dtype):
+    w = H.custom_workload(dtype=dtype, rope_base=10000.0, seed=31, **shape)
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w, flags=Bd.TA_FLAG_FORCE_GENERIC, pos0=5)
+    check(got, oracle_fwd(X, wt, w, pos0=5), dtype, str(shape))
+
+
+def test_prefill_writes_cache():
+    import torch
+    w = H.custom_workload(dtype="fp32", B=2, N=21, d_model=32, n_H=4, r=(2, 8, 10), t=(2, 8, 6), rope=True, seed=3)
+    X, wt = H.host_inputs(w)
+    Lmax = 30
+    Kc = torch.full((2, Lmax, 10), 7.0, device="cuda")
+    Vc = torch.full((2, Lmax, 6), 7.0, device="cuda")
+    gpu_fwd(X, wt, w, caches=(Kc, Vc))
+    _, parts = O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=True, rope=True, return_parts=True)
+    for b in range(2):
+        np.testing.assert_allclose(Kc[b, :21].cpu().numpy(), parts[b]["K"], atol=1e-5)
+        np.testing.assert_allclose(Vc[b, :21].cpu().numpy(), parts[b]["V"], atol=1e-5)
+    assert (Kc[:, 21:] == 7.0).all() and (Vc[:, 21:] == 7.0).all()
+
+
+def test_custom_scale_and_invariants():
+    # scale override; permutation equivariance without mask; causal prefix independence
+    w = H.custom_workload(dtype="fp32", B=1, N=40, d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), causal=False, seed=9)
+    X, wt = H.host_inputs(w)
+    check(gpu_fwd(X, wt, w, scale=0.3), oracle_fwd(X, wt, w, scale=0.3), "fp32", "scale")
+    perm = np.random.default_rng(0).permutation(40)
+    a, b = gpu_fwd(X, wt, w), gpu_fwd(X[:, perm], wt, w)
+    assert np.abs(a[:, perm] - b).max() < 1e-5
+    wc = H.with_(w, causal=True, rope=True)
+    X2 = X.copy()
+    X2[:, 25:] = 0.5
+    a, b = gpu_fwd(X, wt, wc), gpu_fwd(X2, wt, wc)
+    assert np.abs(a[:, :25] - b[:, :25]).max() == 0.0
+    # position-offset invariance of latent RoPE
+    c = gpu_fwd(X, wt, wc, pos0=4096)
+    assert np.abs(a - c).max() < 2e-4
+
+
+# --------------------------------------------------------------------------------------
+# decode
+# --------------------------------------------------------------------------------------
+
+def run_decode(w, B, lens, Lmax, flags=0, append=True):
+    import torch
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    x, Kc, Vc, cache_len = W.make_decode_state(w, B=B, L=max(lens), Lmax=Lmax, cache_len=lens)
+    x, Kc, Vc = (W.round_to_storage(a, w.dtype) for a in (x, Kc, Vc))
+    ref_y, ref_k, ref_v = O.tucker_attn_decode(x, *[wt[k] for k in H.WEIGHT_KEYS], Kc, Vc, cache_len, rope=w.rope,
+                                               rope_base=w.rope_base)
+    dw = H.weights_to_device(wt, w.dtype)
+    Kd, Vd, xd = H.to_device(Kc, w.dtype), H.to_device(Vc, w.dtype), H.to_device(x, w.dtype)
+    ld = torch.from_numpy(cache_len).cuda()
+    y = Bd.tucker_attn_decode(xd, *dw, Kd, Vd, ld, n_H=w.n_H, rope=w.rope, rope_base=w.rope_base, append=append,
+                              flags=flags)
+    assert Bd.last_device_error() == 0
+    y = y.float().cpu().numpy().astype(np.float64)
+    return y, ref_y, (Kd, Vd, Kc, Vc, ref_k, ref_v, cache_len)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_decode_small_generic(dtype):
+    w = H.custom_workload(kind="decode", dtype=dtype, d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 20), rope=True, seed=17)
+    lens = [0, 1, 31, 32, 33, 100]
+    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, 6, lens, 128, flags=Bd.TA_FLAG_FORCE_GENERIC)
+    check(y, ref, dtype, "decode small")
+    tol = 1e-5 if dtype == "fp32" else 2e-2
+    Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
+    for b, L in enumerate(lens):
+        assert np.abs(Kh[b, L] - ref_k[b]).max() < tol and np.abs(Vh[b, L] - ref_v[b]).max() < tol
+        assert np.array_equal(Kh[b, :L], Kc[b, :L].astype(np.float32))        # old slots untouched
+        assert np.array_equal(Kh[b, L + 1:], Kc[b, L + 1:].astype(np.float32))
+
+
+def test_decode_no_append_leaves_cache():
+    w = H.custom_workload(kind="decode", dtype="fp32", d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), rope=True, seed=18)
+    y, ref, (Kd, Vd, Kc, Vc, *_r) = run_decode(w, 2, [5, 9], 16, append=False)
+    check(y, ref, "fp32", "decode no-append")
+    assert np.array_equal(Kd.cpu().numpy(), Kc.astype(np.float32))
+    assert np.array_equal(Vd.cpu().numpy(), Vc.astype(np.float32))
+
+
+def test_decode_bad_cache_len_is_flagged_not_fatal():
+    import torch
+    w = H.custom_workload(kind="decode", dtype="fp32", d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), rope=False, seed=19)
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    dw = H.weights_to_device(wt, "fp32")
+    Kd = torch.zeros(2, 8, 8, device="cuda")
+    Vd = torch.zeros(2, 8, 8, device="cuda")
+    xd = torch.randn(2, 32, device="cuda")
+    ld = torch.tensor([3, 8], dtype=torch.int32, device="cuda")        # 8 == Lmax: out of range
+    Bd.tucker_attn_decode(xd, *dw, Kd, Vd, ld, n_H=4, rope=False)
+    assert Bd.last_device_error() & Bd.TA_DEVERR_BAD_CACHE_LEN
+    assert Bd.last_device_error() == 0                                 # cleared by the read
+
+
+# --------------------------------------------------------------------------------------
+# benchmark-sized workloads, sampled
+# --------------------------------------------------------------------------------------
+
+def sample_rows(N, n, seed):
+    rng = np.random.default_rng(seed)
+    fixed = [r for r in (0, 1, 63, 64, 127, 128, 129, 255, 256, N // 2, N - 2, N - 1) if 0 <= r < N]
+    extra = rng.choice(N, size=min(n, N), replace=False).tolist()
+    return sorted(set(fixed + extra))[: n + len(fixed)]
+
+
+@pytest.mark.parametrize("name,nrows", [("c2", 96), ("c3", 197), ("c4", 40)])
+def test_full_size_prefill_sampled(name, nrows):
+    w = W.get_workload(name)
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w)
+    batches = sorted(set([0, w.B - 1, w.B // 2]))
+    rows = sample_rows(w.N, nrows, w.seed)
+    ref = oracle_fwd(X[batches], wt, w, rows=rows)
+    check(got[batches][:, rows], ref, w.dtype, name)
+
+
+def test_sharp_softmax_variant():
+    # pre-softmax core scaled by 8: peaky rows exercise the online rescaling
+    w = H.with_(W.get_workload("c2"), B=2)
+    X, wt = H.host_inputs(w, core_gain=8.0)
+    got = gpu_fwd(X, wt, w)
+    rows = sample_rows(w.N, 64, 5)
+    check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2")
+
+
+def test_full_size_decode_sampled():
+    # benchmark decode workload: 64 sequences, 32768 cached latent rows each, RoPE at position 32768
+    import torch
+    w = W.get_workload("c5")
+    L, Lmax, B = w.N, w.N + 1, w.B
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    dw = H.weights_to_device(wt, w.dtype)
+    x = W.round_to_storage(W.make_decode_x(w), w.dtype)
+    Kd = torch.zeros(B, Lmax, w.r[2], dtype=torch.bfloat16, device="cuda")
+    Vd = torch.zeros(B, Lmax, w.t[2], dtype=torch.bfloat16, device="cuda")
+    lens = np.full((B,), L, dtype=np.int32)
+    lens[5], lens[40] = 12345, 127            # ragged lengths inside the full-size launch
+    for b in range(B):
+        k, v = W.decode_cache_rows(w, b, int(lens[b]))
+        Kd[b, :lens[b]] = torch.from_numpy(k).to(torch.bfloat16).cuda()
+        Vd[b, :lens[b]] = torch.from_numpy(v).to(torch.bfloat16).cuda()
+    y = Bd.tucker_attn_decode(H.to_device(x, w.dtype), *dw, Kd, Vd, torch.from_numpy(lens).cuda(), n_H=w.n_H,
+                              rope=True, rope_base=w.rope_base, append=True)
+    assert Bd.last_device_error() == 0
+    y = y.float().cpu().numpy().astype(np.float64)
+    sample = [0, 5, 40, 63]
+    Kh = np.stack([Kd[b].float().cpu().numpy() for b in sample]).astype(np.float64)
+    Vh = np.stack([Vd[b].float().cpu().numpy() for b in sample]).astype(np.float64)
+    for i, b in enumerate(sample):        # slot L was appended by the call; the oracle must not see it
+        Kh[i, lens[b]:] = 0
+        Vh[i, lens[b]:] = 0
+    ref, ref_k, _ = O.tucker_attn_decode(x[sample], *[wt[k] for k in H.WEIGHT_KEYS], Kh, Vh, lens[sample], rope=True,
+                                         rope_base=w.rope_base)
+    check(y[sample], ref, w.dtype, "c5 decode")
+    got_k = np.stack([Kd[b, lens[b]].float().cpu().numpy() for b in sample])
+    assert np.abs(got_k - ref_k).max() < 3e-2
