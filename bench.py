@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the Tucker-attention forward library.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c2|c3|c5] [--impl reference]
+
+A step is one pass of the whole hot path (one tucker_attn_fwd or tucker_attn_decode call:
+core contraction, latent projections, per-head queries + latent RoPE, online-softmax
+attention, output-side factors) over one batch of seeded synthetic input.  One JSON line is
+printed by rank 0.  `value` is device-timed throughput with inputs resident in HBM; `e2e`
+times the same call with the step's input copied from pinned host memory and its output
+copied back inside the timed region.  With N > 1 (torchrun) every rank runs an independent
+replica of the workload (batch-sharded replicas, no collective on the data path) and the
+slowest rank sets the time.
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2603_30033_b200 import workloads as W
+
+METRIC = "prefill TFLOP/s & decode GB/s vs B200 roofline (fused Tucker attention)"
+KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                p = json.load(f)
+            return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------
+# GPU arms
+# ----------------------------------------------------------------------------------------
+
+def _dev(a, dtype, torch):
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+    return (t.to(torch.bfloat16) if dtype == "bf16" else t).cuda()
+
+
+class Flusher:
+    def __init__(self, torch, needed: bool):
+        self.buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if needed else None
+
+    def __call__(self):
+        if self.buf is not None:
+            self.buf.fill_(1)
+
+
+def time_steps(torch, Bd, step_fn, steps, warmup, flush, barrier):
+    """Runs warm-up, then `steps` timed steps.  Returns (per-step ms list, per-step dominant-kernel
+    ms list, wall interval)."""
+    for _ in range(warmup):
+        flush()
+        step_fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in kev:      # materialise the handles
+        a.record()
+        b.record()
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    for i in range(steps):
+        flush()
+        Bd.set_profile_events(*kev[i])
+        ev[i][0].record()
+        step_fn()
+        ev[i][1].record()
+    Bd.set_profile_events()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    barrier()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    kms = [a.elapsed_time(b) for a, b in kev]
+    return ms, kms, (t0, t1)
+
+
+def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=None):
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    dw = [_dev(wt[k], w.dtype, torch) for k in KEYS]
+    X32 = torch.from_numpy(W.make_X(w))
+    X_host = (X32.to(torch.bfloat16) if w.dtype == "bf16" else X32).contiguous().pin_memory()
+    del X32
+    X = X_host.cuda()
+    Y = torch.empty_like(X)
+    Y_host = torch.empty_like(X_host).pin_memory()
+    desc = Bd.make_desc(B=w.B, N=w.N, d_model=w.d_model, n_H=w.n_H, r=w.r, t=w.t, causal=w.causal, rope=w.rope,
+                        rope_base=w.rope_base, dtype=Bd.TA_DTYPE_BF16 if w.dtype == "bf16" else Bd.TA_DTYPE_F32)
+    ws = Bd.alloc_workspace(Bd.fwd_workspace_bytes(desc), X.device)
+    kw = dict(n_H=w.n_H, causal=w.causal, rope=w.rope, rope_base=w.rope_base, out=Y, workspace=ws)
+
+    def step():
+        Bd.tucker_attn_fwd(X, *dw, **kw)
+
+    in_bytes = X.numel() * X.element_size()
+    flush = Flusher(torch, needed=in_bytes < 2 * L2_BYTES)
+    if sampler:
+        sampler.start()
+    ms, kms, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    launches = Bd.last_launch_count()
+    path = Bd.last_path()
+    assert Bd.last_device_error() == 0, "device error word set during the benchmark"
+    fl = W.prefill_flops(w)
+    ms_step = sum(ms) / len(ms)
+    res = {
+        "workload": w.name, "unit": "TFLOP/s", "value": fl["total"] / (ms_step * 1e-3) / 1e12, "ms_per_step": ms_step,
+        "ms_best": min(ms), "flops_per_step": fl["total"], "gpu_launches_per_step": launches, "path": path,
+        "l2": "L2 flushed between steps" if flush.buf is not None else "inputs larger than L2",
+    }
+    kms_avg = sum(kms) / len(kms)
+    attn_flops = fl["scores"] + fl["pv"]
+    peak = peaks["bf16_tflops"] if w.dtype == "bf16" else None
+    ach = attn_flops / (kms_avg * 1e-3) / 1e12
+    res["roofline"] = {
+        "kernel": "attention (scores + online softmax + PV)", "bound": "tensor", "achieved": ach, "peak": peak,
+        "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": None, "kernel_ms": kms_avg,
+        "flops_per_launch": attn_flops, "whole_step_frac_of_peak": (res["value"] / peak) if peak else None,
+    }
+    res["clocks"] = clocks
+    if with_e2e:
+        def e2e_step():
+            X.copy_(X_host, non_blocking=True)
+            Bd.tucker_attn_fwd(X, *dw, **kw)
+            Y_host.copy_(Y, non_blocking=True)
+        ems, _, _ = time_steps(torch, Bd, e2e_step, steps, min(warmup, 3), Flusher(torch, False), barrier)
+        e_ms = sum(ems) / len(ems)
+        res["e2e"] = {"value": fl["total"] / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e_ms,
+                      "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": Y.numel() * Y.element_size()}
+    return res
+
+
+def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=None):
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    dw = [_dev(wt[k], w.dtype, torch) for k in KEYS]
+    L, Lmax, B = w.N, w.N + 1, w.B
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    Kc = torch.empty(B, Lmax, w.r[2], dtype=tdt, device="cuda")
+    Vc = torch.empty(B, Lmax, w.t[2], dtype=tdt, device="cuda")
+    for b in range(B):      # cache entries ~ N(0,1), drawn on the device one sequence at a time
+        Kc[b] = torch.randn(Lmax, w.r[2], generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+        Vc[b] = torch.randn(Lmax, w.t[2], generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+    x32 = torch.from_numpy(W.make_decode_x(w))
+    x_host = (x32.to(tdt)).contiguous().pin_memory()
+    x = x_host.cuda()
+    y = torch.empty_like(x)
+    y_host = torch.empty_like(x_host).pin_memory()
+    lens = torch.full((B,), L, dtype=torch.int32, device="cuda")
+    desc = Bd.make_desc(B=B, N=1, d_model=w.d_model, n_H=w.n_H, r=w.r, t=w.t, causal=True, rope=w.rope,
+                        rope_base=w.rope_base, dtype=Bd.TA_DTYPE_BF16 if w.dtype == "bf16" else Bd.TA_DTYPE_F32)
+    ws = Bd.alloc_workspace(Bd.decode_workspace_bytes(desc, Lmax), x.device)
+    kw = dict(n_H=w.n_H, rope=w.rope, rope_base=w.rope_base, append=True, out=y, workspace=ws)
+
+    def step():
+        Bd.tucker_attn_decode(x, *dw, Kc, Vc, lens, **kw)
+
+    by = W.decode_bytes(w)
+    flush = Flusher(torch, needed=by["total"] < 2 * L2_BYTES)
+    if sampler:
+        sampler.start()
+    ms, kms, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    launches, path = Bd.last_launch_count(), Bd.last_path()
+    assert Bd.last_device_error() == 0, "device error word set during the benchmark"
+    ms_step = sum(ms) / len(ms)
+    res = {
+        "workload": w.name, "unit": "GB/s", "value": by["total"] / (ms_step * 1e-3) / 1e9, "ms_per_step": ms_step,
+        "ms_best": min(ms), "bytes_per_step": by["total"], "gpu_launches_per_step": launches, "path": path,
+        "l2": "L2 flushed between steps" if flush.buf is not None else "inputs larger than L2",
+    }
+    kms_avg = sum(kms) / len(kms)
+    ach = by["cache"] / (kms_avg * 1e-3) / 1e9
+    res["roofline"] = {
+        "kernel": "decode attention over the latent KV cache", "bound": "hbm", "achieved": ach,
+        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+        "kernel_ms": kms_avg, "bytes_per_launch": by["cache"],
+        "whole_step_frac_of_peak": res["value"] / peaks["hbm_gbs"],
+    }
+    res["clocks"] = clocks
+    if with_e2e:
+        def e2e_step():
+            x.copy_(x_host, non_blocking=True)
+            Bd.tucker_attn_decode(x, *dw, Kc, Vc, lens, **kw)
+            y_host.copy_(y, non_blocking=True)
+        ems, _, _ = time_steps(torch, Bd, e2e_step, steps, min(warmup, 3), flush, barrier)
+        e_ms = sum(ems) / len(ems)
+        res["e2e"] = {"value": by["total"] / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e_ms,
+                      "h2d_bytes_per_step": x.numel() * x.element_size(),
+                      "d2h_bytes_per_step": y.numel() * y.element_size(),
+                      "note": "the latent KV cache is layer state and stays resident in HBM"}
+    return res
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle arm (bounded sample)
+# ----------------------------------------------------------------------------------------
+
+def oracle_sample(w, budget="default"):
+    """Returns (callable running the oracle on a bounded sample, work in the metric's unit
+    numerator, description, unit)."""
+    from oracle import tucker_oracle as O
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    args = [wt[k] for k in KEYS]
+    if w.kind == "prefill":
+        nrows = {"c4_long_prefill": 256, "c2_gpt2_prefill": 1024, "c3_vit_prefill": 197}.get(w.name, min(w.N, 256))
+        nseq = {"c3_vit_prefill": 8}.get(w.name, 1)
+        rows = sorted(set(np.linspace(0, w.N - 1, nrows).astype(int).tolist()))
+        X = W.round_to_storage(W.make_X(w, B=nseq), w.dtype)
+        r1, r2, r3 = w.r
+        t1, t2, t3 = w.t
+        pairs = sum((r + 1) if w.causal else w.N for r in rows)
+        flops = nseq * (2 * w.N * w.d_model * (r2 + r3 + t3) + 2 * w.n_H * pairs * (r3 + t3)
+                        + len(rows) * (2 * w.n_H * (r2 * r3 + t3 * t2) + 2 * t2 * w.d_model)) \
+            + 2 * w.n_H * (r1 * r2 * r3 + t1 * t2 * t3)
+
+        def run():
+            return O.tucker_attn_fwd(X, *args, causal=w.causal, rope=w.rope, rope_base=w.rope_base, rows=rows)
+        desc = (f"{nseq} of {w.B} sequences, projections for all {w.N} tokens, attention and output for "
+                f"{len(rows)} evenly spaced query rows per sequence")
+        return run, flops / 1e12, desc, "TFLOP/s"
+    nseq = 4
+    L = w.N
+    x = W.round_to_storage(W.make_decode_x(w, B=nseq), w.dtype)
+    Kc = np.zeros((nseq, L + 1, w.r[2]))
+    Vc = np.zeros((nseq, L + 1, w.t[2]))
+    for b in range(nseq):
+        k, v = W.decode_cache_rows(w, b, L)
+        Kc[b, :L], Vc[b, :L] = W.round_to_storage(k, w.dtype), W.round_to_storage(v, w.dtype)
+    lens = np.full((nseq,), L, dtype=np.int32)
+    by = W.decode_bytes(w, B=nseq)
+
+    def run():
+        return O.tucker_attn_decode(x, *args, Kc, Vc, lens, rope=w.rope, rope_base=w.rope_base)
+    return run, by["total"] / 1e9, f"{nseq} of {w.B} sequences with the full {L}-entry cache", "GB/s"
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(w, steps=1, warmup=0):
+    run, work, desc, unit = oracle_sample(w)
+    for _ in range(warmup):
+        run()
+    ts = []
+    for _ in range(steps):
+        t = time.perf_counter()
+        run()
+        ts.append(time.perf_counter() - t)
+    sec = sum(ts) / len(ts)
+    return {"value": work / sec, "unit": unit, "cores": oracle_threads(), "kind": "oracle", "sample": desc,
+            "seconds_per_sample": sec}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    w = W.get_workload(args.workload)
+    cb = time_oracle(w, steps=max(1, args.steps), warmup=min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": cb["value"], "unit": cb["unit"], "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": cb["seconds_per_sample"] * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, **_cfg(w)}, "cpu_baseline": cb,
+        "e2e": {"value": cb["value"], "unit": cb["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def _cfg(w):
+    return {"kind": w.kind, "B": w.B, "N_or_cache_len": w.N, "d_model": w.d_model, "n_H": w.n_H,
+            "ranks_qk": list(w.r), "ranks_vo": list(w.t), "causal": w.causal, "rope": w.rope,
+            "rope_base": w.rope_base, "storage": w.dtype}
+
+
+# ----------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-others", action="store_true", help="skip the secondary workloads")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2603_30033_b200 import binding as Bd
+    Bd.load_library()          # raises if the CUDA library is missing: there is no fallback
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    peaks, peak_kind = load_peaks()
+    w = W.get_workload(args.workload)
+    fn = bench_prefill if w.kind == "prefill" else bench_decode
+    gpu_index = local_rank
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            gpu_index = int(vis.split(",")[local_rank])
+        except Exception:
+            gpu_index = local_rank
+    res = fn(w, args.steps, args.warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=ClockSampler(gpu_index))
+
+    ms = res["ms_per_step"]
+    e2e_ms = res["e2e"]["ms_per_step"]
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    work = res.get("flops_per_step", res.get("bytes_per_step"))
+    div = 1e12 if w.kind == "prefill" else 1e9
+    value = world * work / (ms * 1e-3) / div
+    e2e_value = world * work / (e2e_ms * 1e-3) / div
+
+    others = []
+    if not args.no_others and world == 1:
+        for name in ("c2", "c3", "c4", "c5"):
+            ow = W.get_workload(name)
+            if ow.name == w.name:
+                continue
+            torch.cuda.empty_cache()
+            ofn = bench_prefill if ow.kind == "prefill" else bench_decode
+            o = ofn(ow, max(5, min(args.steps, 20)), 3, torch, Bd, barrier, peaks, with_e2e=False)
+            o.pop("clocks", None)
+            others.append(o)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(w)
+
+    if rank == 0:
+        res["roofline"]["peak_source"] = f"{peak_kind} ({'burst' if w.kind == 'prefill' else 'copy'})"
+        line = {
+            "metric": METRIC, "value": value, "unit": res["unit"], "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, **_cfg(w), "l2": res["l2"],
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "roofline": res["roofline"], "cpu_baseline": cpu_baseline, "clocks": res["clocks"],
+            "e2e": {**res["e2e"], "value": e2e_value, "ms_per_step": e2e_ms},
+            "gpu_launches": res["gpu_launches_per_step"] * args.steps, "path": res["path"],
+            "ms_best": res["ms_best"], "other_workloads": others,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
