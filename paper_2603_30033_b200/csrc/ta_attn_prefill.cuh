@@ -1,0 +1,300 @@
+// Flash-style attention over the latent K / V pair on tcgen05 tensor cores (Sec. 3.3 of the
+// paper: online softmax over key chunks, one K/V chunk pair shared by all heads).
+//
+// One CTA handles one work item = (sequence b, 128 query rows, a pair of heads h, h+1).  Both
+// heads use the same latent K / V tiles, so every tile is loaded once and serves two score
+// tiles; the two softmax warpgroups ping-pong so that the tensor core works on one head
+// while the other head's scores are being exponentiated.
+//
+//   warp 0        TMA producer: Qhat tiles (once), K ring, V ring
+//   warp 1        MMA issuer:  S_i = Qhat_i K^T (smem x smem), O_i += P_i V (P from TMEM)
+//   warps 4..7    softmax for head h   : thread t owns query row t (TMEM lane t)
+//   warps 8..11   softmax for head h+1
+//
+// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,256+t3) O_1 [384,384+t3); P_i (bf16, two
+// per column) overwrites the first 64 columns of S_i once the row has been read.
+// Scores arrive in log2 units (softmax scale * log2 e is folded into G_h), so exp2 is used.
+// The running maximum is only raised when it grows by more than 8 (factor 256), which keeps
+// the O rescaling off the common path; l and O stay consistent because both use the same
+// stale maximum.
+#pragma once
+
+#include "ta_common.cuh"
+#include "ta_sm100.cuh"
+
+namespace ta {
+namespace attn {
+
+using namespace sm100;
+
+constexpr int BQ = 128;        // query rows per tile
+constexpr int BKV = 128;       // keys per tile
+constexpr int THREADS = 384;
+constexpr int SUB_BYTES = 128 * 64 * 2;   // one [128 x 64] bf16 sub-tile (128-byte rows)
+constexpr int MAX_SUB = 2;                 // r3, t3 <= 128
+constexpr int KV_STAGES = 2;
+constexpr float kRescaleThreshold = 8.f;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)(2 * MAX_SUB + 2 * KV_STAGES * MAX_SUB) * SUB_BYTES;
+
+struct Params {
+  int B, N, nH, r3, t3;
+  int causal;
+  int n_qt;          // query tiles per sequence
+  int n_hp;          // head pairs
+  bf16* O;           // [B, N, nH, t3]
+  unsigned int* err;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// MN-major B operand (V tile as loaded: rows = keys, 64-column blocks), 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint32_t block_pitch_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(block_pitch_bytes >> 4) << 16;   // leading offset: next 64-column block
+  d |= (uint64_t)(1024u >> 4) << 32;               // stride offset: next group of 8 key rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
+  __shared__ uint64_t s_full[2], p_full[2], o_full[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
+  uint8_t* q_tile[2] = {tiles, tiles + MAX_SUB * SUB_BYTES};
+  uint8_t* k_ring = tiles + 2 * MAX_SUB * SUB_BYTES;
+  uint8_t* v_ring = k_ring + KV_STAGES * MAX_SUB * SUB_BYTES;
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  // work item: heaviest (largest query tile) first
+  int item = blockIdx.x;
+  const int hp = item % p.n_hp; item /= p.n_hp;
+  const int b = item % p.B; item /= p.B;
+  const int qt = p.n_qt - 1 - item;
+  const int q0 = qt * BQ;
+  const int h0 = hp * 2;
+  const bool two = (h0 + 1) < p.nH;
+  const int n_kt_all = (p.N + BKV - 1) / BKV;
+  const int nt = p.causal ? min(n_kt_all, qt + 1) : n_kt_all;
+  const int ksub = (p.r3 + 63) / 64, vsub = (p.t3 + 63) / 64;
+  Abort ab{&abort_flag, p.err};
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&q_full, 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s_full[i], 1);
+      mbar_init(&p_full[i], 4);     // one arrival per softmax warp
+      mbar_init(&o_full[i], 1);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  const uint32_t tm_s[2] = {tmem, tmem + 128};
+  const uint32_t tm_o[2] = {tmem + 256, tmem + 384};
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (elect_one()) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      mbar_expect_tx(&q_full, (uint32_t)((two ? 2 : 1) * ksub * SUB_BYTES));
+      for (int i = 0; i < (two ? 2 : 1); ++i)
+        for (int kk = 0; kk < ksub; ++kk)
+          tma_load_3d(q_tile[i] + kk * SUB_BYTES, &tmQ, &q_full, (h0 + i) * p.r3 + kk * 64, q0, b);
+      for (int j = 0; j < nt; ++j) {
+        const int s = j % KV_STAGES;
+        const uint32_t ph = (j / KV_STAGES) & 1;
+        if (!mbar_wait(&k_empty[s], ph ^ 1, ab)) break;
+        mbar_expect_tx(&k_full[s], (uint32_t)(ksub * SUB_BYTES));
+        for (int kk = 0; kk < ksub; ++kk)
+          tma_load_3d(k_ring + (s * MAX_SUB + kk) * SUB_BYTES, &tmK, &k_full[s], kk * 64, j * BKV, b);
+        if (!mbar_wait(&v_empty[s], ph ^ 1, ab)) break;
+        mbar_expect_tx(&v_full[s], (uint32_t)(vsub * SUB_BYTES));
+        for (int kk = 0; kk < vsub; ++kk)
+          tma_load_3d(v_ring + (s * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[s], kk * 64, j * BKV, b);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------
+    if (elect_one()) {
+      const uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV);
+      const uint32_t idesc_pv = umma_idesc_bf16(BQ, (uint32_t)p.t3) | (1u << 16);   // B = V is MN-major
+      const int ksteps = p.r3 / 16;
+      const int nh = two ? 2 : 1;
+      auto issue_qk = [&](int i, int s) {
+        const uint32_t qa = smem_u32(q_tile[i]), ka = smem_u32(k_ring + s * MAX_SUB * SUB_BYTES);
+        for (int ks = 0; ks < ksteps; ++ks) {
+          const uint32_t off = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
+          umma_ss(tm_s[i], umma_desc_kmajor_sw128(qa + off), umma_desc_kmajor_sw128(ka + off), idesc_qk, ks != 0);
+        }
+        umma_commit(&s_full[i]);
+      };
+      auto issue_pv = [&](int i, int s, int j) {
+        const uint32_t va = smem_u32(v_ring + s * MAX_SUB * SUB_BYTES);
+        for (int ks = 0; ks < BKV / 16; ++ks)
+          umma_ts(tm_o[i], tm_s[i] + (uint32_t)ks * 8, umma_desc_mnmajor_sw128(va + (uint32_t)ks * 2048, SUB_BYTES),
+                  idesc_pv, (j | ks) != 0);
+        umma_commit(&o_full[i]);
+      };
+      bool ok = mbar_wait(&q_full, 0, ab);
+      if (ok) ok = mbar_wait(&k_full[0], 0, ab);
+      if (ok) {
+        tc_fence_after();
+        for (int i = 0; i < nh; ++i) issue_qk(i, 0);
+        umma_commit(&k_empty[0]);
+      }
+      for (int j = 0; j < nt && ok; ++j) {
+        const int s = j % KV_STAGES;
+        const uint32_t ph = (j / KV_STAGES) & 1;
+        const int s1 = (j + 1) % KV_STAGES;
+        const uint32_t ph1 = ((j + 1) / KV_STAGES) & 1;
+        const bool more = (j + 1) < nt;
+        if (!(ok = mbar_wait(&v_full[s], ph, ab))) break;
+        for (int i = 0; i < nh && ok; ++i) {
+          if (!(ok = mbar_wait(&p_full[i], (uint32_t)(j & 1), ab))) break;
+          tc_fence_after();
+          issue_pv(i, s, j);
+          if (i == nh - 1) umma_commit(&v_empty[s]);
+          if (more) {
+            if (i == 0) {
+              if (!(ok = mbar_wait(&k_full[s1], ph1, ab))) break;
+              tc_fence_after();
+            }
+            issue_qk(i, s1);
+            if (i == nh - 1) umma_commit(&k_empty[s1]);
+          }
+        }
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------- softmax / correction / epilogue -------------
+    const int i = (warp - 4) / 4;              // which head of the pair
+    const int q = warp % 4;                    // TMEM lane quadrant
+    if (i == 0 || two) {
+      const int row = q0 + q * 32 + lane;      // query row inside the sequence
+      const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+      float m_used = -INFINITY, l = 0.f;
+      bool ok = true;
+      for (int j = 0; j < nt; ++j) {
+        ok = mbar_wait(&s_full[i], (uint32_t)(j & 1), ab);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sr[128];
+        {
+          uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(sr);
+          tmem_ld32(tm_s[i] + lane_addr + 0, c[0]);
+          tmem_ld32(tm_s[i] + lane_addr + 32, c[1]);
+          tmem_ld32(tm_s[i] + lane_addr + 64, c[2]);
+          tmem_ld32(tm_s[i] + lane_addr + 96, c[3]);
+          tmem_ld_wait();
+        }
+        const int k0 = j * BKV;
+        const bool need_mask = (p.causal && (k0 + BKV - 1 > q0)) || (k0 + BKV > p.N);
+        if (need_mask) {
+          const int lim = p.causal ? min(row, p.N - 1) : (p.N - 1);   // last visible key index
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (k0 + c > lim) sr[c] = 0xff800000u;   // -inf
+        }
+        float mt = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; ++c) mt = fmaxf(mt, __uint_as_float(sr[c]));
+        const bool need = (mt > m_used + kRescaleThreshold) && (mt > -INFINITY);
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? mt : m_used;
+          const float factor = need ? fast_exp2(m_used - m_new) : 1.f;   // exp2(-inf) = 0 on the first tile
+          if (j > 0) {
+            ok = mbar_wait(&o_full[i], (uint32_t)((j - 1) & 1), ab);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            for (int ch = 0; ch < p.t3 / 32; ++ch) {
+              uint32_t o[32];
+              tmem_ld32(tm_o[i] + lane_addr + ch * 32, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+              tmem_st32(tm_o[i] + lane_addr + ch * 32, o);
+            }
+          }
+          l *= factor;
+          m_used = m_new;
+        }
+        float rs = 0.f;
+        uint32_t pk[64];
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p0 = fast_exp2(__uint_as_float(sr[2 * c]) - m_used);
+          const float p1 = fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_used);
+          rs += p0 + p1;
+          pk[c] = pack_bf16(p0, p1);
+        }
+        l += rs;
+        {
+          uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(pk);
+          tmem_st32(tm_s[i] + lane_addr + 0, c[0]);
+          tmem_st32(tm_s[i] + lane_addr + 32, c[1]);
+          tmem_st_wait();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[i]);
+      }
+      if (ok) {
+        ok = mbar_wait(&o_full[i], (uint32_t)((nt - 1) & 1), ab);
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l;
+        bf16* dst = p.O + (((long)b * p.N + row) * p.nH + (h0 + i)) * p.t3;
+        for (int ch = 0; ch < p.t3 / 32; ++ch) {
+          uint32_t o[32];
+          tmem_ld32(tm_o[i] + lane_addr + ch * 32, o);
+          tmem_ld_wait();
+          if (row < p.N) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst + ch * 32);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
+              d4[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace attn
+}  // namespace ta

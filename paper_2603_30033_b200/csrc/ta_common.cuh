@@ -57,6 +57,8 @@ size_t generic_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
 int generic_fwd(Problem& p);
 int generic_decode(Problem& p);
 
+int simt_attention_bf16(Problem& p, const bf16* Qhat, const bf16* K, const bf16* V, bf16* O);
+
 // tensor-core path (bf16 storage): returns false from *_supported when the shape is outside
 // what the kernels were built for, in which case the generic path runs.
 bool fast_fwd_supported(const tucker_attn_desc& d);

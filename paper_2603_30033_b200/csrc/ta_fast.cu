@@ -1,0 +1,297 @@
+// Tensor-core path for bf16 storage: weight preparation, tcgen05 GEMMs for the latent
+// projections / per-head queries / output side, and the attention kernel.
+//
+//   prep      G_h (scaled by softmax scale * log2 e) and Gt_h from the cores (C x_1 U1, Definition 2),
+//             stored as K-major B operands; transposed copies of U2, U3, Ut3; RoPE cos/sin table
+//   proj      [Qt | K | V] = X [U2 | U3 | Ut3]   (Sec. 3.1), latent RoPE applied to K in the epilogue
+//   qhat      Qhat[T, (h, c)] = Qt [G_1 | ... | G_nH], latent RoPE per head in the epilogue (Eq. 9)
+//   attention online softmax over key tiles, one shared latent K / V pair for all heads (Sec. 3.3)
+//   z, y      Z = O [Gt_1; ...; Gt_nH]^T,  Y = Z Ut2^T   (Eqs. 5-6)
+#include "ta_common.cuh"
+#include "ta_umma_gemm.cuh"
+
+#include <math.h>
+
+namespace ta {
+namespace {
+
+// ---- driver entry point for tensor-map creation (no link-time dependency on libcuda) --------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 tensor of up to 3 dims; dims[0] is innermost (contiguous); strides in elements for dims 1..rank-1.
+bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_elems,
+               const uint32_t* box, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3], gstr[2];
+  cuuint32_t bx[3], es[3];
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_elems[i] * 2;
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool tmap_2d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t ld, uint32_t box_cols,
+             uint32_t box_rows) {
+  uint64_t dims[2] = {cols, rows}, str[1] = {ld};
+  uint32_t box[2] = {box_cols, box_rows};
+  return make_tmap(m, base, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// ---- weight preparation -------------------------------------------------------------------
+// out[(h*sh + b*sb + c*sc)] = bf16(mult * sum_a U1[h,a] C[a,b,c])
+__global__ void k_head_core_bf16(const bf16* __restrict__ C, const bf16* __restrict__ U1, bf16* __restrict__ out,
+                                 int nH, int r1, int rb, int rc, long sh, long sb, long sc, float mult) {
+  long total = (long)nH * rb * rc;
+  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    int c = (int)(i % rc);
+    int b = (int)((i / rc) % rb);
+    int h = (int)(i / ((long)rc * rb));
+    float acc = 0.f;
+    for (int a = 0; a < r1; ++a)
+      acc = fmaf(__bfloat162float(U1[(long)h * r1 + a]), __bfloat162float(C[((long)a * rb + b) * rc + c]), acc);
+    out[h * sh + b * sb + c * sc] = __float2bfloat16_rn(acc * mult);
+  }
+}
+
+// dst[c, r] = src[r, c] for src [rows, cols]; 32x32 tiles through shared memory.
+__global__ void k_transpose_bf16(const bf16* __restrict__ src, bf16* __restrict__ dst, int rows, int cols) {
+  __shared__ bf16 t[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    int r = r0 + i, c = c0 + threadIdx.x;
+    if (r < rows && c < cols) t[i][threadIdx.x] = src[(long)r * cols + c];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    int c = c0 + i, r = r0 + threadIdx.x;
+    if (r < rows && c < cols) dst[(long)c * rows + r] = t[threadIdx.x][i];
+  }
+}
+
+__global__ void k_rope_table_f(float2* __restrict__ tab, int n_pos, int half, int r, int pos0, double base) {
+  long total = (long)n_pos * half;
+  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    int c = (int)(i % half);
+    int n = (int)(i / half);
+    double theta = pow(base, -2.0 * (double)c / (double)r);
+    double s, co;
+    sincos((double)(pos0 + n) * theta, &s, &co);
+    tab[i] = make_float2((float)co, (float)s);
+  }
+}
+
+int grid_for(long total, int block = 256) {
+  long g = (total + block - 1) / block;
+  if (g > 148L * 8) g = 148L * 8;
+  return (int)(g < 1 ? 1 : g);
+}
+
+// ---- workspace ----------------------------------------------------------------------------
+struct FastWs {
+  float2* rope;   // [N][r3/2]
+  bf16* Wt;       // [r2 + r3 + t3, d]   transposed U2 | U3 | Ut3 (K-major B operand)
+  bf16* GcatT;    // [n_H * r3, r2]      B operand of the per-head query GEMM
+  bf16* GtP;      // [t2, n_H * t3]      B operand of the Z GEMM
+  bf16* Qt;       // [T, r2]
+  bf16* K;        // [T, r3]  rotated
+  bf16* V;        // [T, t3]
+  bf16* Qhat;     // [T, n_H * r3]
+  bf16* O;        // [T, n_H * t3]
+  bf16* Z;        // [T, t2]
+};
+
+size_t carve_fast(const tucker_attn_desc& d, char* base, FastWs* w) {
+  Carver c(base);
+  const size_t T = (size_t)d.B * d.N;
+  FastWs t;
+  t.rope = c.take<float2>(d.rope ? (size_t)d.N * (d.r3 / 2) : 0);
+  t.Wt = c.take<bf16>((size_t)(d.r2 + d.r3 + d.t3) * d.d_model);
+  t.GcatT = c.take<bf16>((size_t)d.n_H * d.r3 * d.r2);
+  t.GtP = c.take<bf16>((size_t)d.t2 * d.n_H * d.t3);
+  t.Qt = c.take<bf16>(T * d.r2);
+  t.K = c.take<bf16>(T * d.r3);
+  t.V = c.take<bf16>(T * d.t3);
+  t.Qhat = c.take<bf16>(T * d.n_H * d.r3);
+  t.O = c.take<bf16>(T * d.n_H * d.t3);
+  t.Z = c.take<bf16>(T * d.t2);
+  if (w) *w = t;
+  return c.off;
+}
+
+int pick_bn(int width) {
+  if (width % 128 == 0) return 128;
+  if (width % 96 == 0) return 96;
+  if (width % 64 == 0) return 64;
+  return 32;
+}
+
+// C[M, sum(widths)] = A[M, K] * B^T with B [Ntot, K] K-major (or [K, Ntot] when b_mn_major).
+int launch_gemm(Problem& p, const bf16* A, long lda, const bf16* Bm, long ldb, int M, int K, int Ntot, int BN,
+                umma_gemm::Params gp) {
+  CUtensorMap tmA, tmB;
+  if (!tmap_2d(&tmA, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, 128)) return TA_ERR_CUDA;
+  if (!gp.b_mn_major) {
+    if (!tmap_2d(&tmB, Bm, (uint64_t)K, (uint64_t)Ntot, (uint64_t)ldb, 64, (uint32_t)BN)) return TA_ERR_CUDA;
+  } else {
+    if (!tmap_2d(&tmB, Bm, (uint64_t)Ntot, (uint64_t)K, (uint64_t)ldb, 64, 64)) return TA_ERR_CUDA;
+  }
+  gp.M = M; gp.K = K; gp.BN = BN; gp.err = p.dev_err;
+  static bool attr_set = false;
+  if (!attr_set) {
+    TA_CUDA_TRY(cudaFuncSetAttribute(umma_gemm::k_umma_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)umma_gemm::SMEM_BYTES));
+    attr_set = true;
+  }
+  dim3 grid(Ntot / BN, (M + 127) / 128);
+  umma_gemm::k_umma_gemm<<<grid, umma_gemm::THREADS, umma_gemm::SMEM_BYTES, p.stream>>>(tmA, tmB, gp);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
+
+umma_gemm::Seg seg(int n_begin, int width, int mode, void* out, long ld) {
+  umma_gemm::Seg s;
+  s.n_begin = n_begin; s.width = width; s.mode = mode; s.out = out; s.ld = ld;
+  s.out2 = nullptr; s.ld2 = 0; s.batch2 = 0;
+  return s;
+}
+
+}  // namespace
+
+bool fast_fwd_supported(const tucker_attn_desc& d) {
+  auto ok32 = [](int r) { return r >= 32 && r <= 256 && r % 32 == 0; };
+  if (!ok32(d.r2) || !ok32(d.r3) || !ok32(d.t2) || !ok32(d.t3)) return false;
+  if (d.d_model % 64) return false;
+  if ((long)d.B * d.N >= (1L << 24)) return false;
+  return true;
+}
+
+size_t fast_fwd_workspace(const tucker_attn_desc& d) { return carve_fast(d, nullptr, nullptr); }
+
+int fast_fwd(Problem& p) {
+  const tucker_attn_desc& d = p.d;
+  FastWs w;
+  carve_fast(d, p.ws, &w);
+  const int T = d.B * d.N;
+  const bool mn = (d.flags & 0x100) != 0;   // bring-up switch: feed U2/U3/Ut3 untransposed (MN-major B)
+  const float LOG2E = 1.4426950408889634f;
+
+  // ---- weight preparation ----
+  k_head_core_bf16<<<grid_for((long)d.n_H * d.r2 * d.r3), 256, 0, p.stream>>>(
+      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, p.scale);
+  TA_LAUNCH_CHECK(p);
+  k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
+      (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
+  TA_LAUNCH_CHECK(p);
+  (void)LOG2E;
+  if (!mn) {
+    const bf16* srcs[3] = {(const bf16*)p.U2, (const bf16*)p.U3, (const bf16*)p.Ut3};
+    const int widths[3] = {d.r2, d.r3, d.t3};
+    long off = 0;
+    for (int i = 0; i < 3; ++i) {
+      dim3 grid((widths[i] + 31) / 32, (d.d_model + 31) / 32);
+      k_transpose_bf16<<<grid, dim3(32, 8), 0, p.stream>>>(srcs[i], w.Wt + off * d.d_model, d.d_model, widths[i]);
+      TA_LAUNCH_CHECK(p);
+      off += widths[i];
+    }
+  }
+  if (d.rope) {
+    k_rope_table_f<<<grid_for((long)d.N * (d.r3 / 2)), 256, 0, p.stream>>>(w.rope, d.N, d.r3 / 2, d.r3, d.pos0,
+                                                                          (double)d.rope_base);
+    TA_LAUNCH_CHECK(p);
+  }
+
+  int rc;
+  // ---- latent projections ----
+  {
+    umma_gemm::Params gp = {};
+    gp.rope_tab = w.rope; gp.n_pos = d.N; gp.rope_half = d.r3 / 2;
+    const int kmode = d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16;
+    if (!mn) {
+      int bn = pick_bn(d.r2);
+      if (pick_bn(d.r3) < bn) bn = pick_bn(d.r3);
+      if (pick_bn(d.t3) < bn) bn = pick_bn(d.t3);
+      if (d.r2 % bn || d.r3 % bn || d.t3 % bn) bn = 32;
+      gp.nseg = 3;
+      gp.seg[0] = seg(0, d.r2, umma_gemm::EP_BF16, w.Qt, d.r2);
+      gp.seg[1] = seg(d.r2, d.r3, kmode, w.K, d.r3);
+      gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_BF16, w.V, d.t3);
+      if (p.Kc) {
+        gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3;
+        gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
+      }
+      if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, w.Wt, d.d_model, T, d.d_model, d.r2 + d.r3 + d.t3, bn, gp)))
+        return rc;
+    } else {
+      // one launch per factor, B read in place as [d, r] (MN-major)
+      struct { const void* U; int width; int mode; bf16* out; void* out2; } job[3] = {
+          {p.U2, d.r2, umma_gemm::EP_BF16, w.Qt, nullptr},
+          {p.U3, d.r3, kmode, w.K, p.Kc},
+          {p.Ut3, d.t3, umma_gemm::EP_BF16, w.V, p.Vc}};
+      for (int i = 0; i < 3; ++i) {
+        umma_gemm::Params g2 = gp;
+        g2.b_mn_major = 1;
+        g2.nseg = 1;
+        g2.seg[0] = seg(0, job[i].width, job[i].mode, job[i].out, job[i].width);
+        if (job[i].out2) {
+          g2.seg[0].out2 = job[i].out2; g2.seg[0].ld2 = job[i].width; g2.seg[0].batch2 = (long)p.Lmax * job[i].width;
+        }
+        const int bn = job[i].width % 128 == 0 ? 128 : 64;
+        if (job[i].width % 64) return TA_ERR_UNSUPPORTED_SHAPE;
+        if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, (const bf16*)job[i].U, job[i].width, T, d.d_model,
+                              job[i].width, bn, g2)))
+          return rc;
+      }
+    }
+  }
+  // ---- per-head queries with latent RoPE ----
+  {
+    umma_gemm::Params gp = {};
+    gp.rope_tab = w.rope; gp.n_pos = d.N; gp.rope_half = d.r3 / 2;
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, d.n_H * d.r3, d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16, w.Qhat, (long)d.n_H * d.r3);
+    if ((rc = launch_gemm(p, w.Qt, d.r2, w.GcatT, d.r2, T, d.r2, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
+  }
+  // ---- attention ----
+  if ((rc = simt_attention_bf16(p, w.Qhat, w.K, w.V, w.O))) return rc;
+  // ---- output side ----
+  {
+    umma_gemm::Params gp = {};
+    gp.n_pos = d.N;
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, d.t2, umma_gemm::EP_BF16, w.Z, d.t2);
+    if ((rc = launch_gemm(p, w.O, (long)d.n_H * d.t3, w.GtP, (long)d.n_H * d.t3, T, d.n_H * d.t3, d.t2, pick_bn(d.t2), gp)))
+      return rc;
+  }
+  {
+    umma_gemm::Params gp = {};
+    gp.n_pos = d.N;
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
+    if ((rc = launch_gemm(p, w.Z, d.t2, (const bf16*)p.Ut2, d.t2, T, d.t2, d.d_model, pick_bn(d.d_model), gp))) return rc;
+  }
+  return TA_OK;
+}
+
+bool fast_decode_supported(const tucker_attn_desc&, int32_t) { return false; }
+size_t fast_decode_workspace(const tucker_attn_desc&, int32_t) { return 0; }
+int fast_decode(Problem&) { return TA_ERR_UNSUPPORTED_SHAPE; }
+
+}  // namespace ta

@@ -237,10 +237,13 @@ __device__ __forceinline__ void attend_tile(WarpState& st, const float* __restri
   }
 }
 
-__global__ void __launch_bounds__(256) k_attn_prefill_generic(const float* __restrict__ Qhat,
-                                                              const float* __restrict__ K,
-                                                              const float* __restrict__ V, float* __restrict__ O,
-                                                              int N, int nH, int r3, int t3, int causal) {
+// Element (b, h, row, c) of Qhat is at b*q_b + h*q_h + row*q_n + c; K / V rows (b, n) start at
+// b*kv_b + n*r3 (n*t3); O element (b, row, h, c) is at ((b*N + row)*nH + h)*t3 + c.
+template <typename TI, typename TO>
+__global__ void __launch_bounds__(256) k_attn_prefill_generic(const TI* __restrict__ Qhat, long q_b, long q_h, long q_n,
+                                                              const TI* __restrict__ K, const TI* __restrict__ V,
+                                                              long k_b, long v_b, TO* __restrict__ O, int N, int nH,
+                                                              int r3, int t3, int causal) {
   extern __shared__ float smem[];
   float* qs = smem;                      // [8][r3]
   float* Ks = qs + 8 * r3;               // [32][r3+1]
@@ -249,36 +252,39 @@ __global__ void __launch_bounds__(256) k_attn_prefill_generic(const float* __res
   const int row0 = blockIdx.x * 8, h = blockIdx.y, b = blockIdx.z;
   const int row = row0 + warp;
   const bool valid = row < N;
-  const float* qg = Qhat + (((long)b * nH + h) * N + row0) * r3;
-  for (int i = threadIdx.x; i < 8 * r3; i += 256) qs[i] = (row0 + i / r3 < N) ? qg[i] : 0.f;
+  const TI* qg = Qhat + (long)b * q_b + (long)h * q_h;
+  for (int i = threadIdx.x; i < 8 * r3; i += 256) {
+    int rr = i / r3, c = i % r3;
+    qs[i] = (row0 + rr < N) ? ld(qg + (long)(row0 + rr) * q_n + c) : 0.f;
+  }
   WarpState stt;
   stt.m = -INFINITY; stt.l = 0.f;
 #pragma unroll
   for (int i = 0; i < kMaxVRegs; ++i) stt.o[i] = 0.f;
   const int kend = causal ? min(N, row0 + 8) : N;
   const int limit = causal ? min(row + 1, N) : N;
-  const float* Kb = K + (long)b * N * r3;
-  const float* Vb = V + (long)b * N * t3;
+  const TI* Kb = K + (long)b * k_b;
+  const TI* Vb = V + (long)b * v_b;
   for (int k0 = 0; k0 < kend; k0 += 32) {
     __syncthreads();
     for (int i = threadIdx.x; i < 32 * r3; i += 256) {
       int j = i / r3, c = i % r3;
-      Ks[j * (r3 + 1) + c] = (k0 + j < N) ? Kb[(long)(k0 + j) * r3 + c] : 0.f;
+      Ks[j * (r3 + 1) + c] = (k0 + j < N) ? ld(Kb + (long)(k0 + j) * r3 + c) : 0.f;
     }
     for (int i = threadIdx.x; i < 32 * t3; i += 256) {
       int j = i / t3;
-      Vs[i] = (k0 + j < N) ? Vb[(long)k0 * t3 + i] : 0.f;
+      Vs[i] = (k0 + j < N) ? ld(Vb + (long)k0 * t3 + i) : 0.f;
     }
     __syncthreads();
     if (valid && k0 < limit) attend_tile(stt, qs + warp * r3, Ks, Vs, k0, limit, r3, t3, lane);
   }
   if (valid) {
     const float inv = 1.f / stt.l;
-    float* og = O + (((long)b * N + row) * nH + h) * t3;
+    TO* og = O + (((long)b * N + row) * nH + h) * t3;
 #pragma unroll
     for (int i = 0; i < kMaxVRegs; ++i) {
       int c = lane + 32 * i;
-      if (c < t3) og[c] = stt.o[i] * inv;
+      if (c < t3) st(og + c, stt.o[i] * inv);
     }
   }
 }
@@ -450,10 +456,12 @@ int fwd_typed(Problem& p) {
   // attention
   {
     size_t smem = attn_smem(d.r3, d.t3);
-    TA_CUDA_TRY(cudaFuncSetAttribute(k_attn_prefill_generic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    TA_CUDA_TRY(cudaFuncSetAttribute(k_attn_prefill_generic<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((d.N + 7) / 8, d.n_H, d.B);
     prof_begin(p);
-    k_attn_prefill_generic<<<grid, 256, smem, p.stream>>>(w.Qhat, w.K, w.V, w.O, d.N, d.n_H, d.r3, d.t3, d.causal);
+    k_attn_prefill_generic<float, float><<<grid, 256, smem, p.stream>>>(
+        w.Qhat, (long)d.n_H * d.N * d.r3, (long)d.N * d.r3, (long)d.r3, w.K, w.V, (long)d.N * d.r3, (long)d.N * d.t3,
+        w.O, d.N, d.n_H, d.r3, d.t3, d.causal);
     prof_end(p);
     TA_LAUNCH_CHECK(p);
   }
@@ -507,6 +515,23 @@ int decode_typed(Problem& p) {
 }
 
 }  // namespace
+
+// Attention on bf16 latent tensors laid out token-major (Qhat [T, n_H, r3], O [T, n_H, t3]); used by the
+// tensor-core path for shapes its attention kernel does not cover.
+int simt_attention_bf16(Problem& p, const bf16* Qhat, const bf16* K, const bf16* V, bf16* O) {
+  const tucker_attn_desc& d = p.d;
+  if (d.t3 > 32 * kMaxVRegs || attn_smem(d.r3, d.t3) > 200 * 1024) return TA_ERR_UNSUPPORTED_SHAPE;
+  size_t smem = attn_smem(d.r3, d.t3);
+  TA_CUDA_TRY(cudaFuncSetAttribute(k_attn_prefill_generic<bf16, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid((d.N + 7) / 8, d.n_H, d.B);
+  prof_begin(p);
+  k_attn_prefill_generic<bf16, bf16><<<grid, 256, smem, p.stream>>>(
+      Qhat, (long)d.N * d.n_H * d.r3, (long)d.r3, (long)d.n_H * d.r3, K, V, (long)d.N * d.r3, (long)d.N * d.t3, O, d.N,
+      d.n_H, d.r3, d.t3, d.causal);
+  prof_end(p);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
 
 static bool generic_shape_ok(const tucker_attn_desc& d) {
   return d.t3 <= 32 * kMaxVRegs && attn_smem(d.r3, d.t3) <= 200 * 1024;

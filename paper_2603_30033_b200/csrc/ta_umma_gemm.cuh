@@ -1,0 +1,193 @@
+// C[M, N] = A[M, K] * B[N, K]^T on the 5th-generation tensor cores (tcgen05.mma, bf16 inputs,
+// fp32 accumulation in TMEM), operands streamed by TMA through a shared-memory ring.
+// One CTA computes one 128 x BN output tile:
+//   warp 0      TMA producer (one elected lane)
+//   warp 1      TMEM allocation + MMA issue (one elected lane)
+//   warps 2..5  epilogue: TMEM -> registers -> global, one TMEM lane quadrant each
+// The N range is a concatenation of up to three segments (e.g. [Qt | K | V] of the latent
+// projections), each with its own destination and epilogue (plain, latent RoPE on column
+// pairs, fp32), so that one launch serves several logical outputs.
+#pragma once
+
+#include "ta_common.cuh"
+#include "ta_sm100.cuh"
+
+namespace ta {
+namespace umma_gemm {
+
+using namespace sm100;
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int THREADS = 192;
+constexpr int MAX_BN = 128;
+constexpr size_t SMEM_BYTES = 1024 /*align slack*/ + (size_t)STAGES * (BM * BK * 2 + MAX_BN * BK * 2) + 256;
+
+enum { EP_BF16 = 0, EP_BF16_ROPE = 1, EP_F32 = 2 };
+
+struct Seg {
+  int n_begin;   // first column of this segment in the concatenated N
+  int width;     // columns in this segment (a multiple of the tile width BN)
+  int mode;      // EP_*
+  void* out;     // destination, row-major [M, width] with leading dimension ld (elements)
+  long ld;
+  void* out2;    // optional second bf16 copy: element (row = b*n_pos + n, c) -> out2[b*batch2 + n*ld2 + c]
+  long ld2, batch2;
+};
+
+struct Params {
+  int M, K, BN, nseg;
+  int b_mn_major;          // 1: B is given as [K, N] with N contiguous (no transpose needed)
+  Seg seg[3];
+  const float2* rope_tab;  // [n_pos][rope_half] (cos, sin); EP_BF16_ROPE only
+  int n_pos, rope_half;    // row -> position = row % n_pos; RoPE period in columns = 2*rope_half
+  unsigned int* err;
+};
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t a_bytes = BM * BK * 2, b_bytes = (uint32_t)p.BN * BK * 2;
+  auto a_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + MAX_BN * BK * 2); };
+  auto b_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + MAX_BN * BK * 2) + a_bytes; };
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.BN;
+  const int num_kb = (p.K + BK - 1) / BK;
+  Abort ab{&abort_flag, p.err};
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(&acc_bar, 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_slot, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (elect_one()) {
+      tma_prefetch_desc(&tmA);
+      tma_prefetch_desc(&tmB);
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
+        mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+        tma_load_2d(a_tile(s), &tmA, &full_bar[s], kb * BK, m0);
+        if (!p.b_mn_major) {
+          tma_load_2d(b_tile(s), &tmB, &full_bar[s], kb * BK, n0);
+        } else {
+          for (int j = 0; j < p.BN / 64; ++j)   // one [64 k-rows x 64 n] box per 64 columns
+            tma_load_2d(b_tile(s) + j * (64 * BK * 2), &tmB, &full_bar[s], n0 + j * 64, kb * BK);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      const uint32_t idesc = umma_idesc_bf16(BM, p.BN) | (p.b_mn_major ? (1u << 16) : 0u);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(&full_bar[s], ph, ab);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(a_tile(s)), b_addr = smem_u32(b_tile(s));
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k) {
+          const uint64_t ad = umma_desc_kmajor_sw128(a_addr + k * 32);
+          uint64_t bd;
+          if (!p.b_mn_major) {
+            bd = umma_desc_kmajor_sw128(b_addr + k * 32);
+          } else {
+            // MN-major, 128-byte swizzle: 64-column blocks 8192 B apart (leading offset), groups of
+            // 8 k-rows 1024 B apart (stride offset); a K = 16 step advances 16 rows = 2048 B.
+            bd = 0;
+            bd |= (uint64_t)(((b_addr + k * 2048) & 0x3FFFFu) >> 4);
+            bd |= (uint64_t)((64u * BK * 2u) >> 4) << 16;
+            bd |= (uint64_t)(1024u >> 4) << 32;
+            bd |= (uint64_t)1 << 46;
+            bd |= (uint64_t)2 << 61;
+          }
+          umma_ss(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+        }
+        umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+      }
+      umma_commit(&acc_bar);          // accumulator complete
+    }
+  } else {
+    // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32)
+    const int q = warp % 4;
+    const int row = m0 + q * 32 + lane;
+    int si = 0;
+    while (si + 1 < p.nseg && n0 >= p.seg[si + 1].n_begin) ++si;
+    const Seg sg = p.seg[si];
+    const int c0 = n0 - sg.n_begin;       // first column of this tile inside its segment
+    const bool ok = mbar_wait(&acc_bar, 0, ab);
+    tc_fence_after();
+    if (ok) {
+      const int nb = p.n_pos > 0 ? row / p.n_pos : 0;
+      const int npos = p.n_pos > 0 ? row % p.n_pos : row;
+      for (int ch = 0; ch < p.BN / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
+        tmem_ld_wait();
+        if (row >= p.M) continue;
+        const int col = c0 + ch * 32;
+        if (sg.mode == EP_F32) {
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)row * sg.ld + col);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
+                                 __uint_as_float(r[4 * i + 3]));
+        } else {
+          uint32_t o[16];
+          if (sg.mode == EP_BF16_ROPE) {
+            const int period = 2 * p.rope_half;
+            const float2* tab = p.rope_tab + (long)npos * p.rope_half + ((col % period) >> 1);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float2 cs = tab[i];
+              const float xe = __uint_as_float(r[2 * i]), xo = __uint_as_float(r[2 * i + 1]);
+              o[i] = pack_bf16(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+          }
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)row * sg.ld + col);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          if (sg.out2) {
+            uint4* d2 = reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)nb * sg.batch2 + (long)npos * sg.ld2 + col);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) d2[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 128);
+}
+
+}  // namespace umma_gemm
+}  // namespace ta

@@ -42,9 +42,20 @@ def err_stats(got, ref):
     return float(d.max()), float(d.mean())
 
 
-def tolerances(dtype: str):
-    """(max-abs, mean-abs) bounds: bf16 storage with fp32 accumulation 2e-2 / 2e-3; fp32 1e-4."""
-    return (2e-2, 2e-3) if dtype == "bf16" else (1e-4, 1e-4)
+def tolerances(dtype: str, ref=None):
+    """(max-abs, mean-abs) bounds: bf16 storage with fp32 accumulation 2e-2 / 2e-3; fp32 1e-4.
+
+    The bf16 bounds are absolute and are the ones the five benchmark workloads are held to;
+    their outputs have rms <= 0.16.  bf16 rounding is relative (2^-9 per rounding point: the
+    latent queries / keys / values, P, O, Z, Y), so for the extra stress shapes, whose outputs
+    are several times larger, the bounds scale with the output size: pass `ref` to multiply
+    them by max(1, rms(ref) / 0.2).  fp32 bounds never scale."""
+    if dtype != "bf16":
+        return (1e-4, 1e-4)
+    s = 1.0
+    if ref is not None:
+        s = max(1.0, float(np.sqrt(np.mean(np.asarray(ref, np.float64) ** 2))) / 0.2)
+    return (2e-2 * s, 2e-3 * s)
 
 
 def with_(w: W.Workload, **kw) -> W.Workload:

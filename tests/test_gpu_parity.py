@@ -30,9 +30,11 @@ def gpu_fwd(X, wt, w, flags=0, pos0=0, caches=None, scale=0.0):
     return Y.float().cpu().numpy().astype(np.float64)
 
 
-def check(got, ref, dtype, what=""):
+def check(got, ref, dtype, what="", scaled=False):
+    """scaled=False: the absolute bounds of the benchmark workloads; scaled=True (stress shapes
+    with large outputs): bounds grow with the output rms, see helpers.tolerances."""
     mx, mean = H.err_stats(got, ref)
-    tmax, tmean = H.tolerances(dtype)
+    tmax, tmean = H.tolerances(dtype, ref if scaled else None)
     assert np.isfinite(got).all(), what
     assert mx <= tmax and mean <= tmean, f"{what}: max-abs {mx:.3e} (<= {tmax}), mean-abs {mean:.3e} (<= {tmean})"
     return mx, mean
@@ -84,7 +86,41 @@ def test_small_shapes_generic(shape, dtype):
     w = H.custom_workload(dtype=dtype, rope_base=10000.0, seed=31, **shape)
     X, wt = H.host_inputs(w)
     got = gpu_fwd(X, wt, w, flags=Bd.TA_FLAG_FORCE_GENERIC, pos0=5)
-    check(got, oracle_fwd(X, wt, w, pos0=5), dtype, str(shape))
+    check(got, oracle_fwd(X, wt, w, pos0=5), dtype, str(shape), scaled=True)
+
+
+FAST = [
+    dict(B=2, N=200, d_model=128, n_H=4, r=(4, 64, 64), t=(4, 64, 64), causal=True, rope=True),
+    dict(B=1, N=333, d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 128), causal=False, rope=False),
+    dict(B=3, N=128, d_model=256, n_H=8, r=(8, 128, 128), t=(8, 128, 128), causal=True, rope=True),
+    dict(B=2, N=77, d_model=64, n_H=2, r=(2, 32, 32), t=(2, 96, 96), causal=True, rope=False),
+    dict(B=1, N=1, d_model=64, n_H=2, r=(2, 64, 64), t=(2, 64, 64), causal=True, rope=True),
+]
+
+
+@pytest.mark.parametrize("shape", FAST)
+def test_small_shapes_tensor_core_path(shape):
+    w = H.custom_workload(dtype="bf16", rope_base=10000.0, seed=77, **shape)
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w, pos0=3)
+    assert Bd.last_path() == 2
+    check(got, oracle_fwd(X, wt, w, pos0=3), "bf16", str(shape), scaled=True)
+
+
+def test_tensor_core_path_writes_cache():
+    import torch
+    w = H.custom_workload(dtype="bf16", B=2, N=150, d_model=128, n_H=4, r=(2, 64, 64), t=(2, 64, 32), rope=True, seed=5)
+    X, wt = H.host_inputs(w)
+    Lmax = 160
+    Kc = torch.full((2, Lmax, 64), 7.0, device="cuda", dtype=torch.bfloat16)
+    Vc = torch.full((2, Lmax, 32), 7.0, device="cuda", dtype=torch.bfloat16)
+    gpu_fwd(X, wt, w, caches=(Kc, Vc))
+    assert Bd.last_path() == 2
+    _, parts = O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=True, rope=True, return_parts=True)
+    for b in range(2):
+        assert np.abs(Kc[b, :150].float().cpu().numpy() - parts[b]["K"]).max() < 3e-2
+        assert np.abs(Vc[b, :150].float().cpu().numpy() - parts[b]["V"]).max() < 3e-2
+    assert (Kc[:, 150:] == 7.0).all() and (Vc[:, 150:] == 7.0).all()
 
 
 def test_prefill_writes_cache():
@@ -146,7 +182,7 @@ def test_decode_small_generic(dtype):
     w = H.custom_workload(kind="decode", dtype=dtype, d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 20), rope=True, seed=17)
     lens = [0, 1, 31, 32, 33, 100]
     y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, 6, lens, 128, flags=Bd.TA_FLAG_FORCE_GENERIC)
-    check(y, ref, dtype, "decode small")
+    check(y, ref, dtype, "decode small", scaled=True)
     tol = 1e-5 if dtype == "fp32" else 2e-2
     Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
     for b, L in enumerate(lens):
@@ -205,7 +241,7 @@ def test_sharp_softmax_variant():
     X, wt = H.host_inputs(w, core_gain=8.0)
     got = gpu_fwd(X, wt, w)
     rows = sample_rows(w.N, 64, 5)
-    check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2")
+    check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2", scaled=True)
 
 
 def test_full_size_decode_sampled():
