@@ -9,6 +9,7 @@
 //   z, y      Z = O [Gt_1; ...; Gt_nH]^T,  Y = Z Ut2^T   (Eqs. 5-6)
 #include "ta_common.cuh"
 #include "ta_umma_gemm.cuh"
+#include "ta_attn_prefill.cuh"
 
 #include <math.h>
 
@@ -166,6 +167,41 @@ int launch_gemm(Problem& p, const bf16* A, long lda, const bf16* Bm, long ldb, i
   return TA_OK;
 }
 
+bool tmap_3d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t batches, uint64_t ld,
+             uint64_t batch_stride, uint32_t box_cols, uint32_t box_rows) {
+  uint64_t dims[3] = {cols, rows, batches}, str[2] = {ld, batch_stride};
+  uint32_t box[3] = {box_cols, box_rows, 1};
+  return make_tmap(m, base, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+bool umma_attention_ok(const tucker_attn_desc& d) { return d.r3 <= 128 && d.t3 <= 128; }
+
+int umma_attention(Problem& p, const bf16* Qhat, const bf16* K, const bf16* V, bf16* O) {
+  const tucker_attn_desc& d = p.d;
+  CUtensorMap tmQ, tmK, tmV;
+  const uint64_t qcols = (uint64_t)d.n_H * d.r3;
+  if (!tmap_3d(&tmQ, Qhat, qcols, d.N, d.B, qcols, (uint64_t)d.N * qcols, 64, 128)) return TA_ERR_CUDA;
+  if (!tmap_3d(&tmK, K, d.r3, d.N, d.B, d.r3, (uint64_t)d.N * d.r3, 64, 128)) return TA_ERR_CUDA;
+  if (!tmap_3d(&tmV, V, d.t3, d.N, d.B, d.t3, (uint64_t)d.N * d.t3, 64, 128)) return TA_ERR_CUDA;
+  attn::Params ap;
+  ap.B = d.B; ap.N = d.N; ap.nH = d.n_H; ap.r3 = d.r3; ap.t3 = d.t3; ap.causal = d.causal;
+  ap.n_qt = (d.N + attn::BQ - 1) / attn::BQ;
+  ap.n_hp = (d.n_H + 1) / 2;
+  ap.O = O; ap.err = p.dev_err;
+  static bool attr_set = false;
+  if (!attr_set) {
+    TA_CUDA_TRY(cudaFuncSetAttribute(attn::k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)attn::SMEM_BYTES));
+    attr_set = true;
+  }
+  const long items = (long)ap.n_qt * d.B * ap.n_hp;
+  prof_begin(p);
+  attn::k_attn_prefill<<<(unsigned)items, attn::THREADS, attn::SMEM_BYTES, p.stream>>>(tmQ, tmK, tmV, ap);
+  prof_end(p);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
+
 umma_gemm::Seg seg(int n_begin, int width, int mode, void* out, long ld) {
   umma_gemm::Seg s;
   s.n_begin = n_begin; s.width = width; s.mode = mode; s.out = out; s.ld = ld;
@@ -192,15 +228,15 @@ int fast_fwd(Problem& p) {
   const int T = d.B * d.N;
   const bool mn = (d.flags & 0x100) != 0;   // bring-up switch: feed U2/U3/Ut3 untransposed (MN-major B)
   const float LOG2E = 1.4426950408889634f;
+  const bool tc_attn = umma_attention_ok(d) && !(d.flags & 0x200);   // 0x200: bring-up switch, FMA attention
 
   // ---- weight preparation ----
   k_head_core_bf16<<<grid_for((long)d.n_H * d.r2 * d.r3), 256, 0, p.stream>>>(
-      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, p.scale);
+      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, tc_attn ? p.scale * LOG2E : p.scale);
   TA_LAUNCH_CHECK(p);
   k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
       (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
   TA_LAUNCH_CHECK(p);
-  (void)LOG2E;
   if (!mn) {
     const bf16* srcs[3] = {(const bf16*)p.U2, (const bf16*)p.U3, (const bf16*)p.Ut3};
     const int widths[3] = {d.r2, d.r3, d.t3};
@@ -270,7 +306,11 @@ int fast_fwd(Problem& p) {
     if ((rc = launch_gemm(p, w.Qt, d.r2, w.GcatT, d.r2, T, d.r2, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
   }
   // ---- attention ----
-  if ((rc = simt_attention_bf16(p, w.Qhat, w.K, w.V, w.O))) return rc;
+  if (tc_attn) {
+    if ((rc = umma_attention(p, w.Qhat, w.K, w.V, w.O))) return rc;
+  } else {
+    if ((rc = simt_attention_bf16(p, w.Qhat, w.K, w.V, w.O))) return rc;
+  }
   // ---- output side ----
   {
     umma_gemm::Params gp = {};
