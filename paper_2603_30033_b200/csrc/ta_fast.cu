@@ -10,6 +10,7 @@
 #include "ta_common.cuh"
 #include "ta_umma_gemm.cuh"
 #include "ta_attn_prefill.cuh"
+#include "ta_decode.cuh"
 
 #include <math.h>
 
@@ -146,7 +147,7 @@ int pick_bn(int width) {
 
 // C[M, sum(widths)] = A[M, K] * B^T with B [Ntot, K] K-major (or [K, Ntot] when b_mn_major).
 int launch_gemm(Problem& p, const bf16* A, long lda, const bf16* Bm, long ldb, int M, int K, int Ntot, int BN,
-                umma_gemm::Params gp) {
+                umma_gemm::Params gp, int splits = 1) {
   CUtensorMap tmA, tmB;
   if (!tmap_2d(&tmA, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, 128)) return TA_ERR_CUDA;
   if (!gp.b_mn_major) {
@@ -161,7 +162,7 @@ int launch_gemm(Problem& p, const bf16* A, long lda, const bf16* Bm, long ldb, i
                                      (int)umma_gemm::SMEM_BYTES));
     attr_set = true;
   }
-  dim3 grid(Ntot / BN, (M + 127) / 128);
+  dim3 grid(Ntot / BN, (M + 127) / 128, splits);
   umma_gemm::k_umma_gemm<<<grid, umma_gemm::THREADS, umma_gemm::SMEM_BYTES, p.stream>>>(tmA, tmB, gp);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
@@ -330,8 +331,176 @@ int fast_fwd(Problem& p) {
   return TA_OK;
 }
 
-bool fast_decode_supported(const tucker_attn_desc&, int32_t) { return false; }
-size_t fast_decode_workspace(const tucker_attn_desc&, int32_t) { return 0; }
-int fast_decode(Problem&) { return TA_ERR_UNSUPPORTED_SHAPE; }
+// ---------------------------------------------------------------------------------------------
+// decode
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kProjSplits = 16;
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+// number of K splits of the decode projection GEMM: the largest divisor of the K-block count <= kProjSplits
+int proj_splits(int d_model) {
+  const int nkb = d_model / 64;
+  for (int s = kProjSplits; s > 1; --s)
+    if (nkb % s == 0) return s;
+  return 1;
+}
+
+int decode_grid() { return sm_count() < dec::MAX_GRID ? sm_count() : dec::MAX_GRID; }
+
+struct FastDecWs {
+  bf16 *Wt, *GcatT, *GtP;
+  float* proj_part;   // [splits][128][r2 + r3 + t3]
+  bf16 *qt, *knew, *vnew, *qhat, *z;
+  float2* rope_row;   // [B][r3/2]
+  float *part_o, *part_ml;
+};
+
+size_t carve_fast_dec(const tucker_attn_desc& d, char* base, FastDecWs* w) {
+  Carver c(base);
+  FastDecWs t;
+  const size_t Mpad = (size_t)((d.B + 127) / 128) * 128;
+  const size_t ncol = (size_t)d.r2 + d.r3 + d.t3;
+  t.Wt = c.take<bf16>(ncol * d.d_model);
+  t.GcatT = c.take<bf16>((size_t)d.n_H * d.r3 * d.r2);
+  t.GtP = c.take<bf16>((size_t)d.t2 * d.n_H * d.t3);
+  t.proj_part = c.take<float>((size_t)kProjSplits * Mpad * ncol);
+  t.qt = c.take<bf16>((size_t)d.B * d.r2);
+  t.knew = c.take<bf16>((size_t)d.B * d.r3);
+  t.vnew = c.take<bf16>((size_t)d.B * d.t3);
+  t.qhat = c.take<bf16>((size_t)d.B * d.n_H * d.r3);
+  t.z = c.take<bf16>((size_t)d.B * d.t2);
+  t.rope_row = c.take<float2>((size_t)d.B * ((d.r3 + 1) / 2));
+  const size_t slots = (size_t)dec::MAX_GRID + d.B;
+  t.part_o = c.take<float>(slots * 32 * d.t3);
+  t.part_ml = c.take<float>(slots * 64);
+  if (w) *w = t;
+  return c.off;
+}
+
+template <int R3, int T3>
+int launch_dec_attn(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const dec::Params& dp) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    TA_CUDA_TRY(cudaFuncSetAttribute(dec::k_dec_attn<R3, T3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)dec::SMEM_BYTES));
+    attr_set = true;
+  }
+  prof_begin(p);
+  dec::k_dec_attn<R3, T3><<<dp.grid, dec::THREADS, dec::SMEM_BYTES, p.stream>>>(tmK, tmV, dp);
+  prof_end(p);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
+
+bool dec_rank_ok(int r3, int t3) {
+  return (r3 == 128 && t3 == 128) || (r3 == 64 && t3 == 64) || (r3 == 96 && t3 == 96) || (r3 == 128 && t3 == 64) ||
+         (r3 == 64 && t3 == 128);
+}
+
+}  // namespace
+
+bool fast_decode_supported(const tucker_attn_desc& d, int32_t Lmax) {
+  auto ok32 = [](int r) { return r >= 32 && r <= 256 && r % 32 == 0; };
+  if (!ok32(d.r2) || !ok32(d.t2) || !dec_rank_ok(d.r3, d.t3)) return false;
+  if (d.d_model % 64 || d.n_H > 32 || d.B > 4096) return false;
+  if (d.t2 % 16) return false;
+  (void)Lmax;
+  return true;
+}
+
+size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t) { return carve_fast_dec(d, nullptr, nullptr); }
+
+int fast_decode(Problem& p) {
+  const tucker_attn_desc& d = p.d;
+  FastDecWs w;
+  carve_fast_dec(d, p.ws, &w);
+  const float LOG2E = 1.4426950408889634f;
+  const int ncol = d.r2 + d.r3 + d.t3;
+  const int Mpad = (d.B + 127) / 128 * 128;
+  const int splits = proj_splits(d.d_model);
+  int rc;
+  // ---- weight preparation (head-mode core contraction; transposed factors) ----
+  k_head_core_bf16<<<grid_for((long)d.n_H * d.r2 * d.r3), 256, 0, p.stream>>>(
+      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, p.scale * LOG2E);
+  TA_LAUNCH_CHECK(p);
+  k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
+      (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
+  TA_LAUNCH_CHECK(p);
+  {
+    const bf16* srcs[3] = {(const bf16*)p.U2, (const bf16*)p.U3, (const bf16*)p.Ut3};
+    const int widths[3] = {d.r2, d.r3, d.t3};
+    long off = 0;
+    for (int i = 0; i < 3; ++i) {
+      dim3 grid((widths[i] + 31) / 32, (d.d_model + 31) / 32);
+      k_transpose_bf16<<<grid, dim3(32, 8), 0, p.stream>>>(srcs[i], w.Wt + off * d.d_model, d.d_model, widths[i]);
+      TA_LAUNCH_CHECK(p);
+      off += widths[i];
+    }
+  }
+  // ---- projections of the new tokens: split-K partial sums, then finish (RoPE, append) ----
+  {
+    umma_gemm::Params gp = {};
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, ncol, umma_gemm::EP_F32, w.proj_part, ncol);
+    gp.kb_per_split = (d.d_model / 64) / splits;
+    gp.split_stride = (long)Mpad * ncol;
+    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, w.Wt, d.d_model, d.B, d.d_model, ncol, 32, gp, splits)))
+      return rc;
+  }
+  dec::k_dec_finish<<<d.B, 128, ncol * sizeof(float), p.stream>>>(
+      w.proj_part, splits, (long)Mpad * ncol, d.B, d.r2, d.r3, d.t3, w.qt, w.knew, w.vnew, w.rope_row, (bf16*)p.Kc,
+      (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, (double)d.rope_base, p.append, p.dev_err);
+  TA_LAUNCH_CHECK(p);
+  // ---- per-head queries, rotated at each sequence's own position ----
+  {
+    umma_gemm::Params gp = {};
+    gp.rope_tab = w.rope_row; gp.n_pos = d.B; gp.rope_half = d.r3 / 2;
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, d.n_H * d.r3, d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16, w.qhat, (long)d.n_H * d.r3);
+    if ((rc = launch_gemm(p, w.qt, d.r2, w.GcatT, d.r2, d.B, d.r2, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
+  }
+  // ---- attention over the latent cache ----
+  {
+    CUtensorMap tmK, tmV;
+    if (!tmap_3d(&tmK, p.Kc, d.r3, p.Lmax, d.B, d.r3, (uint64_t)p.Lmax * d.r3, 64, 128)) return TA_ERR_CUDA;
+    if (!tmap_3d(&tmV, p.Vc, d.t3, p.Lmax, d.B, d.t3, (uint64_t)p.Lmax * d.t3, 64, 128)) return TA_ERR_CUDA;
+    dec::Params dp;
+    dp.B = d.B; dp.nH = d.n_H; dp.Lmax = p.Lmax; dp.grid = decode_grid();
+    dp.cache_len = p.cache_len; dp.qhat = w.qhat; dp.knew = w.knew; dp.vnew = w.vnew;
+    dp.part_o = w.part_o; dp.part_ml = w.part_ml; dp.err = p.dev_err;
+    if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);
+    else if (d.r3 == 64 && d.t3 == 64) rc = launch_dec_attn<64, 64>(p, tmK, tmV, dp);
+    else if (d.r3 == 96 && d.t3 == 96) rc = launch_dec_attn<96, 96>(p, tmK, tmV, dp);
+    else if (d.r3 == 128 && d.t3 == 64) rc = launch_dec_attn<128, 64>(p, tmK, tmV, dp);
+    else rc = launch_dec_attn<64, 128>(p, tmK, tmV, dp);
+    if (rc) return rc;
+    // ---- merge the partials, output-side core ----
+    const size_t smem = sizeof(float) * (32 * (size_t)d.t3 + (size_t)dec::MAX_GRID * 32);
+    dec::k_dec_merge<<<dim3(d.t2 / 16, d.B), 256, smem, p.stream>>>(w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H,
+                                                                    d.t3, d.t2, dp.grid, w.GtP, w.z);
+    TA_LAUNCH_CHECK(p);
+  }
+  // ---- y = z Ut2^T ----
+  {
+    umma_gemm::Params gp = {};
+    gp.n_pos = d.B;
+    gp.nseg = 1;
+    gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
+    if ((rc = launch_gemm(p, w.z, d.t2, (const bf16*)p.Ut2, d.t2, d.B, d.t2, d.d_model, pick_bn(d.d_model), gp))) return rc;
+  }
+  return TA_OK;
+}
 
 }  // namespace ta

@@ -42,6 +42,8 @@ struct Params {
   Seg seg[3];
   const float2* rope_tab;  // [n_pos][rope_half] (cos, sin); EP_BF16_ROPE only
   int n_pos, rope_half;    // row -> position = row % n_pos; RoPE period in columns = 2*rope_half
+  int kb_per_split;        // split-K: 64-wide K blocks per blockIdx.z (0 = no split); EP_F32 outputs only
+  long split_stride;       // elements between the partial outputs of consecutive splits
   unsigned int* err;
 };
 
@@ -60,7 +62,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.BN;
-  const int num_kb = (p.K + BK - 1) / BK;
+  const int num_kb_all = (p.K + BK - 1) / BK;
+  const int kb_begin = p.kb_per_split > 0 ? (int)blockIdx.z * p.kb_per_split : 0;
+  const int num_kb = p.kb_per_split > 0 ? min(p.kb_per_split, num_kb_all - kb_begin) : num_kb_all;
   Abort ab{&abort_flag, p.err};
 
   if (threadIdx.x == 0) {
@@ -90,12 +94,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
         mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-        tma_load_2d(a_tile(s), &tmA, &full_bar[s], kb * BK, m0);
+        const int kx = (kb_begin + kb) * BK;
+        tma_load_2d(a_tile(s), &tmA, &full_bar[s], kx, m0);
         if (!p.b_mn_major) {
-          tma_load_2d(b_tile(s), &tmB, &full_bar[s], kb * BK, n0);
+          tma_load_2d(b_tile(s), &tmB, &full_bar[s], kx, n0);
         } else {
           for (int j = 0; j < p.BN / 64; ++j)   // one [64 k-rows x 64 n] box per 64 columns
-            tma_load_2d(b_tile(s) + j * (64 * BK * 2), &tmB, &full_bar[s], n0 + j * 64, kb * BK);
+            tma_load_2d(b_tile(s) + j * (64 * BK * 2), &tmB, &full_bar[s], n0 + j * 64, kx);
         }
       }
     }
@@ -152,7 +157,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (row >= p.M) continue;
         const int col = c0 + ch * 32;
         if (sg.mode == EP_F32) {
-          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)row * sg.ld + col);
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)blockIdx.z * p.split_stride +
+                                                  (long)row * sg.ld + col);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),

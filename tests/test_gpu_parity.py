@@ -191,6 +191,52 @@ def test_decode_small_generic(dtype):
         assert np.array_equal(Kh[b, L + 1:], Kc[b, L + 1:].astype(np.float32))
 
 
+DEC_FAST = [
+    dict(d_model=256, n_H=4, r=(2, 64, 64), t=(2, 64, 64), lens=[0, 1, 127, 128, 129, 300, 1000], Lmax=1024),
+    dict(d_model=256, n_H=32, r=(8, 128, 128), t=(8, 128, 128), lens=[511, 5, 2047, 256, 255], Lmax=2048),
+    dict(d_model=192, n_H=12, r=(4, 96, 96), t=(4, 32, 96), lens=[700, 33], Lmax=777),
+    dict(d_model=128, n_H=2, r=(2, 32, 128), t=(2, 64, 64), lens=[100] * 3 + [4000] + [0] * 200, Lmax=4001),
+    dict(d_model=128, n_H=8, r=(2, 64, 64), t=(2, 32, 128), lens=[50000], Lmax=50001),
+]
+
+
+@pytest.mark.parametrize("append", [True, False])
+@pytest.mark.parametrize("case", DEC_FAST)
+def test_decode_tensor_core_path(case, append):
+    case = dict(case)
+    lens, Lmax = case.pop("lens"), case.pop("Lmax")
+    w = H.custom_workload(kind="decode", dtype="bf16", rope=True, rope_base=500000.0, seed=23, **case)
+    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, len(lens), lens, Lmax, append=append)
+    assert Bd.last_path() == 2
+    check(y, ref, "bf16", f"decode {case}", scaled=True)
+    Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
+    for b, L in enumerate(lens[:8]):
+        if append:
+            assert np.abs(Kh[b, L] - ref_k[b]).max() < 3e-2 and np.abs(Vh[b, L] - ref_v[b]).max() < 3e-2
+            Kh[b, L], Vh[b, L] = Kc[b, L], Vc[b, L]
+        assert np.array_equal(Kh[b], Kc[b].astype(np.float32)) and np.array_equal(Vh[b], Vc[b].astype(np.float32))
+
+
+def test_decode_garbage_beyond_cache_len_is_ignored():
+    # slots at and after cache_len hold NaN / Inf bit patterns: they must not leak into the result
+    import torch
+    w = H.custom_workload(kind="decode", dtype="bf16", d_model=256, n_H=4, r=(2, 64, 64), t=(2, 64, 64), rope=True, seed=29)
+    lens = [5, 130, 255]
+    Lmax = 300
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    x, Kc, Vc, cache_len = W.make_decode_state(w, B=3, L=max(lens), Lmax=Lmax, cache_len=lens)
+    x, Kc, Vc = (W.round_to_storage(a, w.dtype) for a in (x, Kc, Vc))
+    ref, _, _ = O.tucker_attn_decode(x, *[wt[k] for k in H.WEIGHT_KEYS], Kc, Vc, cache_len, rope=True, rope_base=w.rope_base)
+    Kd, Vd = H.to_device(Kc, "bf16"), H.to_device(Vc, "bf16")
+    for b, L in enumerate(lens):
+        Kd[b, L:] = float("nan")
+        Vd[b, L:] = float("inf")
+    y = Bd.tucker_attn_decode(H.to_device(x, "bf16"), *H.weights_to_device(wt, "bf16"), Kd, Vd,
+                              torch.from_numpy(cache_len).cuda(), n_H=4, rope=True, rope_base=w.rope_base, append=False)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == 2
+    check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "garbage tail", scaled=True)
+
+
 def test_decode_no_append_leaves_cache():
     w = H.custom_workload(kind="decode", dtype="fp32", d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), rope=True, seed=18)
     y, ref, (Kd, Vd, Kc, Vc, *_r) = run_decode(w, 2, [5, 9], 16, append=False)
