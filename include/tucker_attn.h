@@ -12,12 +12,12 @@
  *   G_h  = sum_a U1[h,a]  C[a,:,:]                   head-mode core contraction C x_1 U1 (Def. 2, Sec. 3.3)
  *   Gt_h = sum_a Ut1[h,a] Ct[a,:,:]
  *   Qhat_h = Qt G_h                                  per-head latent queries (Def. 2)
- *   latent RoPE: Qhat_{h,m} R(m,r3),  K_n R(n,r3)    rotation in the latent key dimension (Eq. 9, App. C.2)
+ *   latent RoPE: Qhat_{h,m} R(m,r3),  K_n R(n,r3)    rotation in the latent key dimension (Eq. 12, App. C.2)
  *   S_h = Qhat_h K^T * scale, causal mask, row softmax (online, never materialised; Sec. 3.3)
  *   O_h = P_h V
  *   Z   = sum_h O_h Gt_h^T ;  Y = Z Ut2^T            value/output-side factors (Eqs. 5-6)
  *
- * and the cached decode step of Eq. 8 for one new token per sequence.
+ * and the cached decode step of Eq. 9 for one new token per sequence.
  *
  * General conventions
  *   - Every data pointer is CALLER-OWNED DEVICE memory unless stated otherwise; row-major,
@@ -106,7 +106,7 @@ TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * One cached decode step (Eq. 8, "KV Caching"): for every sequence b the new token x[b] at
+ * One cached decode step (Eq. 9, "KV Caching"): for every sequence b the new token x[b] at
  * position L = cache_len[b] attends to cache slots 0..L-1 and to itself.
  *   x         [B, d_model]                     in
  *   Kcache    [B, Lmax, r3] rotated latent keys, Vcache [B, Lmax, t3]   in (and out if append)

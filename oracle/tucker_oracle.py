@@ -104,7 +104,7 @@ def tucker_attn_fwd(X, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, *, causal=False, rope=F
     Steps, in the paper's order:
       K = X U3, V = X Ut3 (the latent KV cache, Sec. 3.1); Qt = X U2
       Qhat = C x_1 U1 x_2 (X U2)            -> per head h: Qhat_h = Qt G_h     (Def. 2)
-      latent RoPE: Qhat_{h,m} R(m, r3), K_n R(n, r3)                            (Eq. 9 / App. C.2)
+      latent RoPE: Qhat_{h,m} R(m, r3), K_n R(n, r3)                            (Eq. 12 / App. C.2)
       S_h = Qhat_h K^T / sqrt(d_H); causal mask; row softmax                    (Eq. 4)
       O_h = P_h V;  Y = sum_h O_h Gt_h^T Ut2^T   (Eqs. 5-6 with Wt = Ct x_j Ut_j: the value
       mode of Gt_h contracts with V, its output mode with Ut2)

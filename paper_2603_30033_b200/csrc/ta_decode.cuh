@@ -1,4 +1,4 @@
-// Decode step over the latent KV cache (Eq. 8, "KV Caching"): kernels of the bf16 path.
+// Decode step over the latent KV cache (Eq. 9, "KV Caching"): kernels of the bf16 path.
 //
 // k_dec_attn streams every sequence's latent K / V cache exactly once.  The cache is cut into
 // tiles of 128 keys; the flat list of tiles of all sequences is divided evenly over the CTAs

@@ -4,7 +4,7 @@
 //   prep      G_h (scaled by softmax scale * log2 e) and Gt_h from the cores (C x_1 U1, Definition 2),
 //             stored as K-major B operands; transposed copies of U2, U3, Ut3; RoPE cos/sin table
 //   proj      [Qt | K | V] = X [U2 | U3 | Ut3]   (Sec. 3.1), latent RoPE applied to K in the epilogue
-//   qhat      Qhat[T, (h, c)] = Qt [G_1 | ... | G_nH], latent RoPE per head in the epilogue (Eq. 9)
+//   qhat      Qhat[T, (h, c)] = Qt [G_1 | ... | G_nH], latent RoPE per head in the epilogue (Eq. 12)
 //   attention online softmax over key tiles, one shared latent K / V pair for all heads (Sec. 3.3)
 //   z, y      Z = O [Gt_1; ...; Gt_nH]^T,  Y = Z Ut2^T   (Eqs. 5-6)
 #include "ta_common.cuh"

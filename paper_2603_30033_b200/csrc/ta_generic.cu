@@ -3,9 +3,9 @@
 // and for bf16 shapes the tensor-core kernels do not cover.  Intermediates are fp32.
 //
 // Steps follow Sec. 3 of the paper: latent projections (Sec. 3.1), head-mode core
-// contraction and per-head queries (Definition 2), latent RoPE (Eq. 9), online-softmax
+// contraction and per-head queries (Definition 2), latent RoPE (Eq. 12), online-softmax
 // attention with one shared latent K/V pair for all heads (Sec. 3.3), output-side factors
-// (Eqs. 5-6), and the cached decode step (Eq. 8).
+// (Eqs. 5-6), and the cached decode step (Eq. 9).
 #include "ta_common.cuh"
 
 namespace ta {
