@@ -124,6 +124,42 @@ TA_API int tucker_attn_decode(const tucker_attn_desc* desc, const void* x,
                        const int32_t* cache_len, int32_t append,
                        void* y, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Decode step without a caller-supplied workspace (the paper has no counterpart: this is a
+ * packaging variant of tucker_attn_decode, same arithmetic, same kernels).
+ *
+ * For callers that cannot allocate device memory on this path -- a serving loop whose memory
+ * was carved up once at start-up by an allocator it does not own, a plug-in whose host
+ * framework forbids cudaMalloc outside its own pool, a latency-critical loop that cannot
+ * take the device-wide synchronisation cudaMalloc / cudaFree imply.  The scratch space lives
+ * in a static device array of TA_STATIC_SCRATCH_BYTES inside the library; every GPU that
+ * loads the library holds that much memory until the process exits.  The call itself makes
+ * no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Arguments are those of tucker_attn_decode without `workspace` / `workspace_bytes`; inputs
+ * and outputs remain caller-owned device memory.
+ *
+ * Limits and behaviour
+ *   - Returns TA_ERR_WORKSPACE_TOO_SMALL, before anything is launched, when
+ *     tucker_attn_decode_workspace_bytes(desc, Lmax) exceeds TA_STATIC_SCRATCH_BYTES
+ *     (the benchmark decode shape, B = 64, n_H = 32, d = 4096, ranks 128, fits); use
+ *     tucker_attn_decode with your own buffer for larger problems.  Other errors as for
+ *     tucker_attn_decode.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Calls that may overlap on the GPU
+ *     (different streams, or different host threads) race on it: serialise them, e.g. keep
+ *     them on one stream.  Nothing in the scratch needs to start at zero -- each call
+ *     rewrites what it reads -- so back-to-back calls need no clearing in between.
+ */
+#define TA_STATIC_SCRATCH_BYTES (16u << 20)
+TA_API int tucker_attn_decode_static(const tucker_attn_desc* desc, const void* x,
+                              const void* C, const void* U1, const void* U2, const void* U3,
+                              const void* Ct, const void* Ut1, const void* Ut2, const void* Ut3,
+                              void* Kcache, void* Vcache, int32_t Lmax,
+                              const int32_t* cache_len, int32_t append,
+                              void* y, void* cuda_stream);
+
 /* Human-readable name of a status code (static storage). */
 TA_API const char* tucker_attn_status_string(int status);
 

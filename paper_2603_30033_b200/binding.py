@@ -23,7 +23,9 @@ EXPORTS = (
     "tucker_attn_fwd_workspace_bytes", "tucker_attn_decode_workspace_bytes", "tucker_attn_fwd",
     "tucker_attn_decode", "tucker_attn_status_string", "tucker_attn_last_device_error",
     "tucker_attn_last_path", "tucker_attn_last_launch_count", "tucker_attn_set_profile_events",
+    "tucker_attn_decode_static",
 )
+TA_STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class TuckerAttnDesc(ctypes.Structure):
@@ -67,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_attn_fwd.argtypes = [dp] + [vp] * 12 + [i32, vp, sz, vp]
     lib.tucker_attn_decode.restype = ctypes.c_int
     lib.tucker_attn_decode.argtypes = [dp] + [vp] * 11 + [i32, vp, i32, vp, vp, sz, vp]
+    lib.tucker_attn_decode_static.restype = ctypes.c_int
+    lib.tucker_attn_decode_static.argtypes = [dp] + [vp] * 11 + [i32, vp, i32, vp, vp]
     lib.tucker_attn_status_string.restype = ctypes.c_char_p
     lib.tucker_attn_status_string.argtypes = [ctypes.c_int]
     lib.tucker_attn_last_device_error.restype = ctypes.c_int
@@ -225,6 +229,41 @@ def tucker_attn_decode(x, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, Kcache, Vcache, cach
                                     _stream_ptr(dev))
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_attn_decode")
+    return out
+
+
+def tucker_attn_decode_static(x, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, Kcache, Vcache, cache_len, out, *, n_H: int,
+                              rope: bool, rope_base: float = 10000.0, scale: float = 0.0, append: bool = True,
+                              flags: int = 0):
+    """Decode step for callers that cannot allocate: same arguments and result as
+    tucker_attn_decode, but the output tensor `out` [B, d] is mandatory and no workspace is
+    passed -- the library uses its built-in static scratch array (TA_STATIC_SCRATCH_BYTES).
+    Neither this wrapper nor the C entry point allocates device memory.  Raises
+    TuckerAttnError("workspace too small") when the problem needs more scratch than that.
+    Calls share the one array: do not let two of them overlap on the GPU."""
+    torch = _torch()
+    lib = load_library()
+    if x.dim() != 2:
+        raise ValueError("x must be [B, d_model]")
+    B, d = x.shape
+    dev, dt = x.device, x.dtype
+    _check(x, "x", (B, d), dt, dev)
+    r, t = _weights_check((C, U1, U2, U3, Ct, Ut1, Ut2, Ut3), d, n_H, dt, dev)
+    Lmax = Kcache.shape[1]
+    _check(Kcache, "Kcache", (B, Lmax, r[2]), dt, dev)
+    _check(Vcache, "Vcache", (B, Lmax, t[2]), dt, dev)
+    _check(cache_len, "cache_len", (B,), torch.int32, dev)
+    _check(out, "out", (B, d), dt, dev)
+    desc = make_desc(B=B, N=1, d_model=d, n_H=n_H, r=r, t=t, causal=True, rope=rope, rope_base=rope_base,
+                     pos0=0, scale=scale, dtype=_dtype_code(x), flags=flags)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_attn_decode_static(ctypes.byref(desc), x.data_ptr(), C.data_ptr(), U1.data_ptr(),
+                                           U2.data_ptr(), U3.data_ptr(), Ct.data_ptr(), Ut1.data_ptr(),
+                                           Ut2.data_ptr(), Ut3.data_ptr(), Kcache.data_ptr(), Vcache.data_ptr(),
+                                           int(Lmax), cache_len.data_ptr(), int(bool(append)), out.data_ptr(),
+                                           _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_attn_decode_static")
     return out
 
 
