@@ -364,76 +364,161 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------------------------------
-// Sums the split-K partials of the decode projections, applies latent RoPE at position
-// cache_len[b] to the new key, stores bf16 copies for the later kernels, appends to the
-// caches, and writes the (cos, sin) row used for the per-head queries.
-// part: [splits][Mpad][r2 + r3 + t3] fp32 (row b valid for b < B)
+// Per sequence b (one CTA): finishes the new token's latent projections and forms its
+// per-head queries.
+//   row      = sum over the split-K partials of [qt | k | v]            (fp32)
+//   k, v     -> latent RoPE on k at position L = cache_len[b]; bf16 copies for the attention
+//               kernel; appended to the caches at slot L when `append`
+//   w[a, :]  = qt C[a]                        (the core contracted with the query first:
+//   qhat_h   = mult * sum_a U1[h, a] w[a, :]   C x_2 qt x_1 U1, Eq. 9, so that the n_H
+//                                              per-head matrices G_h are never formed)
+//   qhat_h  <- qhat_h R(L, r3), stored bf16 [B, nH, r3]
+// part: [splits][Mpad][r2 + r3 + t3] fp32.  Dynamic shared memory: see dec_qhat_smem().
 // ---------------------------------------------------------------------------------------
-__global__ void k_dec_finish(const float* __restrict__ part, int splits, long split_stride, int B, int r2, int r3,
-                             int t3, bf16* __restrict__ qt, bf16* __restrict__ knew, bf16* __restrict__ vnew,
-                             float2* __restrict__ rope_row, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
-                             const int32_t* __restrict__ cache_len, int rope, double base, int append,
-                             unsigned int* err) {
+__host__ __device__ inline size_t dec_qhat_smem(int nH, int r1, int r2, int r3, int t3) {
+  return sizeof(float) * ((size_t)(r2 + r3 + t3) + (size_t)r1 * r3 + (size_t)nH * r1) + sizeof(float2) * (size_t)(r3 / 2);
+}
+
+__global__ void __launch_bounds__(256)
+k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH, int r1, int r2, int r3, int t3,
+           const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
+           bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
+           const int32_t* __restrict__ cache_len, int rope, double base, int append, unsigned int* err) {
+  extern __shared__ __align__(16) float dq_smem[];
+  const int ncol = r2 + r3 + t3, half = r3 / 2;
+  float2* cs_s = reinterpret_cast<float2*>(dq_smem);   // [r3/2] (cos, sin) at position L
+  float* row = dq_smem + 2 * half;          // [ncol]
+  float* w_s = row + ncol;                  // [r1][r3]
+  float* u1_s = w_s + r1 * r3;              // [nH][r1]
   const int b = blockIdx.x;
-  const int ncol = r2 + r3 + t3;
   int L = cache_len[b];
   if (L < 0 || L >= Lmax) {
     if (threadIdx.x == 0) atomicOr(err, (unsigned)TA_DEVERR_BAD_CACHE_LEN);
     L = clamp_len(L, Lmax);
   }
-  extern __shared__ float row[];   // [ncol]
   for (int c = threadIdx.x; c < ncol; c += blockDim.x) {
     float acc = 0.f;
     for (int s = 0; s < splits; ++s) acc += part[s * split_stride + (long)b * ncol + c];
     row[c] = acc;
   }
-  __syncthreads();
-  for (int c = threadIdx.x; c < r2; c += blockDim.x) qt[(long)b * r2 + c] = __float2bfloat16_rn(row[c]);
-  const int half = r3 / 2;
+  for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
+  for (int i = threadIdx.x; i < r1 * r3; i += blockDim.x) w_s[i] = 0.f;
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    float xe = row[r2 + 2 * i], xo = row[r2 + 2 * i + 1];
     float2 cs = make_float2(1.f, 0.f);
     if (rope) {
-      double theta = pow(base, -2.0 * (double)i / (double)r3);
-      double s, co;
-      sincos((double)L * theta, &s, &co);
-      cs = make_float2((float)co, (float)s);
-      const float ne = xe * cs.x - xo * cs.y, no = xe * cs.y + xo * cs.x;
-      xe = ne; xo = no;
+      const double theta = pow(base, -2.0 * (double)i / (double)r3);
+      double sn, co;
+      sincos((double)L * theta, &sn, &co);
+      cs = make_float2((float)co, (float)sn);
     }
-    rope_row[(long)b * half + i] = cs;
-    const __nv_bfloat162 v = __floats2bfloat162_rn(xe, xo);
+    cs_s[i] = cs;
+  }
+  __syncthreads();
+  // new key (rotated) and value
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    const float xe = row[r2 + 2 * i], xo = row[r2 + 2 * i + 1];
+    const float2 cs = cs_s[i];
+    const __nv_bfloat162 v = __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
     *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + 2 * i) = v;
     if (append) *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + 2 * i) = v;
-  }
-  if (r3 & 1) {   // odd r3 is only possible without RoPE
-    const int c = r3 - 1;
-    if (threadIdx.x == 0) {
-      knew[(long)b * r3 + c] = __float2bfloat16_rn(row[r2 + c]);
-      if (append) Kc[((long)b * Lmax + L) * r3 + c] = __float2bfloat16_rn(row[r2 + c]);
-    }
   }
   for (int c = threadIdx.x; c < t3; c += blockDim.x) {
     const bf16 v = __float2bfloat16_rn(row[r2 + r3 + c]);
     vnew[(long)b * t3 + c] = v;
     if (append) Vc[((long)b * Lmax + L) * t3 + c] = v;
   }
+  // w[a, c] = sum_q qt[q] C[a, q, c].  A thread owns one 16-byte chunk (8 values of c) of the core
+  // rows q = rg, rg + nrg, ... ; the loads of slice a + 1 are issued before the FMAs of slice a so
+  // that a full batch of independent 16-byte loads is always in flight; the row groups of a CTA are
+  // combined with shared-memory atomic adds (w_s was zeroed above).
+  {
+    constexpr int PF = 8;                      // loads in flight per thread and slice
+    const int nch = r3 / 8;                    // 16-byte chunks per core row (r3 is a multiple of 32)
+    const int nrg = blockDim.x / nch;          // row groups
+    const int ch = threadIdx.x % nch, rg = threadIdx.x / nch;
+    if (rg < nrg) {
+      const uint4* Cq = reinterpret_cast<const uint4*>(C);
+      for (int q0 = rg; q0 < r2; q0 += nrg * PF) {
+        uint4 v[PF];
+#pragma unroll
+        for (int u = 0; u < PF; ++u) {
+          const int q = q0 + u * nrg;
+          v[u] = q < r2 ? Cq[(long)q * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        for (int a = 0; a < r1; ++a) {
+          uint4 vn[PF];
+          if (a + 1 < r1) {
+#pragma unroll
+            for (int u = 0; u < PF; ++u) {
+              const int q = q0 + u * nrg;
+              vn[u] = q < r2 ? Cq[((long)(a + 1) * r2 + q) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
+            }
+          }
+          float acc[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll
+          for (int u = 0; u < PF; ++u) {
+            const int q = q0 + u * nrg;
+            const float xq = q < r2 ? row[q] : 0.f;
+            const uint32_t wv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 cv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[e]));
+              acc[2 * e] = fmaf(xq, cv.x, acc[2 * e]);
+              acc[2 * e + 1] = fmaf(xq, cv.y, acc[2 * e + 1]);
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) atomicAdd(&w_s[a * r3 + ch * 8 + e], acc[e]);
+          if (a + 1 < r1) {
+#pragma unroll
+            for (int u = 0; u < PF; ++u) v[u] = vn[u];
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  for (int item = threadIdx.x; item < nH * half; item += blockDim.x) {
+    const int h = item / half, cp = item % half;
+    float xe = 0.f, xo = 0.f;
+    for (int a = 0; a < r1; ++a) {
+      const float u = u1_s[h * r1 + a];
+      xe = fmaf(u, w_s[a * r3 + 2 * cp], xe);
+      xo = fmaf(u, w_s[a * r3 + 2 * cp + 1], xo);
+    }
+    xe *= mult; xo *= mult;
+    const float2 cs = cs_s[cp];
+    *reinterpret_cast<__nv_bfloat162*>(qhat + ((long)b * nH + h) * r3 + 2 * cp) =
+        __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+  }
 }
 
 // ---------------------------------------------------------------------------------------
-// Per sequence: log-sum-exp merge of the partials written by the CTAs whose tile range
-// intersected it, then z[b, j] = sum_{h,c} o_h[c] Gt_h[j, c] for 16 outputs j per CTA.
-// GtP is [t2][nH][t3] bf16; z is bf16 [B, t2].  grid = (t2 / 16, B), 256 threads.
+// Per sequence b (one CTA): log-sum-exp merge of the partials written by the attention CTAs
+// whose tile range intersected the sequence, then the output-side core with the head mode
+// contracted first (the n_H matrices Gt_h are never formed):
+//   o_h      = merged, normalised attention output of head h             [nH][t3]
+//   u[a, :]  = sum_h Ut1[h, a] o_h                                       [t1][t3]
+//   z[j]     = sum_a sum_c Ct[a, j, c] u[a, c]                           [t2]   (= sum_h Gt_h o_h)
+// z is written as bf16 [B, t2].  Dynamic shared memory: see dec_out_smem().
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_dec_merge(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                   const int32_t* __restrict__ cache_len, int B, int Lmax, int nH,
-                                                   int t3, int t2, int grid_attn, const bf16* __restrict__ GtP,
-                                                   bf16* __restrict__ z) {
-  extern __shared__ float sm[];
-  float* o_s = sm;                         // [32][t3]
-  float* w_s = sm + 32 * t3;               // [MAX_GRID][32]
+__host__ __device__ inline size_t dec_out_smem(int nH, int t1, int t3) {
+  return sizeof(float) * (32 * (size_t)t3 + (size_t)MAX_GRID * 32 + (size_t)t1 * t3 + (size_t)nH * t1);
+}
+
+__global__ void __launch_bounds__(256)
+k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ cache_len,
+          int B, int Lmax, int nH, int t1, int t2, int t3, int grid_attn, const bf16* __restrict__ Ct,
+          const bf16* __restrict__ Ut1, bf16* __restrict__ z) {
+  extern __shared__ __align__(16) float do_smem[];
+  float* o_s = do_smem;                    // [32][t3]
+  float* w_s = o_s + 32 * t3;              // [MAX_GRID][32]
+  float* u_s = w_s + MAX_GRID * 32;        // [t1][t3]
+  float* ut1_s = u_s + t1 * t3;            // [nH][t1]
   __shared__ float inv_l[32];
-  const int b = blockIdx.y;
+  const int b = blockIdx.x;
   long total = 0, first = 0;
   for (int i = 0; i < B; ++i) {
     if (i == b) first = total;
@@ -447,6 +532,7 @@ __global__ void __launch_bounds__(256) k_dec_merge(const float* __restrict__ par
   long i1 = i0;
   while (i1 + 1 < grid_attn && cta_first_tile(i1 + 1, total, grid_attn) < first + nt) ++i1;
   const int np = (int)(i1 - i0 + 1);
+  for (int i = threadIdx.x; i < nH * t1; i += blockDim.x) ut1_s[i] = __bfloat162float(Ut1[i]);
   if (threadIdx.x < 32) {
     const int h = threadIdx.x;
     float M = -INFINITY;
@@ -469,31 +555,83 @@ __global__ void __launch_bounds__(256) k_dec_merge(const float* __restrict__ par
     inv_l[h] = 1.f / Lsum;
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < 32 * t3; e += 256) {
-    const int h = e / t3;
-    float acc = 0.f;
+  for (int e4 = threadIdx.x; e4 < nH * t3 / 4; e4 += blockDim.x) {
+    const int h = (e4 * 4) / t3;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int k = 0; k < np; ++k) {
       const float wgt = w_s[k * 32 + h];
-      if (wgt != 0.f) acc += wgt * part_o[(i0 + k + b) * 32 * t3 + e];
+      if (wgt != 0.f) {
+        const float4 v = reinterpret_cast<const float4*>(part_o + (i0 + k + b) * 32 * t3)[e4];
+        acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+      }
     }
-    o_s[e] = acc * inv_l[h];
+    const float il = inv_l[h];
+    reinterpret_cast<float4*>(o_s)[e4] = make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il);
   }
   __syncthreads();
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int n_hc = nH * t3;
-  for (int jj = warp; jj < 16; jj += 8) {
-    const int j = blockIdx.x * 16 + jj;
-    if (j >= t2) break;
-    const bf16* grow = GtP + (long)j * n_hc;
+  for (int e = threadIdx.x; e < t1 * t3; e += blockDim.x) {
+    const int a = e / t3, c = e % t3;
     float acc = 0.f;
-    for (int e = lane * 2; e < n_hc; e += 64) {
-      const __nv_bfloat162 gv = *reinterpret_cast<const __nv_bfloat162*>(grow + e);
-      acc = fmaf(o_s[e], __bfloat162float(gv.x), acc);
-      acc = fmaf(o_s[e + 1], __bfloat162float(gv.y), acc);
+    for (int h = 0; h < nH; ++h) acc = fmaf(ut1_s[h * t1 + a], o_s[h * t3 + c], acc);
+    u_s[e] = acc;
+  }
+  __syncthreads();
+  // z[j] = sum_{a,c} Ct[a, j, c] u[a, c].  A warp takes JB output rows j at a time; its lanes are
+  // split into groups of nch = t3 / 8 lanes, each group reading one core row (a, j, :) in 16-byte
+  // chunks, so that JB * ceil(t1 / rows-per-load) independent loads are in flight per lane.
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int nwarp = blockDim.x / 32;
+  constexpr int JB = 4;
+  const int nch = t3 / 8;                 // 8, 12 or 16
+  const int rpl = 32 / nch;               // core rows per warp-wide load
+  const int la = lane / nch, ch = lane % nch;
+  const bool lane_on = la < rpl;
+  const uint4* Cq = reinterpret_cast<const uint4*>(Ct);
+  for (int j0 = warp * JB; j0 < t2; j0 += nwarp * JB) {
+    float acc[JB];
+#pragma unroll
+    for (int jj = 0; jj < JB; ++jj) acc[jj] = 0.f;
+    if (lane_on) {
+      for (int a0 = la; a0 < t1; a0 += rpl * 4) {
+        uint4 v[4][JB];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int a = a0 + u * rpl;
+#pragma unroll
+          for (int jj = 0; jj < JB; ++jj) {
+            const int j = j0 + jj;
+            v[u][jj] = (a < t1 && j < t2) ? Cq[((long)a * t2 + j) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int a = a0 + u * rpl;
+          if (a < t1) {
+            const float4 u0 = reinterpret_cast<const float4*>(u_s + a * t3 + ch * 8)[0];
+            const float4 u1 = reinterpret_cast<const float4*>(u_s + a * t3 + ch * 8)[1];
+#pragma unroll
+            for (int jj = 0; jj < JB; ++jj) {
+              const uint32_t wv[4] = {v[u][jj].x, v[u][jj].y, v[u][jj].z, v[u][jj].w};
+              const float2 c0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[0]));
+              const float2 c1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[1]));
+              const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[2]));
+              const float2 c3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[3]));
+              float t = acc[jj];
+              t = fmaf(u0.x, c0.x, t); t = fmaf(u0.y, c0.y, t); t = fmaf(u0.z, c1.x, t); t = fmaf(u0.w, c1.y, t);
+              t = fmaf(u1.x, c2.x, t); t = fmaf(u1.y, c2.y, t); t = fmaf(u1.z, c3.x, t); t = fmaf(u1.w, c3.y, t);
+              acc[jj] = t;
+            }
+          }
+        }
+      }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) z[(long)b * t2 + j] = __float2bfloat16_rn(acc);
+    for (int jj = 0; jj < JB; ++jj) {
+      float t = acc[jj];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+      if (lane == 0 && j0 + jj < t2) z[(long)b * t2 + j0 + jj] = __float2bfloat16_rn(t);
+    }
   }
 }
 

@@ -2,8 +2,9 @@
 // projections / per-head queries / output side, and the attention kernel.
 //
 //   prep      G_h (scaled by softmax scale * log2 e) and Gt_h from the cores (C x_1 U1, Definition 2),
-//             stored as K-major B operands; transposed copies of U2, U3, Ut3; RoPE cos/sin table
-//   proj      [Qt | K | V] = X [U2 | U3 | Ut3]   (Sec. 3.1), latent RoPE applied to K in the epilogue
+//             stored as K-major B operands; RoPE cos/sin table
+//   proj      [Qt | K | V] = X [U2 | U3 | Ut3]   (Sec. 3.1), the three factors read in place as
+//             MN-major B operands; latent RoPE applied to K in the epilogue
 //   qhat      Qhat[T, (h, c)] = Qt [G_1 | ... | G_nH], latent RoPE per head in the epilogue (Eq. 12)
 //   attention online softmax over key tiles, one shared latent K / V pair for all heads (Sec. 3.3)
 //   z, y      Z = O [Gt_1; ...; Gt_nH]^T,  Y = Z Ut2^T   (Eqs. 5-6)
@@ -73,21 +74,6 @@ __global__ void k_head_core_bf16(const bf16* __restrict__ C, const bf16* __restr
   }
 }
 
-// dst[c, r] = src[r, c] for src [rows, cols]; 32x32 tiles through shared memory.
-__global__ void k_transpose_bf16(const bf16* __restrict__ src, bf16* __restrict__ dst, int rows, int cols) {
-  __shared__ bf16 t[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-    int r = r0 + i, c = c0 + threadIdx.x;
-    if (r < rows && c < cols) t[i][threadIdx.x] = src[(long)r * cols + c];
-  }
-  __syncthreads();
-  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-    int c = c0 + i, r = r0 + threadIdx.x;
-    if (r < rows && c < cols) dst[(long)c * rows + r] = t[threadIdx.x][i];
-  }
-}
-
 __global__ void k_rope_table_f(float2* __restrict__ tab, int n_pos, int half, int r, int pos0, double base) {
   long total = (long)n_pos * half;
   for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
@@ -109,7 +95,6 @@ int grid_for(long total, int block = 256) {
 // ---- workspace ----------------------------------------------------------------------------
 struct FastWs {
   float2* rope;   // [N][r3/2]
-  bf16* Wt;       // [r2 + r3 + t3, d]   transposed U2 | U3 | Ut3 (K-major B operand)
   bf16* GcatT;    // [n_H * r3, r2]      B operand of the per-head query GEMM
   bf16* GtP;      // [t2, n_H * t3]      B operand of the Z GEMM
   bf16* Qt;       // [T, r2]
@@ -125,7 +110,6 @@ size_t carve_fast(const tucker_attn_desc& d, char* base, FastWs* w) {
   const size_t T = (size_t)d.B * d.N;
   FastWs t;
   t.rope = c.take<float2>(d.rope ? (size_t)d.N * (d.r3 / 2) : 0);
-  t.Wt = c.take<bf16>((size_t)(d.r2 + d.r3 + d.t3) * d.d_model);
   t.GcatT = c.take<bf16>((size_t)d.n_H * d.r3 * d.r2);
   t.GtP = c.take<bf16>((size_t)d.t2 * d.n_H * d.t3);
   t.Qt = c.take<bf16>(T * d.r2);
@@ -145,27 +129,50 @@ int pick_bn(int width) {
   return 32;
 }
 
-// C[M, sum(widths)] = A[M, K] * B^T with B [Ntot, K] K-major (or [K, Ntot] when b_mn_major).
-int launch_gemm(Problem& p, const bf16* A, long lda, const bf16* Bm, long ldb, int M, int K, int Ntot, int BN,
+// One B operand of a GEMM: K-major [n, K] (row = output column) or, with Params::b_mn_major,
+// MN-major [K, n] (row = K index); `ld` = elements between rows.
+struct BOperand {
+  const bf16* ptr;
+  long ld;
+  int n;
+};
+
+// C[M, Ntot] = A[M, K] * B^T, the N range being the concatenation of gp.seg[], each segment
+// taking its columns from B operand seg.bmap starting at column seg.b_n_off.
+int launch_gemm(Problem& p, const bf16* A, long lda, int M, int K, const BOperand* bops, int nb, int Ntot, int BN,
                 umma_gemm::Params gp, int splits = 1) {
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB[3];
   if (!tmap_2d(&tmA, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, 64, 128)) return TA_ERR_CUDA;
-  if (!gp.b_mn_major) {
-    if (!tmap_2d(&tmB, Bm, (uint64_t)K, (uint64_t)Ntot, (uint64_t)ldb, 64, (uint32_t)BN)) return TA_ERR_CUDA;
-  } else {
-    if (!tmap_2d(&tmB, Bm, (uint64_t)Ntot, (uint64_t)K, (uint64_t)ldb, 64, 64)) return TA_ERR_CUDA;
+  for (int i = 0; i < 3; ++i) {
+    const BOperand& b = bops[i < nb ? i : 0];
+    if (!gp.b_mn_major) {
+      if (!tmap_2d(&tmB[i], b.ptr, (uint64_t)K, (uint64_t)b.n, (uint64_t)b.ld, 64, (uint32_t)BN)) return TA_ERR_CUDA;
+    } else {
+      if (!tmap_2d(&tmB[i], b.ptr, (uint64_t)b.n, (uint64_t)K, (uint64_t)b.ld, 64, 64)) return TA_ERR_CUDA;
+    }
   }
+  const int num_kb = gp.kb_per_split > 0 ? gp.kb_per_split : (K + 63) / 64;
   gp.M = M; gp.K = K; gp.BN = BN; gp.err = p.dev_err;
+  gp.stages = num_kb < 3 ? (num_kb < 1 ? 1 : num_kb) : 3;
   static bool attr_set = false;
   if (!attr_set) {
     TA_CUDA_TRY(cudaFuncSetAttribute(umma_gemm::k_umma_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)umma_gemm::SMEM_BYTES));
+                                     (int)umma_gemm::smem_bytes(umma_gemm::MAX_STAGES, umma_gemm::MAX_BN, 1)));
     attr_set = true;
   }
   dim3 grid(Ntot / BN, (M + 127) / 128, splits);
-  umma_gemm::k_umma_gemm<<<grid, umma_gemm::THREADS, umma_gemm::SMEM_BYTES, p.stream>>>(tmA, tmB, gp);
+  umma_gemm::k_umma_gemm<<<grid, umma_gemm::THREADS, umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major), p.stream>>>(
+      tmA, tmB[0], tmB[1], tmB[2], gp);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
+}
+
+// Widest tile width (128 / 96 / 64 / 32) dividing all three widths.
+int common_bn(int a, int b, int c) {
+  const int cand[4] = {128, 96, 64, 32};
+  for (int bn : cand)
+    if (a % bn == 0 && b % bn == 0 && c % bn == 0) return bn;
+  return 0;
 }
 
 bool tmap_3d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t batches, uint64_t ld,
@@ -207,6 +214,7 @@ umma_gemm::Seg seg(int n_begin, int width, int mode, void* out, long ld) {
   umma_gemm::Seg s;
   s.n_begin = n_begin; s.width = width; s.mode = mode; s.out = out; s.ld = ld;
   s.out2 = nullptr; s.ld2 = 0; s.batch2 = 0;
+  s.bmap = 0; s.b_n_off = n_begin;
   return s;
 }
 
@@ -227,7 +235,6 @@ int fast_fwd(Problem& p) {
   FastWs w;
   carve_fast(d, p.ws, &w);
   const int T = d.B * d.N;
-  const bool mn = (d.flags & 0x100) != 0;   // bring-up switch: feed U2/U3/Ut3 untransposed (MN-major B)
   const float LOG2E = 1.4426950408889634f;
   const bool tc_attn = umma_attention_ok(d) && !(d.flags & 0x200);   // 0x200: bring-up switch, FMA attention
 
@@ -238,17 +245,6 @@ int fast_fwd(Problem& p) {
   k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
       (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
   TA_LAUNCH_CHECK(p);
-  if (!mn) {
-    const bf16* srcs[3] = {(const bf16*)p.U2, (const bf16*)p.U3, (const bf16*)p.Ut3};
-    const int widths[3] = {d.r2, d.r3, d.t3};
-    long off = 0;
-    for (int i = 0; i < 3; ++i) {
-      dim3 grid((widths[i] + 31) / 32, (d.d_model + 31) / 32);
-      k_transpose_bf16<<<grid, dim3(32, 8), 0, p.stream>>>(srcs[i], w.Wt + off * d.d_model, d.d_model, widths[i]);
-      TA_LAUNCH_CHECK(p);
-      off += widths[i];
-    }
-  }
   if (d.rope) {
     k_rope_table_f<<<grid_for((long)d.N * (d.r3 / 2)), 256, 0, p.stream>>>(w.rope, d.N, d.r3 / 2, d.r3, d.pos0,
                                                                           (double)d.rope_base);
@@ -256,47 +252,25 @@ int fast_fwd(Problem& p) {
   }
 
   int rc;
-  // ---- latent projections ----
+  // ---- latent projections: one launch, the three factors read in place ([d, r], MN-major B) ----
   {
     umma_gemm::Params gp = {};
     gp.rope_tab = w.rope; gp.n_pos = d.N; gp.rope_half = d.r3 / 2;
+    gp.b_mn_major = 1;
     const int kmode = d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16;
-    if (!mn) {
-      int bn = pick_bn(d.r2);
-      if (pick_bn(d.r3) < bn) bn = pick_bn(d.r3);
-      if (pick_bn(d.t3) < bn) bn = pick_bn(d.t3);
-      if (d.r2 % bn || d.r3 % bn || d.t3 % bn) bn = 32;
-      gp.nseg = 3;
-      gp.seg[0] = seg(0, d.r2, umma_gemm::EP_BF16, w.Qt, d.r2);
-      gp.seg[1] = seg(d.r2, d.r3, kmode, w.K, d.r3);
-      gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_BF16, w.V, d.t3);
-      if (p.Kc) {
-        gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3;
-        gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
-      }
-      if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, w.Wt, d.d_model, T, d.d_model, d.r2 + d.r3 + d.t3, bn, gp)))
-        return rc;
-    } else {
-      // one launch per factor, B read in place as [d, r] (MN-major)
-      struct { const void* U; int width; int mode; bf16* out; void* out2; } job[3] = {
-          {p.U2, d.r2, umma_gemm::EP_BF16, w.Qt, nullptr},
-          {p.U3, d.r3, kmode, w.K, p.Kc},
-          {p.Ut3, d.t3, umma_gemm::EP_BF16, w.V, p.Vc}};
-      for (int i = 0; i < 3; ++i) {
-        umma_gemm::Params g2 = gp;
-        g2.b_mn_major = 1;
-        g2.nseg = 1;
-        g2.seg[0] = seg(0, job[i].width, job[i].mode, job[i].out, job[i].width);
-        if (job[i].out2) {
-          g2.seg[0].out2 = job[i].out2; g2.seg[0].ld2 = job[i].width; g2.seg[0].batch2 = (long)p.Lmax * job[i].width;
-        }
-        const int bn = job[i].width % 128 == 0 ? 128 : 64;
-        if (job[i].width % 64) return TA_ERR_UNSUPPORTED_SHAPE;
-        if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, (const bf16*)job[i].U, job[i].width, T, d.d_model,
-                              job[i].width, bn, g2)))
-          return rc;
-      }
+    const int bn = common_bn(d.r2, d.r3, d.t3);
+    if (!bn) return TA_ERR_UNSUPPORTED_SHAPE;
+    gp.nseg = 3;
+    gp.seg[0] = seg(0, d.r2, umma_gemm::EP_BF16, w.Qt, d.r2);
+    gp.seg[1] = seg(d.r2, d.r3, kmode, w.K, d.r3);
+    gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_BF16, w.V, d.t3);
+    for (int i = 0; i < 3; ++i) { gp.seg[i].bmap = i; gp.seg[i].b_n_off = 0; }
+    if (p.Kc) {
+      gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3;
+      gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
     }
+    const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
+    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, T, d.d_model, bops, 3, d.r2 + d.r3 + d.t3, bn, gp))) return rc;
   }
   // ---- per-head queries with latent RoPE ----
   {
@@ -304,7 +278,8 @@ int fast_fwd(Problem& p) {
     gp.rope_tab = w.rope; gp.n_pos = d.N; gp.rope_half = d.r3 / 2;
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.n_H * d.r3, d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16, w.Qhat, (long)d.n_H * d.r3);
-    if ((rc = launch_gemm(p, w.Qt, d.r2, w.GcatT, d.r2, T, d.r2, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
+    const BOperand bop = {w.GcatT, d.r2, d.n_H * d.r3};
+    if ((rc = launch_gemm(p, w.Qt, d.r2, T, d.r2, &bop, 1, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
   }
   // ---- attention ----
   if (tc_attn) {
@@ -318,15 +293,16 @@ int fast_fwd(Problem& p) {
     gp.n_pos = d.N;
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.t2, umma_gemm::EP_BF16, w.Z, d.t2);
-    if ((rc = launch_gemm(p, w.O, (long)d.n_H * d.t3, w.GtP, (long)d.n_H * d.t3, T, d.n_H * d.t3, d.t2, pick_bn(d.t2), gp)))
-      return rc;
+    const BOperand bop = {w.GtP, (long)d.n_H * d.t3, d.t2};
+    if ((rc = launch_gemm(p, w.O, (long)d.n_H * d.t3, T, d.n_H * d.t3, &bop, 1, d.t2, pick_bn(d.t2), gp))) return rc;
   }
   {
     umma_gemm::Params gp = {};
     gp.n_pos = d.N;
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
-    if ((rc = launch_gemm(p, w.Z, d.t2, (const bf16*)p.Ut2, d.t2, T, d.t2, d.d_model, pick_bn(d.d_model), gp))) return rc;
+    const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
+    if ((rc = launch_gemm(p, w.Z, d.t2, T, d.t2, &bop, 1, d.d_model, pick_bn(d.d_model), gp))) return rc;
   }
   return TA_OK;
 }
@@ -360,10 +336,10 @@ int proj_splits(int d_model) {
 int decode_grid() { return sm_count() < dec::MAX_GRID ? sm_count() : dec::MAX_GRID; }
 
 struct FastDecWs {
-  bf16 *Wt, *GcatT, *GtP;
-  float* proj_part;   // [splits][128][r2 + r3 + t3]
-  bf16 *qt, *knew, *vnew, *qhat, *z;
-  float2* rope_row;   // [B][r3/2]
+  float* proj_part;   // [splits][Mpad][r2 + r3 + t3] split-K partial sums of the new tokens' projections
+  bf16 *knew, *vnew;  // [B][r3] rotated new key, [B][t3] new value
+  bf16* qhat;         // [B][n_H][r3] rotated, scaled per-head queries
+  bf16* z;            // [B][t2]
   float *part_o, *part_ml;
 };
 
@@ -372,16 +348,11 @@ size_t carve_fast_dec(const tucker_attn_desc& d, char* base, FastDecWs* w) {
   FastDecWs t;
   const size_t Mpad = (size_t)((d.B + 127) / 128) * 128;
   const size_t ncol = (size_t)d.r2 + d.r3 + d.t3;
-  t.Wt = c.take<bf16>(ncol * d.d_model);
-  t.GcatT = c.take<bf16>((size_t)d.n_H * d.r3 * d.r2);
-  t.GtP = c.take<bf16>((size_t)d.t2 * d.n_H * d.t3);
   t.proj_part = c.take<float>((size_t)kProjSplits * Mpad * ncol);
-  t.qt = c.take<bf16>((size_t)d.B * d.r2);
   t.knew = c.take<bf16>((size_t)d.B * d.r3);
   t.vnew = c.take<bf16>((size_t)d.B * d.t3);
   t.qhat = c.take<bf16>((size_t)d.B * d.n_H * d.r3);
   t.z = c.take<bf16>((size_t)d.B * d.t2);
-  t.rope_row = c.take<float2>((size_t)d.B * ((d.r3 + 1) / 2));
   const size_t slots = (size_t)dec::MAX_GRID + d.B;
   t.part_o = c.take<float>(slots * 32 * d.t3);
   t.part_ml = c.take<float>(slots * 64);
@@ -415,13 +386,19 @@ bool fast_decode_supported(const tucker_attn_desc& d, int32_t Lmax) {
   auto ok32 = [](int r) { return r >= 32 && r <= 256 && r % 32 == 0; };
   if (!ok32(d.r2) || !ok32(d.t2) || !dec_rank_ok(d.r3, d.t3)) return false;
   if (d.d_model % 64 || d.n_H > 32 || d.B > 4096) return false;
-  if (d.t2 % 16) return false;
+  if (d.r1 > 32 || d.t1 > 32) return false;      // shared-memory tables of the per-sequence kernels
   (void)Lmax;
   return true;
 }
 
 size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t) { return carve_fast_dec(d, nullptr, nullptr); }
 
+// Launch sequence of one decode step (Eq. 9):
+//   1  split-K GEMM   partial [qt | k | v] = x [U2 | U3 | Ut3]           (factors read in place)
+//   2  k_dec_qhat     finish the projections, latent RoPE, cache append, per-head queries
+//   3  k_dec_attn     stream the latent caches once (all heads per tile)
+//   4  k_dec_out      merge the partials, output-side core -> z
+//   5  GEMM           y = z Ut2^T
 int fast_decode(Problem& p) {
   const tucker_attn_desc& d = p.d;
   FastDecWs w;
@@ -431,47 +408,28 @@ int fast_decode(Problem& p) {
   const int Mpad = (d.B + 127) / 128 * 128;
   const int splits = proj_splits(d.d_model);
   int rc;
-  // ---- weight preparation (head-mode core contraction; transposed factors) ----
-  k_head_core_bf16<<<grid_for((long)d.n_H * d.r2 * d.r3), 256, 0, p.stream>>>(
-      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, p.scale * LOG2E);
-  TA_LAUNCH_CHECK(p);
-  k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
-      (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
-  TA_LAUNCH_CHECK(p);
-  {
-    const bf16* srcs[3] = {(const bf16*)p.U2, (const bf16*)p.U3, (const bf16*)p.Ut3};
-    const int widths[3] = {d.r2, d.r3, d.t3};
-    long off = 0;
-    for (int i = 0; i < 3; ++i) {
-      dim3 grid((widths[i] + 31) / 32, (d.d_model + 31) / 32);
-      k_transpose_bf16<<<grid, dim3(32, 8), 0, p.stream>>>(srcs[i], w.Wt + off * d.d_model, d.d_model, widths[i]);
-      TA_LAUNCH_CHECK(p);
-      off += widths[i];
-    }
-  }
-  // ---- projections of the new tokens: split-K partial sums, then finish (RoPE, append) ----
+  // ---- 1: projections of the new tokens, split over K ----
   {
     umma_gemm::Params gp = {};
-    gp.nseg = 1;
-    gp.seg[0] = seg(0, ncol, umma_gemm::EP_F32, w.proj_part, ncol);
+    gp.b_mn_major = 1;
+    gp.nseg = 3;
+    gp.seg[0] = seg(0, d.r2, umma_gemm::EP_F32, w.proj_part, ncol);
+    gp.seg[1] = seg(d.r2, d.r3, umma_gemm::EP_F32, w.proj_part + d.r2, ncol);
+    gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_F32, w.proj_part + d.r2 + d.r3, ncol);
+    for (int i = 0; i < 3; ++i) { gp.seg[i].bmap = i; gp.seg[i].b_n_off = 0; }
     gp.kb_per_split = (d.d_model / 64) / splits;
     gp.split_stride = (long)Mpad * ncol;
-    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, w.Wt, d.d_model, d.B, d.d_model, ncol, 32, gp, splits)))
-      return rc;
+    const int bn = (d.r2 % 64 == 0 && d.r3 % 64 == 0 && d.t3 % 64 == 0) ? 64 : 32;
+    const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
+    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, d.B, d.d_model, bops, 3, ncol, bn, gp, splits))) return rc;
   }
-  dec::k_dec_finish<<<d.B, 128, ncol * sizeof(float), p.stream>>>(
-      w.proj_part, splits, (long)Mpad * ncol, d.B, d.r2, d.r3, d.t3, w.qt, w.knew, w.vnew, w.rope_row, (bf16*)p.Kc,
-      (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, (double)d.rope_base, p.append, p.dev_err);
+  // ---- 2: finish, RoPE, append, per-head queries ----
+  dec::k_dec_qhat<<<d.B, 256, dec::dec_qhat_smem(d.n_H, d.r1, d.r2, d.r3, d.t3), p.stream>>>(
+      w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3, (const bf16*)p.C, (const bf16*)p.U1,
+      p.scale * LOG2E, w.qhat, w.knew, w.vnew, (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope,
+      (double)d.rope_base, p.append, p.dev_err);
   TA_LAUNCH_CHECK(p);
-  // ---- per-head queries, rotated at each sequence's own position ----
-  {
-    umma_gemm::Params gp = {};
-    gp.rope_tab = w.rope_row; gp.n_pos = d.B; gp.rope_half = d.r3 / 2;
-    gp.nseg = 1;
-    gp.seg[0] = seg(0, d.n_H * d.r3, d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16, w.qhat, (long)d.n_H * d.r3);
-    if ((rc = launch_gemm(p, w.qt, d.r2, w.GcatT, d.r2, d.B, d.r2, d.n_H * d.r3, pick_bn(d.r3), gp))) return rc;
-  }
-  // ---- attention over the latent cache ----
+  // ---- 3: attention over the latent cache ----
   {
     CUtensorMap tmK, tmV;
     if (!tmap_3d(&tmK, p.Kc, d.r3, p.Lmax, d.B, d.r3, (uint64_t)p.Lmax * d.r3, 64, 128)) return TA_ERR_CUDA;
@@ -486,19 +444,26 @@ int fast_decode(Problem& p) {
     else if (d.r3 == 128 && d.t3 == 64) rc = launch_dec_attn<128, 64>(p, tmK, tmV, dp);
     else rc = launch_dec_attn<64, 128>(p, tmK, tmV, dp);
     if (rc) return rc;
-    // ---- merge the partials, output-side core ----
-    const size_t smem = sizeof(float) * (32 * (size_t)d.t3 + (size_t)dec::MAX_GRID * 32);
-    dec::k_dec_merge<<<dim3(d.t2 / 16, d.B), 256, smem, p.stream>>>(w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H,
-                                                                    d.t3, d.t2, dp.grid, w.GtP, w.z);
+    // ---- 4: merge the partials, output-side core ----
+    static bool out_attr_set = false;
+    if (!out_attr_set) {
+      TA_CUDA_TRY(cudaFuncSetAttribute(dec::k_dec_out, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)dec::dec_out_smem(32, 32, 128)));
+      out_attr_set = true;
+    }
+    dec::k_dec_out<<<d.B, 256, dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream>>>(
+        w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H, d.t1, d.t2, d.t3, dp.grid, (const bf16*)p.Ct,
+        (const bf16*)p.Ut1, w.z);
     TA_LAUNCH_CHECK(p);
   }
-  // ---- y = z Ut2^T ----
+  // ---- 5: y = z Ut2^T ----
   {
     umma_gemm::Params gp = {};
     gp.n_pos = d.B;
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
-    if ((rc = launch_gemm(p, w.z, d.t2, (const bf16*)p.Ut2, d.t2, d.B, d.t2, d.d_model, pick_bn(d.d_model), gp))) return rc;
+    const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
+    if ((rc = launch_gemm(p, w.z, d.t2, d.B, d.t2, &bop, 1, d.d_model, pick_bn(d.d_model), gp))) return rc;
   }
   return TA_OK;
 }

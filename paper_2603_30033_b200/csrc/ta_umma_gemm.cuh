@@ -19,10 +19,18 @@ using namespace sm100;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 4;
 constexpr int THREADS = 192;
 constexpr int MAX_BN = 128;
-constexpr size_t SMEM_BYTES = 1024 /*align slack*/ + (size_t)STAGES * (BM * BK * 2 + MAX_BN * BK * 2) + 256;
+// Dynamic shared memory of one CTA: the ring is sized for the stage count and tile width of
+// the launch, so that short-K problems (one or two K blocks) leave room for several CTAs
+// per SM and one CTA's epilogue overlaps another's loads and MMAs.
+__host__ __device__ constexpr size_t smem_bytes(int stages, int bn, int b_mn_major) {
+  return 1024 /*align slack*/ +
+         (size_t)stages * (BM * BK * 2 + (size_t)(b_mn_major ? (bn + 63) / 64 * 64 : bn) * BK * 2);
+}
+// TMEM columns to allocate for a tile width (power of two >= 32).
+__host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : (bn <= 64 ? 64u : 128u); }
 
 enum { EP_BF16 = 0, EP_BF16_ROPE = 1, EP_F32 = 2 };
 
@@ -34,10 +42,13 @@ struct Seg {
   long ld;
   void* out2;    // optional second bf16 copy: element (row = b*n_pos + n, c) -> out2[b*batch2 + n*ld2 + c]
   long ld2, batch2;
+  int bmap;      // which B tensor map (0..2) holds this segment's columns
+  int b_n_off;   // N coordinate of the segment's first column inside that map
 };
 
 struct Params {
   int M, K, BN, nseg;
+  int stages;              // ring depth, 1..MAX_STAGES
   int b_mn_major;          // 1: B is given as [K, N] with N contiguous (no transpose needed)
   Seg seg[3];
   const float2* rope_tab;  // [n_pos][rope_half] (cos, sin); EP_BF16_ROPE only
@@ -47,18 +58,24 @@ struct Params {
   unsigned int* err;
 };
 
-__global__ void __launch_bounds__(THREADS, 1)
-k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+__global__ void __launch_bounds__(THREADS, 2)
+k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+            const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const Params p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], acc_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t a_bytes = BM * BK * 2, b_bytes = (uint32_t)p.BN * BK * 2;
-  auto a_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + MAX_BN * BK * 2); };
-  auto b_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + MAX_BN * BK * 2) + a_bytes; };
+  // MN-major B arrives as [64 k-rows x 64 columns] boxes: a tile of BN columns takes ceil(BN / 64) of
+  // them (columns past the tensor's edge are zero-filled by TMA and never multiplied).
+  const int n_bbox = (p.BN + 63) / 64;
+  const uint32_t a_bytes = BM * BK * 2;
+  const uint32_t b_bytes = p.b_mn_major ? (uint32_t)n_bbox * (64 * BK * 2) : (uint32_t)p.BN * BK * 2;
+  auto a_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + b_bytes); };
+  auto b_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + b_bytes) + a_bytes; };
+  const int STAGES = p.stages;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.BN;
@@ -66,6 +83,12 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int kb_begin = p.kb_per_split > 0 ? (int)blockIdx.z * p.kb_per_split : 0;
   const int num_kb = p.kb_per_split > 0 ? min(p.kb_per_split, num_kb_all - kb_begin) : num_kb_all;
   Abort ab{&abort_flag, p.err};
+  // segment of this tile's columns, and where they sit in their B tensor map
+  int si = 0;
+  while (si + 1 < p.nseg && n0 >= p.seg[si + 1].n_begin) ++si;
+  const int bn0 = n0 - p.seg[si].n_begin + p.seg[si].b_n_off;
+  const CUtensorMap* tmB = p.seg[si].bmap == 0 ? &tmB0 : (p.seg[si].bmap == 1 ? &tmB1 : &tmB2);
+  const uint32_t ncols_tmem = tmem_cols(p.BN);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -77,7 +100,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(&tmem_base_slot, 128);
+    tmem_alloc(&tmem_base_slot, ncols_tmem);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -88,7 +111,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 0) {
     if (elect_one()) {
       tma_prefetch_desc(&tmA);
-      tma_prefetch_desc(&tmB);
+      tma_prefetch_desc(tmB);
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
@@ -97,10 +120,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int kx = (kb_begin + kb) * BK;
         tma_load_2d(a_tile(s), &tmA, &full_bar[s], kx, m0);
         if (!p.b_mn_major) {
-          tma_load_2d(b_tile(s), &tmB, &full_bar[s], kx, n0);
+          tma_load_2d(b_tile(s), tmB, &full_bar[s], kx, bn0);
         } else {
-          for (int j = 0; j < p.BN / 64; ++j)   // one [64 k-rows x 64 n] box per 64 columns
-            tma_load_2d(b_tile(s) + j * (64 * BK * 2), &tmB, &full_bar[s], n0 + j * 64, kx);
+          for (int j = 0; j < n_bbox; ++j)   // one [64 k-rows x 64 n] box per 64 columns
+            tma_load_2d(b_tile(s) + j * (64 * BK * 2), tmB, &full_bar[s], bn0 + j * 64, kx);
         }
       }
     }
@@ -141,8 +164,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32)
     const int q = warp % 4;
     const int row = m0 + q * 32 + lane;
-    int si = 0;
-    while (si + 1 < p.nseg && n0 >= p.seg[si + 1].n_begin) ++si;
     const Seg sg = p.seg[si];
     const int c0 = n0 - sg.n_begin;       // first column of this tile inside its segment
     const bool ok = mbar_wait(&acc_bar, 0, ab);
@@ -192,7 +213,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, 128);
+  if (warp == 1) tmem_dealloc(tmem_base, ncols_tmem);
 }
 
 }  // namespace umma_gemm
