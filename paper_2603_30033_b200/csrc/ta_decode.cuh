@@ -364,146 +364,168 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------------------------------
-// Per sequence b (one CTA): finishes the new token's latent projections and forms its
-// per-head queries.
+// k_dec_qhat: grid (B, r3 / 32), 256 threads.  CTA (b, y) finishes the new token's latent
+// projections and forms its per-head queries for the 32 latent key coordinates
+// [32 y, 32 y + 32):
 //   row      = sum over the split-K partials of [qt | k | v]            (fp32)
 //   k, v     -> latent RoPE on k at position L = cache_len[b]; bf16 copies for the attention
 //               kernel; appended to the caches at slot L when `append`
-//   w[a, :]  = qt C[a]                        (the core contracted with the query first:
+//   w[a, c]  = sum_q qt[q] C[a, q, c]         (the core contracted with the query first:
 //   qhat_h   = mult * sum_a U1[h, a] w[a, :]   C x_2 qt x_1 U1, Eq. 9, so that the n_H
 //                                              per-head matrices G_h are never formed)
 //   qhat_h  <- qhat_h R(L, r3), stored bf16 [B, nH, r3]
-// part: [splits][Mpad][r2 + r3 + t3] fp32.  Dynamic shared memory: see dec_qhat_smem().
+// The core is read with 16-byte loads that are all issued before anything waits on them:
+// warp w, lane (rg = lane / 4, ch = lane % 4) owns chunk ch of the CTA's 64-byte column range
+// in the core rows q = 8 w + rg + 64 i, for AB = 16 / NQ slices a at a time (NQ = ceil(r2/64)).
+// part: [splits][Mpad][r2 + r3 + t3] fp32.
 // ---------------------------------------------------------------------------------------
-__host__ __device__ inline size_t dec_qhat_smem(int nH, int r1, int r2, int r3, int t3) {
-  return sizeof(float) * ((size_t)(r2 + r3 + t3) + (size_t)r1 * r3 + (size_t)nH * r1) + sizeof(float2) * (size_t)(r3 / 2);
-}
+constexpr int DQ_CW = 32;       // latent key coordinates per CTA
+constexpr int DQ_MAX_R1 = 32;   // head ranks r1, t1 supported by the shared-memory tables
+constexpr int DQ_MAX_R2 = 256;
 
+template <int NQ>
 __global__ void __launch_bounds__(256)
 k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH, int r1, int r2, int r3, int t3,
            const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
            const int32_t* __restrict__ cache_len, int rope, double base, int append, unsigned int* err) {
-  extern __shared__ __align__(16) float dq_smem[];
-  const int ncol = r2 + r3 + t3, half = r3 / 2;
-  float2* cs_s = reinterpret_cast<float2*>(dq_smem);   // [r3/2] (cos, sin) at position L
-  float* row = dq_smem + 2 * half;          // [ncol]
-  float* w_s = row + ncol;                  // [r1][r3]
-  float* u1_s = w_s + r1 * r3;              // [nH][r1]
-  const int b = blockIdx.x;
+  constexpr int AB = 16 / NQ;                       // core slices per batch
+  __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
+  __shared__ float k_s[DQ_CW];                      // this CTA's coordinates of the new key (unrotated)
+  __shared__ float2 cs_s[DQ_CW / 2];                // (cos, sin) at position L for this CTA's pairs
+  __shared__ float u1_s[32 * DQ_MAX_R1];            // U1 as fp32
+  __shared__ float w_s[DQ_MAX_R1][DQ_CW];
+  __shared__ float red_s[8][AB][DQ_CW];
+  const int b = blockIdx.x, c0 = blockIdx.y * DQ_CW;
+  const int ncol = r2 + r3 + t3;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int rg = lane / 4, ch = lane % 4;
+  const uint4* Cq = reinterpret_cast<const uint4*>(C);
+  const int nch = r3 / 8;                           // 16-byte chunks per core row
+  const int chunk = c0 / 8 + ch;
+
+  auto load_batch = [&](int a0, uint4 (&v)[AB * NQ]) {
+#pragma unroll
+    for (int u = 0; u < AB * NQ; ++u) {
+      const int a = a0 + u / NQ, q = warp * 8 + rg + 64 * (u % NQ);
+      v[u] = (a < r1 && q < r2) ? Cq[((long)a * r2 + q) * nch + chunk] : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  uint4 v[AB * NQ];
+  load_batch(0, v);                                 // in flight while the projections are finished
+
   int L = cache_len[b];
   if (L < 0 || L >= Lmax) {
-    if (threadIdx.x == 0) atomicOr(err, (unsigned)TA_DEVERR_BAD_CACHE_LEN);
+    if (threadIdx.x == 0 && blockIdx.y == 0) atomicOr(err, (unsigned)TA_DEVERR_BAD_CACHE_LEN);
     L = clamp_len(L, Lmax);
   }
-  for (int c = threadIdx.x; c < ncol; c += blockDim.x) {
+  // split-K sums: all of qt, this CTA's 32 key coordinates, and the value coordinates c with
+  // (c / 32) % gridDim.y == blockIdx.y
+  const float* prow = part + (long)b * ncol;
+  for (int c = threadIdx.x; c < r2 + DQ_CW; c += blockDim.x) {
+    const int col = c < r2 ? c : r2 + c0 + (c - r2);
     float acc = 0.f;
-    for (int s = 0; s < splits; ++s) acc += part[s * split_stride + (long)b * ncol + c];
-    row[c] = acc;
+    for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + col];
+    if (c < r2) qt_s[c] = acc; else k_s[c - r2] = acc;
+  }
+  for (int c = threadIdx.x; c < t3; c += blockDim.x) {
+    if ((c / DQ_CW) % gridDim.y != blockIdx.y) continue;
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + r2 + r3 + c];
+    const bf16 vv = __float2bfloat16_rn(acc);
+    vnew[(long)b * t3 + c] = vv;
+    if (append) Vc[((long)b * Lmax + L) * t3 + c] = vv;
   }
   for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
-  for (int i = threadIdx.x; i < r1 * r3; i += blockDim.x) w_s[i] = 0.f;
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+  if (threadIdx.x < DQ_CW / 2) {
     float2 cs = make_float2(1.f, 0.f);
     if (rope) {
-      const double theta = pow(base, -2.0 * (double)i / (double)r3);
+      const double theta = pow(base, -2.0 * (double)(c0 / 2 + threadIdx.x) / (double)r3);
       double sn, co;
       sincos((double)L * theta, &sn, &co);
       cs = make_float2((float)co, (float)sn);
     }
-    cs_s[i] = cs;
+    cs_s[threadIdx.x] = cs;
   }
   __syncthreads();
-  // new key (rotated) and value
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    const float xe = row[r2 + 2 * i], xo = row[r2 + 2 * i + 1];
+  if (threadIdx.x < DQ_CW / 2) {                    // new key, rotated
+    const int i = threadIdx.x;
+    const float xe = k_s[2 * i], xo = k_s[2 * i + 1];
     const float2 cs = cs_s[i];
-    const __nv_bfloat162 v = __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
-    *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + 2 * i) = v;
-    if (append) *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + 2 * i) = v;
+    const __nv_bfloat162 kv = __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+    *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + c0 + 2 * i) = kv;
+    if (append) *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + c0 + 2 * i) = kv;
   }
-  for (int c = threadIdx.x; c < t3; c += blockDim.x) {
-    const bf16 v = __float2bfloat16_rn(row[r2 + r3 + c]);
-    vnew[(long)b * t3 + c] = v;
-    if (append) Vc[((long)b * Lmax + L) * t3 + c] = v;
-  }
-  // w[a, c] = sum_q qt[q] C[a, q, c].  A thread owns one 16-byte chunk (8 values of c) of the core
-  // rows q = rg, rg + nrg, ... ; the loads of slice a + 1 are issued before the FMAs of slice a so
-  // that a full batch of independent 16-byte loads is always in flight; the row groups of a CTA are
-  // combined with shared-memory atomic adds (w_s was zeroed above).
-  {
-    constexpr int PF = 8;                      // loads in flight per thread and slice
-    const int nch = r3 / 8;                    // 16-byte chunks per core row (r3 is a multiple of 32)
-    const int nrg = blockDim.x / nch;          // row groups
-    const int ch = threadIdx.x % nch, rg = threadIdx.x / nch;
-    if (rg < nrg) {
-      const uint4* Cq = reinterpret_cast<const uint4*>(C);
-      for (int q0 = rg; q0 < r2; q0 += nrg * PF) {
-        uint4 v[PF];
+  // ---- w[a, c0 + .] for batches of AB slices ----
+  for (int a0 = 0; a0 < r1; a0 += AB) {
+    float acc[AB][8];
 #pragma unroll
-        for (int u = 0; u < PF; ++u) {
-          const int q = q0 + u * nrg;
-          v[u] = q < r2 ? Cq[(long)q * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
-        }
-        for (int a = 0; a < r1; ++a) {
-          uint4 vn[PF];
-          if (a + 1 < r1) {
+    for (int j = 0; j < AB; ++j)
 #pragma unroll
-            for (int u = 0; u < PF; ++u) {
-              const int q = q0 + u * nrg;
-              vn[u] = q < r2 ? Cq[((long)(a + 1) * r2 + q) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
-            }
-          }
-          float acc[8];
+      for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int u = 0; u < AB * NQ; ++u) {
+      const int q = warp * 8 + rg + 64 * (u % NQ);
+      const float xq = q < r2 ? qt_s[q] : 0.f;
+      const uint32_t wv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
-          for (int u = 0; u < PF; ++u) {
-            const int q = q0 + u * nrg;
-            const float xq = q < r2 ? row[q] : 0.f;
-            const uint32_t wv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float2 cv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[e]));
-              acc[2 * e] = fmaf(xq, cv.x, acc[2 * e]);
-              acc[2 * e + 1] = fmaf(xq, cv.y, acc[2 * e + 1]);
-            }
-          }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) atomicAdd(&w_s[a * r3 + ch * 8 + e], acc[e]);
-          if (a + 1 < r1) {
-#pragma unroll
-            for (int u = 0; u < PF; ++u) v[u] = vn[u];
-          }
-        }
+      for (int e = 0; e < 4; ++e) {
+        const float2 cv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[e]));
+        acc[u / NQ][2 * e] = fmaf(xq, cv.x, acc[u / NQ][2 * e]);
+        acc[u / NQ][2 * e + 1] = fmaf(xq, cv.y, acc[u / NQ][2 * e + 1]);
       }
     }
+    if (a0 + AB < r1) load_batch(a0 + AB, v);       // next batch in flight during the reduction
+#pragma unroll
+    for (int j = 0; j < AB; ++j)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float t = acc[j][e];
+        t += __shfl_xor_sync(0xffffffffu, t, 4);
+        t += __shfl_xor_sync(0xffffffffu, t, 8);
+        t += __shfl_xor_sync(0xffffffffu, t, 16);
+        if (rg == 0) red_s[warp][j][ch * 8 + e] = t;
+      }
+    __syncthreads();
+    for (int i = threadIdx.x; i < AB * DQ_CW; i += blockDim.x) {
+      const int j = i / DQ_CW, c = i % DQ_CW;
+      if (a0 + j < r1) {
+        float t = 0.f;
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) t += red_s[w8][j][c];
+        w_s[a0 + j][c] = t;
+      }
+    }
+    __syncthreads();
   }
-  __syncthreads();
-  for (int item = threadIdx.x; item < nH * half; item += blockDim.x) {
-    const int h = item / half, cp = item % half;
+  // ---- qhat_h for this CTA's coordinates ----
+  for (int item = threadIdx.x; item < nH * (DQ_CW / 2); item += blockDim.x) {
+    const int h = item / (DQ_CW / 2), cp = item % (DQ_CW / 2);
     float xe = 0.f, xo = 0.f;
     for (int a = 0; a < r1; ++a) {
       const float u = u1_s[h * r1 + a];
-      xe = fmaf(u, w_s[a * r3 + 2 * cp], xe);
-      xo = fmaf(u, w_s[a * r3 + 2 * cp + 1], xo);
+      xe = fmaf(u, w_s[a][2 * cp], xe);
+      xo = fmaf(u, w_s[a][2 * cp + 1], xo);
     }
     xe *= mult; xo *= mult;
     const float2 cs = cs_s[cp];
-    *reinterpret_cast<__nv_bfloat162*>(qhat + ((long)b * nH + h) * r3 + 2 * cp) =
+    *reinterpret_cast<__nv_bfloat162*>(qhat + ((long)b * nH + h) * r3 + c0 + 2 * cp) =
         __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
   }
 }
 
 // ---------------------------------------------------------------------------------------
-// Per sequence b (one CTA): log-sum-exp merge of the partials written by the attention CTAs
-// whose tile range intersected the sequence, then the output-side core with the head mode
-// contracted first (the n_H matrices Gt_h are never formed):
+// k_dec_out: grid (B, DO_JS), 256 threads.  Every CTA of a sequence merges the partials of
+// the attention CTAs whose tile range intersected the sequence (log-sum-exp weights), then
+// applies the output-side core with the head mode contracted first (the n_H matrices Gt_h are
+// never formed), for its share of the t2 output coordinates:
 //   o_h      = merged, normalised attention output of head h             [nH][t3]
 //   u[a, :]  = sum_h Ut1[h, a] o_h                                       [t1][t3]
-//   z[j]     = sum_a sum_c Ct[a, j, c] u[a, c]                           [t2]   (= sum_h Gt_h o_h)
+//   z[j]     = sum_a sum_c Ct[a, j, c] u[a, c]                           (= sum_h Gt_h o_h)
 // z is written as bf16 [B, t2].  Dynamic shared memory: see dec_out_smem().
 // ---------------------------------------------------------------------------------------
+constexpr int DO_JS = 4;        // CTAs per sequence (t2 is a multiple of 32, so each gets >= 8 rows)
+
 __host__ __device__ inline size_t dec_out_smem(int nH, int t1, int t3) {
   return sizeof(float) * (32 * (size_t)t3 + (size_t)MAX_GRID * 32 + (size_t)t1 * t3 + (size_t)nH * t1);
 }
@@ -519,6 +541,16 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
   float* ut1_s = u_s + t1 * t3;            // [nH][t1]
   __shared__ float inv_l[32];
   const int b = blockIdx.x;
+  const int jn = t2 / DO_JS, jbeg = blockIdx.y * jn;      // this CTA's output rows [jbeg, jbeg + jn)
+  const int nch = t3 / 8;                  // 16-byte chunks per core row: 8, 12 or 16
+  // pull this CTA's rows of the output core towards L2 while the merge runs
+  {
+    const char* cbase = reinterpret_cast<const char*>(Ct);
+    const long row_bytes = (long)t3 * 2, span = (long)jn * row_bytes;
+    for (int a = 0; a < t1; ++a)
+      for (long off = (long)threadIdx.x * 128; off < span; off += (long)blockDim.x * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(cbase + ((long)a * t2 + jbeg) * row_bytes + off));
+  }
   long total = 0, first = 0;
   for (int i = 0; i < B; ++i) {
     if (i == b) first = total;
@@ -561,8 +593,8 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
     for (int k = 0; k < np; ++k) {
       const float wgt = w_s[k * 32 + h];
       if (wgt != 0.f) {
-        const float4 v = reinterpret_cast<const float4*>(part_o + (i0 + k + b) * 32 * t3)[e4];
-        acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+        const float4 pv = reinterpret_cast<const float4*>(part_o + (i0 + k + b) * 32 * t3)[e4];
+        acc.x += wgt * pv.x; acc.y += wgt * pv.y; acc.z += wgt * pv.z; acc.w += wgt * pv.w;
       }
     }
     const float il = inv_l[h];
@@ -576,62 +608,43 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
     u_s[e] = acc;
   }
   __syncthreads();
-  // z[j] = sum_{a,c} Ct[a, j, c] u[a, c].  A warp takes JB output rows j at a time; its lanes are
-  // split into groups of nch = t3 / 8 lanes, each group reading one core row (a, j, :) in 16-byte
-  // chunks, so that JB * ceil(t1 / rows-per-load) independent loads are in flight per lane.
+  // z[j]: lane group g = lane / nch of warp w owns output row j = jbeg + (w * rpl + g) + 8 * rpl * jj and
+  // walks the slices a with 16-byte loads, PF of them in flight.
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int nwarp = blockDim.x / 32;
-  constexpr int JB = 4;
-  const int nch = t3 / 8;                 // 8, 12 or 16
-  const int rpl = 32 / nch;               // core rows per warp-wide load
-  const int la = lane / nch, ch = lane % nch;
-  const bool lane_on = la < rpl;
+  const int rpl = 32 / nch;                // rows per warp-wide load: 4, 2 or 2
+  const int g = lane / nch, ch = lane % nch;
   const uint4* Cq = reinterpret_cast<const uint4*>(Ct);
-  for (int j0 = warp * JB; j0 < t2; j0 += nwarp * JB) {
-    float acc[JB];
+  constexpr int PF = 8;
+  for (int jl = warp * rpl + (g < rpl ? g : 0); jl < jn; jl += 8 * rpl) {     // uniform trip count per warp
+    const int j = jbeg + jl;
+    float acc = 0.f;
+    for (int a0 = 0; a0 < t1; a0 += PF) {
+      uint4 v[PF];
 #pragma unroll
-    for (int jj = 0; jj < JB; ++jj) acc[jj] = 0.f;
-    if (lane_on) {
-      for (int a0 = la; a0 < t1; a0 += rpl * 4) {
-        uint4 v[4][JB];
+      for (int u = 0; u < PF; ++u)
+        v[u] = (g < rpl && a0 + u < t1) ? Cq[((long)(a0 + u) * t2 + j) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int a = a0 + u * rpl;
-#pragma unroll
-          for (int jj = 0; jj < JB; ++jj) {
-            const int j = j0 + jj;
-            v[u][jj] = (a < t1 && j < t2) ? Cq[((long)a * t2 + j) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int a = a0 + u * rpl;
-          if (a < t1) {
-            const float4 u0 = reinterpret_cast<const float4*>(u_s + a * t3 + ch * 8)[0];
-            const float4 u1 = reinterpret_cast<const float4*>(u_s + a * t3 + ch * 8)[1];
-#pragma unroll
-            for (int jj = 0; jj < JB; ++jj) {
-              const uint32_t wv[4] = {v[u][jj].x, v[u][jj].y, v[u][jj].z, v[u][jj].w};
-              const float2 c0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[0]));
-              const float2 c1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[1]));
-              const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[2]));
-              const float2 c3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[3]));
-              float t = acc[jj];
-              t = fmaf(u0.x, c0.x, t); t = fmaf(u0.y, c0.y, t); t = fmaf(u0.z, c1.x, t); t = fmaf(u0.w, c1.y, t);
-              t = fmaf(u1.x, c2.x, t); t = fmaf(u1.y, c2.y, t); t = fmaf(u1.z, c3.x, t); t = fmaf(u1.w, c3.y, t);
-              acc[jj] = t;
-            }
-          }
+      for (int u = 0; u < PF; ++u) {
+        if (a0 + u < t1) {
+          const float4 u0 = reinterpret_cast<const float4*>(u_s + (a0 + u) * t3 + ch * 8)[0];
+          const float4 u1 = reinterpret_cast<const float4*>(u_s + (a0 + u) * t3 + ch * 8)[1];
+          const uint32_t wv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+          const float2 k0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[0]));
+          const float2 k1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[1]));
+          const float2 k2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[2]));
+          const float2 k3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[3]));
+          acc = fmaf(u0.x, k0.x, acc); acc = fmaf(u0.y, k0.y, acc); acc = fmaf(u0.z, k1.x, acc); acc = fmaf(u0.w, k1.y, acc);
+          acc = fmaf(u1.x, k2.x, acc); acc = fmaf(u1.y, k2.y, acc); acc = fmaf(u1.z, k3.x, acc); acc = fmaf(u1.w, k3.y, acc);
         }
       }
     }
-#pragma unroll
-    for (int jj = 0; jj < JB; ++jj) {
-      float t = acc[jj];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-      if (lane == 0 && j0 + jj < t2) z[(long)b * t2 + j0 + jj] = __float2bfloat16_rn(t);
+    // sum over the nch lanes of the group (groups are aligned to multiples of nch lanes)
+    if (g >= rpl) acc = 0.f;
+    for (int off = 1; off < nch; off <<= 1) {
+      const float t = __shfl_down_sync(0xffffffffu, acc, off);
+      if (ch + off < nch) acc += t;
     }
+    if (g < rpl && ch == 0) z[(long)b * t2 + j] = __float2bfloat16_rn(acc);
   }
 }
 

@@ -395,7 +395,8 @@ size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t) { return carve_
 
 // Launch sequence of one decode step (Eq. 9):
 //   1  split-K GEMM   partial [qt | k | v] = x [U2 | U3 | Ut3]           (factors read in place)
-//   2  k_dec_qhat     finish the projections, latent RoPE, cache append, per-head queries
+//   2  k_dec_qhat     finish the projections, latent RoPE, cache append, per-head queries (core
+//                     contracted with the query first; no per-head G_h)
 //   3  k_dec_attn     stream the latent caches once (all heads per tile)
 //   4  k_dec_out      merge the partials, output-side core -> z
 //   5  GEMM           y = z Ut2^T
@@ -424,11 +425,22 @@ int fast_decode(Problem& p) {
     if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, d.B, d.d_model, bops, 3, ncol, bn, gp, splits))) return rc;
   }
   // ---- 2: finish, RoPE, append, per-head queries ----
-  dec::k_dec_qhat<<<d.B, 256, dec::dec_qhat_smem(d.n_H, d.r1, d.r2, d.r3, d.t3), p.stream>>>(
-      w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3, (const bf16*)p.C, (const bf16*)p.U1,
-      p.scale * LOG2E, w.qhat, w.knew, w.vnew, (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope,
-      (double)d.rope_base, p.append, p.dev_err);
-  TA_LAUNCH_CHECK(p);
+  {
+    const dim3 grid(d.B, d.r3 / dec::DQ_CW);
+    auto launch = [&](auto kernel) {
+      kernel<<<grid, 256, 0, p.stream>>>(w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3,
+                                         (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
+                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, (double)d.rope_base,
+                                         p.append, p.dev_err);
+    };
+    switch ((d.r2 + 63) / 64) {
+      case 1: launch(dec::k_dec_qhat<1>); break;
+      case 2: launch(dec::k_dec_qhat<2>); break;
+      case 3: launch(dec::k_dec_qhat<3>); break;
+      default: launch(dec::k_dec_qhat<4>); break;
+    }
+    TA_LAUNCH_CHECK(p);
+  }
   // ---- 3: attention over the latent cache ----
   {
     CUtensorMap tmK, tmV;
@@ -451,7 +463,7 @@ int fast_decode(Problem& p) {
                                        (int)dec::dec_out_smem(32, 32, 128)));
       out_attr_set = true;
     }
-    dec::k_dec_out<<<d.B, 256, dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream>>>(
+    dec::k_dec_out<<<dim3(d.B, dec::DO_JS), 256, dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream>>>(
         w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H, d.t1, d.t2, d.t3, dp.grid, (const bf16*)p.Ct,
         (const bf16*)p.Ut1, w.z);
     TA_LAUNCH_CHECK(p);
