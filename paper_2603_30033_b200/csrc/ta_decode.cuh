@@ -57,6 +57,18 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// (cos, sin) of pos * base^(-2 i / r).  The angle is formed in double precision (positions of
+// tens of thousands would lose ~1e-3 rad in fp32), reduced to a fraction of a turn in double,
+// and only then handed to the fp32 sincospi.  log2_base = log2(base).
+__device__ __forceinline__ float2 rope_cos_sin(int pos, int i, int r, double log2_base) {
+  const double theta = exp2(-2.0 * (double)i / (double)r * log2_base);
+  double turns = (double)pos * theta * 0.15915494309189535;   // angle / (2 pi)
+  turns -= rint(turns);
+  float sn, co;
+  sincospif((float)(2.0 * turns), &sn, &co);
+  return make_float2(co, sn);
+}
+
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -388,7 +400,7 @@ __global__ void __launch_bounds__(256)
 k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH, int r1, int r2, int r3, int t3,
            const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
-           const int32_t* __restrict__ cache_len, int rope, double base, int append, unsigned int* err) {
+           const int32_t* __restrict__ cache_len, int rope, double log2_base, int append, unsigned int* err) {
   constexpr int AB = 16 / NQ;                       // core slices per batch
   __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
   __shared__ float k_s[DQ_CW];                      // this CTA's coordinates of the new key (unrotated)
@@ -438,14 +450,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
   }
   for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
   if (threadIdx.x < DQ_CW / 2) {
-    float2 cs = make_float2(1.f, 0.f);
-    if (rope) {
-      const double theta = pow(base, -2.0 * (double)(c0 / 2 + threadIdx.x) / (double)r3);
-      double sn, co;
-      sincos((double)L * theta, &sn, &co);
-      cs = make_float2((float)co, (float)sn);
-    }
-    cs_s[threadIdx.x] = cs;
+    cs_s[threadIdx.x] = rope ? rope_cos_sin(L, c0 / 2 + threadIdx.x, r3, log2_base) : make_float2(1.f, 0.f);
   }
   __syncthreads();
   if (threadIdx.x < DQ_CW / 2) {                    // new key, rotated
@@ -540,6 +545,7 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
   float* u_s = w_s + MAX_GRID * 32;        // [t1][t3]
   float* ut1_s = u_s + t1 * t3;            // [nH][t1]
   __shared__ float inv_l[32];
+  __shared__ int on_s[MAX_GRID];
   const int b = blockIdx.x;
   const int jn = t2 / DO_JS, jbeg = blockIdx.y * jn;      // this CTA's output rows [jbeg, jbeg + jn)
   const int nch = t3 / 8;                  // 16-byte chunks per core row: 8, 12 or 16
@@ -565,36 +571,59 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
   while (i1 + 1 < grid_attn && cta_first_tile(i1 + 1, total, grid_attn) < first + nt) ++i1;
   const int np = (int)(i1 - i0 + 1);
   for (int i = threadIdx.x; i < nH * t1; i += blockDim.x) ut1_s[i] = __bfloat162float(Ut1[i]);
+  // which of the np candidate CTAs wrote a partial for this sequence (a CTA whose tile range is
+  // empty wrote nothing: its slot holds stale bytes that must not be used as numbers)
+  for (int k = threadIdx.x; k < np; k += blockDim.x) {
+    const long i = i0 + k;
+    on_s[k] = cta_first_tile(i, total, grid_attn) != cta_first_tile(i + 1, total, grid_attn);
+  }
+  __syncthreads();
   if (threadIdx.x < 32) {
+    // log-sum-exp over the partials of head h; four (max, sum) pairs are loaded at a time
     const int h = threadIdx.x;
-    float M = -INFINITY;
-    for (int k = 0; k < np; ++k) {
-      const long i = i0 + k;
-      if (cta_first_tile(i, total, grid_attn) == cta_first_tile(i + 1, total, grid_attn)) continue;   // empty CTA
-      M = fmaxf(M, part_ml[((i + b) * 32 + h) * 2]);
-    }
-    float Lsum = 0.f;
-    for (int k = 0; k < np; ++k) {
-      const long i = i0 + k;
-      float wgt = 0.f;
-      if (cta_first_tile(i, total, grid_attn) != cta_first_tile(i + 1, total, grid_attn)) {
-        const float m = part_ml[((i + b) * 32 + h) * 2], l = part_ml[((i + b) * 32 + h) * 2 + 1];
-        wgt = (m == -INFINITY) ? 0.f : ex2(m - M);
-        Lsum += wgt * l;
+    const float2* ml = reinterpret_cast<const float2*>(part_ml) + (i0 + b) * 32 + h;
+    float M = -INFINITY, Lsum = 0.f;
+    for (int k0 = 0; k0 < np; k0 += 4) {
+      float2 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = (k0 + u < np) ? ml[(long)(k0 + u) * 32] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (k0 + u < np && on_s[k0 + u] && v[u].x > -INFINITY) {
+          const float Mn = fmaxf(M, v[u].x);
+          Lsum = Lsum * ex2(M - Mn) + v[u].y * ex2(v[u].x - Mn);
+          M = Mn;
+        }
       }
-      w_s[k * 32 + h] = wgt;
+    }
+    for (int k0 = 0; k0 < np; k0 += 4) {
+      float2 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = (k0 + u < np) ? ml[(long)(k0 + u) * 32] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (k0 + u < np) w_s[(k0 + u) * 32 + h] = (on_s[k0 + u] && v[u].x > -INFINITY) ? ex2(v[u].x - M) : 0.f;
     }
     inv_l[h] = 1.f / Lsum;
   }
   __syncthreads();
   for (int e4 = threadIdx.x; e4 < nH * t3 / 4; e4 += blockDim.x) {
     const int h = (e4 * 4) / t3;
+    const float4* po = reinterpret_cast<const float4*>(part_o + (i0 + b) * 32 * t3) + e4;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = 0; k < np; ++k) {
-      const float wgt = w_s[k * 32 + h];
-      if (wgt != 0.f) {
-        const float4 pv = reinterpret_cast<const float4*>(part_o + (i0 + k + b) * 32 * t3)[e4];
-        acc.x += wgt * pv.x; acc.y += wgt * pv.y; acc.z += wgt * pv.z; acc.w += wgt * pv.w;
+    for (int k0 = 0; k0 < np; k0 += 4) {
+      float4 v[4];
+      float wg[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        wg[u] = (k0 + u < np) ? w_s[(k0 + u) * 32 + h] : 0.f;
+        v[u] = (k0 + u < np) ? po[(long)(k0 + u) * 8 * t3] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (wg[u] != 0.f) {     // a zero weight marks a slot whose bytes are not numbers to be used
+          acc.x += wg[u] * v[u].x; acc.y += wg[u] * v[u].y; acc.z += wg[u] * v[u].z; acc.w += wg[u] * v[u].w;
+        }
       }
     }
     const float il = inv_l[h];

@@ -74,16 +74,10 @@ __global__ void k_head_core_bf16(const bf16* __restrict__ C, const bf16* __restr
   }
 }
 
-__global__ void k_rope_table_f(float2* __restrict__ tab, int n_pos, int half, int r, int pos0, double base) {
+__global__ void k_rope_table_f(float2* __restrict__ tab, int n_pos, int half, int r, int pos0, double log2_base) {
   long total = (long)n_pos * half;
-  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
-    int c = (int)(i % half);
-    int n = (int)(i / half);
-    double theta = pow(base, -2.0 * (double)c / (double)r);
-    double s, co;
-    sincos((double)(pos0 + n) * theta, &s, &co);
-    tab[i] = make_float2((float)co, (float)s);
-  }
+  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x)
+    tab[i] = dec::rope_cos_sin(pos0 + (int)(i / half), (int)(i % half), r, log2_base);
 }
 
 int grid_for(long total, int block = 256) {
@@ -247,7 +241,7 @@ int fast_fwd(Problem& p) {
   TA_LAUNCH_CHECK(p);
   if (d.rope) {
     k_rope_table_f<<<grid_for((long)d.N * (d.r3 / 2)), 256, 0, p.stream>>>(w.rope, d.N, d.r3 / 2, d.r3, d.pos0,
-                                                                          (double)d.rope_base);
+                                                                          log2((double)d.rope_base));
     TA_LAUNCH_CHECK(p);
   }
 
@@ -430,7 +424,7 @@ int fast_decode(Problem& p) {
     auto launch = [&](auto kernel) {
       kernel<<<grid, 256, 0, p.stream>>>(w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3,
                                          (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
-                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, (double)d.rope_base,
+                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, log2((double)d.rope_base),
                                          p.append, p.dev_err);
     };
     switch ((d.r2 + 63) / 64) {
