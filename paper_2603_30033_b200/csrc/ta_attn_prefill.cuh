@@ -51,6 +51,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Register budget per warpgroup: the producer / MMA warpgroup gives registers to the two softmax
+// warpgroups, which hold a whole 128-column score row per thread.
+__device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
+__device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
+
 // MN-major B operand (V tile as loaded: rows = keys, 64-column blocks), 128-byte swizzle.
 __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint32_t block_pitch_bytes) {
   uint64_t d = 0;
@@ -116,7 +126,9 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   const uint32_t tm_s[2] = {tmem, tmem + 128};
   const uint32_t tm_o[2] = {tmem + 256, tmem + 384};
 
-  if (warp == 0) {
+  if (warp < 4) {
+   regs_dec();
+   if (warp == 0) {
     // ------------------------------- TMA producer -------------------------------
     if (elect_one()) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -189,7 +201,9 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
       }
     }
-  } else if (warp >= 4) {
+   }
+  } else {
+    regs_inc();
     // ------------------------------- softmax / correction / epilogue -------------
     const int i = (warp - 4) / 4;              // which head of the pair
     const int q = warp % 4;                    // TMEM lane quadrant
@@ -220,9 +234,18 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           for (int c = 0; c < 128; ++c)
             if (k0 + c > lim) sr[c] = 0xff800000u;   // -inf
         }
-        float mt = -INFINITY;
+        float mt;
+        {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;   // four independent chains
 #pragma unroll
-        for (int c = 0; c < 128; ++c) mt = fmaxf(mt, __uint_as_float(sr[c]));
+          for (int c = 0; c < 128; c += 8) {
+            m0 = max3(m0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+            m1 = max3(m1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
+            m2 = max3(m2, __uint_as_float(sr[c + 4]), __uint_as_float(sr[c + 5]));
+            m3 = max3(m3, __uint_as_float(sr[c + 6]), __uint_as_float(sr[c + 7]));
+          }
+          mt = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        }
         const bool need = (mt > m_used + kRescaleThreshold) && (mt > -INFINITY);
         if (__any_sync(0xffffffffu, need)) {
           const float m_new = need ? mt : m_used;
@@ -244,18 +267,23 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           l *= factor;
           m_used = m_new;
         }
-        float rs = 0.f;
-        uint32_t pk[64];
-#pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float p0 = fast_exp2(__uint_as_float(sr[2 * c]) - m_used);
-          const float p1 = fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_used);
-          rs += p0 + p1;
-          pk[c] = pack_bf16(p0, p1);
-        }
-        l += rs;
+        // p = exp2(s - m) two at a time (packed fp32 add), row sum in four packed accumulators;
+        // the bf16 pairs overwrite the score registers in place (pair c lands in sr[c])
         {
-          uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(pk);
+          const float2 negm = make_float2(-m_used, -m_used);
+          float2 rs[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            const float2 x = __fadd2_rn(make_float2(__uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1])), negm);
+            const float2 pp = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+            rs[c & 3] = __fadd2_rn(rs[c & 3], pp);
+            sr[c] = pack_bf16(pp.x, pp.y);
+          }
+          const float2 r01 = __fadd2_rn(rs[0], rs[1]), r23 = __fadd2_rn(rs[2], rs[3]);
+          l += (r01.x + r01.y) + (r23.x + r23.y);
+        }
+        {
+          uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(sr);
           tmem_st32(tm_s[i] + lane_addr + 0, c[0]);
           tmem_st32(tm_s[i] + lane_addr + 32, c[1]);
           tmem_st_wait();
