@@ -189,10 +189,14 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
     }
     kms_avg = sum(kms) / len(kms)
     attn_flops = fl["scores"] + fl["pv"]
+    fused_q = w.dtype == "bf16" and max(w.r[1], w.r[2], w.t[2]) <= 128   # the kernel then also forms the per-head queries
+    if fused_q:
+        attn_flops += fl["qhat"]
     peak = peaks["bf16_tflops"] if w.dtype == "bf16" else None
     ach = attn_flops / (kms_avg * 1e-3) / 1e12
     res["roofline"] = {
-        "kernel": "attention (scores + online softmax + PV)", "bound": "tensor", "achieved": ach, "peak": peak,
+        "kernel": ("attention (per-head queries + scores + online softmax + PV)" if fused_q
+                   else "attention (scores + online softmax + PV)"), "bound": "tensor", "achieved": ach, "peak": peak,
         "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": None, "kernel_ms": kms_avg,
         "flops_per_launch": attn_flops, "whole_step_frac_of_peak": (res["value"] / peak) if peak else None,
     }

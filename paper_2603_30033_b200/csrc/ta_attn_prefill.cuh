@@ -1,22 +1,30 @@
 // Flash-style attention over the latent K / V pair on tcgen05 tensor cores (Sec. 3.3 of the
-// paper: online softmax over key chunks, one K/V chunk pair shared by all heads).
+// paper: online softmax over key chunks, one K/V chunk pair shared by all heads), with the
+// per-head latent queries of Definition 2 formed inside the kernel.
 //
-// One CTA handles one work item = (sequence b, 128 query rows, a pair of heads h, h+1).  Both
-// heads use the same latent K / V tiles, so every tile is loaded once and serves two score
-// tiles; the two softmax warpgroups ping-pong so that the tensor core works on one head
-// while the other head's scores are being exponentiated.
+// One CTA handles one work item = (sequence b, 128 query rows, a run of head pairs).  For every
+// head pair (h, h+1) of its run:
+//   prologue   Qhat_i = Qt G_{h+i} on the tensor core (Qt tile loaded once per CTA, G tiles
+//              streamed through the V ring), latent RoPE applied while the result moves
+//              TMEM -> registers -> shared memory (bf16, the swizzled K-major layout UMMA reads)
+//   main loop  both heads use the same latent K / V tiles, so every tile is loaded once and
+//              serves two score tiles; the two softmax warpgroups ping-pong so that the tensor
+//              core works on one head while the other head's scores are being exponentiated
+//   epilogue   O_i / l written as bf16
+// In the unfused mode (query rank r2 > 128: the Qt tile would not fit) Qhat is read from
+// global memory instead and a CTA handles a single head pair.
 //
-//   warp 0        TMA producer: Qhat tiles (once), K ring, V ring
-//   warp 1        MMA issuer:  S_i = Qhat_i K^T (smem x smem), O_i += P_i V (P from TMEM)
+//   warp 0        TMA producer: Qt (once), G tiles, K ring, V ring
+//   warp 1        MMA issuer:  Qhat_i = Qt G_i^T, S_i = Qhat_i K^T (smem x smem), O_i += P_i V (P from TMEM)
 //   warps 4..7    softmax for head h   : thread t owns query row t (TMEM lane t)
 //   warps 8..11   softmax for head h+1
 //
-// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,256+t3) O_1 [384,384+t3); P_i (bf16, two
-// per column) overwrites the first 64 columns of S_i once the row has been read.
-// Scores arrive in log2 units (softmax scale * log2 e is folded into G_h), so exp2 is used.
-// The running maximum is only raised when it grows by more than 8 (factor 256), which keeps
-// the O rescaling off the common path; l and O stay consistent because both use the same
-// stale maximum.
+// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,256+t3) O_1 [384,384+t3); the prologue
+// result occupies S_i; P_i (bf16, two per column) overwrites the first 64 columns of S_i once
+// the row has been read.  Scores arrive in log2 units (softmax scale * log2 e is folded into
+// G_h), so exp2 is used.  The running maximum is only raised when it grows by more than 8
+// (factor 256), which keeps the O rescaling off the common path; l and O stay consistent
+// because both use the same stale maximum.
 #pragma once
 
 #include "ta_common.cuh"
@@ -31,16 +39,21 @@ constexpr int BQ = 128;        // query rows per tile
 constexpr int BKV = 128;       // keys per tile
 constexpr int THREADS = 384;
 constexpr int SUB_BYTES = 128 * 64 * 2;   // one [128 x 64] bf16 sub-tile (128-byte rows)
-constexpr int MAX_SUB = 2;                 // r3, t3 <= 128
+constexpr int MAX_SUB = 2;                 // r2 (fused), r3, t3 <= 128
 constexpr int KV_STAGES = 2;
 constexpr float kRescaleThreshold = 8.f;
-constexpr size_t SMEM_BYTES = 1024 + (size_t)(2 * MAX_SUB + 2 * KV_STAGES * MAX_SUB) * SUB_BYTES;
+// Qt tile | Qhat_0 | Qhat_1 | K ring | V ring
+constexpr size_t SMEM_BYTES = 1024 + (size_t)(3 * MAX_SUB + 2 * KV_STAGES * MAX_SUB) * SUB_BYTES;
 
 struct Params {
-  int B, N, nH, r3, t3;
+  int B, N, nH, r2, r3, t3;
   int causal;
   int n_qt;          // query tiles per sequence
   int n_hp;          // head pairs
+  int hp_per_item;   // consecutive head pairs handled by one CTA (1 in the unfused mode)
+  int n_hg;          // head-pair groups = ceil(n_hp / hp_per_item)
+  int fused;         // 1: tmQ is the map of Qt [B, N, r2] and Qhat is formed in the prologue
+  const float2* rope;   // [N][r3/2] (cos, sin) for rows of this call, or nullptr (fused mode only)
   bf16* O;           // [B, N, nH, t3]
   unsigned int* err;
 };
@@ -50,7 +63,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -73,32 +85,33 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV, const Params p) {
+k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
+               const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
-  __shared__ uint64_t s_full[2], p_full[2], o_full[2];
+  __shared__ uint64_t s_full[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* q_tile[2] = {tiles, tiles + MAX_SUB * SUB_BYTES};
-  uint8_t* k_ring = tiles + 2 * MAX_SUB * SUB_BYTES;
+  uint8_t* qt_tile = tiles;
+  uint8_t* q_tile[2] = {tiles + MAX_SUB * SUB_BYTES, tiles + 2 * MAX_SUB * SUB_BYTES};
+  uint8_t* k_ring = tiles + 3 * MAX_SUB * SUB_BYTES;
   uint8_t* v_ring = k_ring + KV_STAGES * MAX_SUB * SUB_BYTES;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   // work item: heaviest (largest query tile) first
   int item = blockIdx.x;
-  const int hp = item % p.n_hp; item /= p.n_hp;
+  const int hg = item % p.n_hg; item /= p.n_hg;
   const int b = item % p.B; item /= p.B;
   const int qt = p.n_qt - 1 - item;
   const int q0 = qt * BQ;
-  const int h0 = hp * 2;
-  const bool two = (h0 + 1) < p.nH;
+  const int hp_begin = hg * p.hp_per_item;
+  const int hp_end = min(p.n_hp, hp_begin + p.hp_per_item);
   const int n_kt_all = (p.N + BKV - 1) / BKV;
   const int nt = p.causal ? min(n_kt_all, qt + 1) : n_kt_all;
-  const int ksub = (p.r3 + 63) / 64, vsub = (p.t3 + 63) / 64;
+  const int qsub = (p.r2 + 63) / 64, ksub = (p.r3 + 63) / 64, vsub = (p.t3 + 63) / 64;
   Abort ab{&abort_flag, p.err};
 
   if (threadIdx.x == 0) {
@@ -112,6 +125,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_init(&s_full[i], 1);
       mbar_init(&p_full[i], 4);     // one arrival per softmax warp
       mbar_init(&o_full[i], 1);
+      mbar_init(&qh_done[i], 1);
+      mbar_init(&qh_ready[i], 4);   // one arrival per softmax warp
     }
     fence_barrier_init();
   }
@@ -132,30 +147,52 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     // ------------------------------- TMA producer -------------------------------
     if (elect_one()) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-      mbar_expect_tx(&q_full, (uint32_t)((two ? 2 : 1) * ksub * SUB_BYTES));
-      for (int i = 0; i < (two ? 2 : 1); ++i)
-        for (int kk = 0; kk < ksub; ++kk)
-          tma_load_3d(q_tile[i] + kk * SUB_BYTES, &tmQ, &q_full, (h0 + i) * p.r3 + kk * 64, q0, b);
-      for (int j = 0; j < nt; ++j) {
-        const int s = j % KV_STAGES;
-        const uint32_t ph = (j / KV_STAGES) & 1;
-        if (!mbar_wait(&k_empty[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&k_full[s], (uint32_t)(ksub * SUB_BYTES));
-        for (int kk = 0; kk < ksub; ++kk)
-          tma_load_3d(k_ring + (s * MAX_SUB + kk) * SUB_BYTES, &tmK, &k_full[s], kk * 64, j * BKV, b);
-        if (!mbar_wait(&v_empty[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&v_full[s], (uint32_t)(vsub * SUB_BYTES));
-        for (int kk = 0; kk < vsub; ++kk)
-          tma_load_3d(v_ring + (s * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[s], kk * 64, j * BKV, b);
+      if (p.fused) tma_prefetch_desc(&tmG);
+      int it_k = 0, it_v = 0;          // ring iterations issued so far
+      bool ok = true;
+      for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
+        const int h0 = hp * 2;
+        const int nh = (h0 + 1) < p.nH ? 2 : 1;
+        if (p.fused) {
+          if (hp == hp_begin) {
+            mbar_expect_tx(&q_full, (uint32_t)(qsub * SUB_BYTES));
+            for (int kk = 0; kk < qsub; ++kk) tma_load_3d(qt_tile + kk * SUB_BYTES, &tmQ, &q_full, kk * 64, q0, b);
+          }
+          // G_{h0+i} (stored [r3 rows, r2] K-major) travels through the V ring
+          for (int i = 0; i < nh && ok; ++i, ++it_v) {
+            const int s = it_v % KV_STAGES;
+            if (!(ok = mbar_wait(&v_empty[s], ((it_v / KV_STAGES) & 1) ^ 1, ab))) break;
+            mbar_expect_tx(&v_full[s], (uint32_t)(qsub * p.r3 * 128));
+            for (int kk = 0; kk < qsub; ++kk)
+              tma_load_2d(v_ring + (s * MAX_SUB + kk) * SUB_BYTES, &tmG, &v_full[s], kk * 64, (h0 + i) * p.r3);
+          }
+        } else {
+          mbar_expect_tx(&q_full, (uint32_t)(nh * ksub * SUB_BYTES));
+          for (int i = 0; i < nh; ++i)
+            for (int kk = 0; kk < ksub; ++kk)
+              tma_load_3d(q_tile[i] + kk * SUB_BYTES, &tmQ, &q_full, (h0 + i) * p.r3 + kk * 64, q0, b);
+        }
+        for (int j = 0; j < nt && ok; ++j, ++it_k, ++it_v) {
+          const int sk = it_k % KV_STAGES, sv = it_v % KV_STAGES;
+          if (!(ok = mbar_wait(&k_empty[sk], ((it_k / KV_STAGES) & 1) ^ 1, ab))) break;
+          mbar_expect_tx(&k_full[sk], (uint32_t)(ksub * SUB_BYTES));
+          for (int kk = 0; kk < ksub; ++kk)
+            tma_load_3d(k_ring + (sk * MAX_SUB + kk) * SUB_BYTES, &tmK, &k_full[sk], kk * 64, j * BKV, b);
+          if (!(ok = mbar_wait(&v_empty[sv], ((it_v / KV_STAGES) & 1) ^ 1, ab))) break;
+          mbar_expect_tx(&v_full[sv], (uint32_t)(vsub * SUB_BYTES));
+          for (int kk = 0; kk < vsub; ++kk)
+            tma_load_3d(v_ring + (sv * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[sv], kk * 64, j * BKV, b);
+        }
       }
     }
-  } else if (warp == 1) {
+   } else if (warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (elect_one()) {
       const uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV);
       const uint32_t idesc_pv = umma_idesc_bf16(BQ, (uint32_t)p.t3) | (1u << 16);   // B = V is MN-major
+      const uint32_t idesc_qh = umma_idesc_bf16(BQ, (uint32_t)p.r3);
       const int ksteps = p.r3 / 16;
-      const int nh = two ? 2 : 1;
+      int it_k = 0, it_v = 0, jt = 0;  // ring iterations / tiles consumed so far
       auto issue_qk = [&](int i, int s) {
         const uint32_t qa = smem_u32(q_tile[i]), ka = smem_u32(k_ring + s * MAX_SUB * SUB_BYTES);
         for (int ks = 0; ks < ksteps; ++ks) {
@@ -171,33 +208,60 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                   idesc_pv, (j | ks) != 0);
         umma_commit(&o_full[i]);
       };
-      bool ok = mbar_wait(&q_full, 0, ab);
-      if (ok) ok = mbar_wait(&k_full[0], 0, ab);
-      if (ok) {
-        tc_fence_after();
-        for (int i = 0; i < nh; ++i) issue_qk(i, 0);
-        umma_commit(&k_empty[0]);
-      }
-      for (int j = 0; j < nt && ok; ++j) {
-        const int s = j % KV_STAGES;
-        const uint32_t ph = (j / KV_STAGES) & 1;
-        const int s1 = (j + 1) % KV_STAGES;
-        const uint32_t ph1 = ((j + 1) / KV_STAGES) & 1;
-        const bool more = (j + 1) < nt;
-        if (!(ok = mbar_wait(&v_full[s], ph, ab))) break;
-        for (int i = 0; i < nh && ok; ++i) {
-          if (!(ok = mbar_wait(&p_full[i], (uint32_t)(j & 1), ab))) break;
-          tc_fence_after();
-          issue_pv(i, s, j);
-          if (i == nh - 1) umma_commit(&v_empty[s]);
-          if (more) {
-            if (i == 0) {
-              if (!(ok = mbar_wait(&k_full[s1], ph1, ab))) break;
-              tc_fence_after();
+      bool ok = true;
+      for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
+        const int g = hp - hp_begin;
+        const int nh = (hp * 2 + 1) < p.nH ? 2 : 1;
+        if (p.fused) {
+          if (g == 0 && !(ok = mbar_wait(&q_full, 0, ab))) break;
+          for (int i = 0; i < nh && ok; ++i, ++it_v) {
+            const int s = it_v % KV_STAGES;
+            if (!(ok = mbar_wait(&v_full[s], (it_v / KV_STAGES) & 1, ab))) break;
+            tc_fence_after();
+            const uint32_t qa = smem_u32(qt_tile), ga = smem_u32(v_ring + s * MAX_SUB * SUB_BYTES);
+            for (int ks = 0; ks < p.r2 / 16; ++ks) {
+              const uint32_t off = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
+              umma_ss(tm_s[i], umma_desc_kmajor_sw128(qa + off), umma_desc_kmajor_sw128(ga + off), idesc_qh, ks != 0);
             }
-            issue_qk(i, s1);
-            if (i == nh - 1) umma_commit(&k_empty[s1]);
+            umma_commit(&qh_done[i]);
+            umma_commit(&v_empty[s]);
           }
+          if (!ok) break;
+        } else {
+          if (!(ok = mbar_wait(&q_full, 0, ab))) break;
+        }
+        {
+          const int s = it_k % KV_STAGES;
+          if (!(ok = mbar_wait(&k_full[s], (it_k / KV_STAGES) & 1, ab))) break;
+          for (int i = 0; i < nh && ok; ++i) {
+            if (p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)(g & 1), ab))) break;
+            tc_fence_after();
+            issue_qk(i, s);
+          }
+          if (!ok) break;
+          umma_commit(&k_empty[s]);
+          ++it_k;
+        }
+        for (int j = 0; j < nt && ok; ++j, ++jt, ++it_v) {
+          const int sv = it_v % KV_STAGES;
+          const bool more = (j + 1) < nt;
+          const int sk = it_k % KV_STAGES;
+          if (!(ok = mbar_wait(&v_full[sv], (it_v / KV_STAGES) & 1, ab))) break;
+          for (int i = 0; i < nh && ok; ++i) {
+            if (!(ok = mbar_wait(&p_full[i], (uint32_t)(jt & 1), ab))) break;
+            tc_fence_after();
+            issue_pv(i, sv, j);
+            if (i == nh - 1) umma_commit(&v_empty[sv]);
+            if (more) {
+              if (i == 0) {
+                if (!(ok = mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab))) break;
+                tc_fence_after();
+              }
+              issue_qk(i, sk);
+              if (i == nh - 1) umma_commit(&k_empty[sk]);
+            }
+          }
+          if (more) ++it_k;
         }
       }
     }
@@ -207,13 +271,57 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     // ------------------------------- softmax / correction / epilogue -------------
     const int i = (warp - 4) / 4;              // which head of the pair
     const int q = warp % 4;                    // TMEM lane quadrant
-    if (i == 0 || two) {
-      const int row = q0 + q * 32 + lane;      // query row inside the sequence
-      const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const int rloc = q * 32 + lane;            // row inside the tile
+    const int row = q0 + rloc;                 // query row inside the sequence
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    int jt = 0;                                // tiles consumed so far (parity of s_full / p_full / o_full)
+    bool ok = true;
+    for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
+      const int g = hp - hp_begin;
+      const int h0 = hp * 2;
+      if (i == 1 && (h0 + 1) >= p.nH) break;   // odd head count: the last pair has one head
+      if (p.fused) {
+        // ---- prologue: Qhat row from TMEM, latent RoPE, bf16, swizzled K-major store ----
+        ok = mbar_wait(&qh_done[i], (uint32_t)(g & 1), ab);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const float2* tab = (p.rope && row < p.N) ? p.rope + (long)row * (p.r3 / 2) : nullptr;
+        for (int ch = 0; ch < p.r3 / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tm_s[i] + lane_addr + ch * 32, r);
+          tmem_ld_wait();
+          uint32_t o[16];
+          if (tab) {
+            const float4* t4 = reinterpret_cast<const float4*>(tab + ch * 16);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const float4 cs = t4[c];      // (cos, sin) of two consecutive pairs
+              const float xe0 = __uint_as_float(r[4 * c]), xo0 = __uint_as_float(r[4 * c + 1]);
+              const float xe1 = __uint_as_float(r[4 * c + 2]), xo1 = __uint_as_float(r[4 * c + 3]);
+              o[2 * c] = pack_bf16(xe0 * cs.x - xo0 * cs.y, xe0 * cs.y + xo0 * cs.x);
+              o[2 * c + 1] = pack_bf16(xe1 * cs.z - xo1 * cs.w, xe1 * cs.w + xo1 * cs.z);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) o[c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
+          }
+          uint8_t* dst = q_tile[i] + (ch >> 1) * SUB_BYTES + rloc * 128;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            const int chunk = (ch & 1) * 4 + v;
+            *reinterpret_cast<uint4*>(dst + ((chunk ^ (rloc & 7)) << 4)) =
+                make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+          }
+        }
+        tc_fence_before();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&qh_ready[i]);
+      }
       float m_used = -INFINITY, l = 0.f;
-      bool ok = true;
-      for (int j = 0; j < nt; ++j) {
-        ok = mbar_wait(&s_full[i], (uint32_t)(j & 1), ab);
+      for (int j = 0; j < nt; ++j, ++jt) {
+        ok = mbar_wait(&s_full[i], (uint32_t)(jt & 1), ab);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -251,7 +359,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const float m_new = need ? mt : m_used;
           const float factor = need ? fast_exp2(m_used - m_new) : 1.f;   // exp2(-inf) = 0 on the first tile
           if (j > 0) {
-            ok = mbar_wait(&o_full[i], (uint32_t)((j - 1) & 1), ab);
+            ok = mbar_wait(&o_full[i], (uint32_t)((jt - 1) & 1), ab);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -292,31 +400,30 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[i]);
       }
-      if (ok) {
-        ok = mbar_wait(&o_full[i], (uint32_t)((nt - 1) & 1), ab);
-        ok = __all_sync(0xffffffffu, ok);
-      }
-      if (ok) {
-        tc_fence_after();
-        const float inv = 1.f / l;
-        bf16* dst = p.O + (((long)b * p.N + row) * p.nH + (h0 + i)) * p.t3;
-        for (int ch = 0; ch < p.t3 / 32; ++ch) {
-          uint32_t o[32];
-          tmem_ld32(tm_o[i] + lane_addr + ch * 32, o);
-          tmem_ld_wait();
-          if (row < p.N) {
-            uint4* d4 = reinterpret_cast<uint4*>(dst + ch * 32);
+      if (!ok) break;
+      ok = mbar_wait(&o_full[i], (uint32_t)((jt - 1) & 1), ab);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = 1.f / l;
+      bf16* dst = p.O + (((long)b * p.N + row) * p.nH + (h0 + i)) * p.t3;
+      for (int ch = 0; ch < p.t3 / 32; ++ch) {
+        uint32_t o[32];
+        tmem_ld32(tm_o[i] + lane_addr + ch * 32, o);
+        tmem_ld_wait();
+        if (row < p.N) {
+          uint4* d4 = reinterpret_cast<uint4*>(dst + ch * 32);
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e)
-                w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
-              d4[v] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+            for (int e = 0; e < 4; ++e)
+              w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
+            d4[v] = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
       }
+      tc_fence_before();   // the next head pair's MMAs overwrite S_i / O_i after these reads
     }
   }
   tc_fence_before();

@@ -86,6 +86,13 @@ int grid_for(long total, int block = 256) {
   return (int)(g < 1 ? 1 : g);
 }
 
+bool umma_attention_ok(const tucker_attn_desc& d) { return d.r3 <= 128 && d.t3 <= 128; }
+// The per-head queries are formed inside the attention kernel when the Qt tile fits next to the
+// other tiles in shared memory.
+bool attention_fuses_qhat(const tucker_attn_desc& d) {
+  return umma_attention_ok(d) && d.r2 <= 128 && !(d.flags & (0x200 | 0x400));   // 0x200: FMA attention, 0x400: unfused (bring-up switches)
+}
+
 // ---- workspace ----------------------------------------------------------------------------
 struct FastWs {
   float2* rope;   // [N][r3/2]
@@ -109,7 +116,7 @@ size_t carve_fast(const tucker_attn_desc& d, char* base, FastWs* w) {
   t.Qt = c.take<bf16>(T * d.r2);
   t.K = c.take<bf16>(T * d.r3);
   t.V = c.take<bf16>(T * d.t3);
-  t.Qhat = c.take<bf16>(T * d.n_H * d.r3);
+  t.Qhat = c.take<bf16>(attention_fuses_qhat(d) ? 0 : T * d.n_H * d.r3);
   t.O = c.take<bf16>(T * d.n_H * d.t3);
   t.Z = c.take<bf16>(T * d.t2);
   if (w) *w = t;
@@ -176,19 +183,47 @@ bool tmap_3d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uin
   return make_tmap(m, base, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-bool umma_attention_ok(const tucker_attn_desc& d) { return d.r3 <= 128 && d.t3 <= 128; }
+int sm_count();
 
-int umma_attention(Problem& p, const bf16* Qhat, const bf16* K, const bf16* V, bf16* O) {
+// Consecutive head pairs per CTA.  Causal work items differ in size, so many small items balance
+// best; without a mask all items are equal and a CTA that keeps several head pairs amortises its
+// set-up, as long as the number of waves does not grow.
+int head_pairs_per_item(const tucker_attn_desc& d, int n_qt, int n_hp) {
+  if (d.causal) return 1;
+  const long sms = sm_count();
+  int best = 1;
+  long best_cost = -1;
+  for (int hpi = 1; hpi <= n_hp; ++hpi) {
+    const long items = (long)n_qt * d.B * ((n_hp + hpi - 1) / hpi);
+    const long cost = ((items + sms - 1) / sms) * hpi;
+    if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = hpi; }
+  }
+  return best;
+}
+
+// Q: Qt [T, r2] when the kernel forms Qhat itself (G = GcatT [n_H * r3, r2] then), else Qhat [T, n_H * r3].
+int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const float2* rope, const bf16* K,
+                   const bf16* V, bf16* O) {
   const tucker_attn_desc& d = p.d;
-  CUtensorMap tmQ, tmK, tmV;
-  const uint64_t qcols = (uint64_t)d.n_H * d.r3;
-  if (!tmap_3d(&tmQ, Qhat, qcols, d.N, d.B, qcols, (uint64_t)d.N * qcols, 64, 128)) return TA_ERR_CUDA;
+  CUtensorMap tmQ, tmG, tmK, tmV;
+  if (fused) {
+    if (!tmap_3d(&tmQ, Q, d.r2, d.N, d.B, d.r2, (uint64_t)d.N * d.r2, 64, 128)) return TA_ERR_CUDA;
+    if (!tmap_2d(&tmG, G, (uint64_t)d.r2, (uint64_t)d.n_H * d.r3, (uint64_t)d.r2, 64, (uint32_t)d.r3)) return TA_ERR_CUDA;
+  } else {
+    const uint64_t qcols = (uint64_t)d.n_H * d.r3;
+    if (!tmap_3d(&tmQ, Q, qcols, d.N, d.B, qcols, (uint64_t)d.N * qcols, 64, 128)) return TA_ERR_CUDA;
+    tmG = tmQ;
+  }
   if (!tmap_3d(&tmK, K, d.r3, d.N, d.B, d.r3, (uint64_t)d.N * d.r3, 64, 128)) return TA_ERR_CUDA;
   if (!tmap_3d(&tmV, V, d.t3, d.N, d.B, d.t3, (uint64_t)d.N * d.t3, 64, 128)) return TA_ERR_CUDA;
   attn::Params ap;
-  ap.B = d.B; ap.N = d.N; ap.nH = d.n_H; ap.r3 = d.r3; ap.t3 = d.t3; ap.causal = d.causal;
+  ap.B = d.B; ap.N = d.N; ap.nH = d.n_H; ap.r2 = d.r2; ap.r3 = d.r3; ap.t3 = d.t3; ap.causal = d.causal;
   ap.n_qt = (d.N + attn::BQ - 1) / attn::BQ;
   ap.n_hp = (d.n_H + 1) / 2;
+  ap.hp_per_item = fused ? head_pairs_per_item(d, ap.n_qt, ap.n_hp) : 1;
+  ap.n_hg = (ap.n_hp + ap.hp_per_item - 1) / ap.hp_per_item;
+  ap.fused = fused ? 1 : 0;
+  ap.rope = (fused && d.rope) ? rope : nullptr;
   ap.O = O; ap.err = p.dev_err;
   static bool attr_set = false;
   if (!attr_set) {
@@ -196,9 +231,9 @@ int umma_attention(Problem& p, const bf16* Qhat, const bf16* K, const bf16* V, b
                                      (int)attn::SMEM_BYTES));
     attr_set = true;
   }
-  const long items = (long)ap.n_qt * d.B * ap.n_hp;
+  const long items = (long)ap.n_qt * d.B * ap.n_hg;
   prof_begin(p);
-  attn::k_attn_prefill<<<(unsigned)items, attn::THREADS, attn::SMEM_BYTES, p.stream>>>(tmQ, tmK, tmV, ap);
+  attn::k_attn_prefill<<<(unsigned)items, attn::THREADS, attn::SMEM_BYTES, p.stream>>>(tmQ, tmG, tmK, tmV, ap);
   prof_end(p);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
@@ -266,8 +301,9 @@ int fast_fwd(Problem& p) {
     const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
     if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, T, d.d_model, bops, 3, d.r2 + d.r3 + d.t3, bn, gp))) return rc;
   }
-  // ---- per-head queries with latent RoPE ----
-  {
+  const bool fuse_q = tc_attn && attention_fuses_qhat(d);
+  // ---- per-head queries with latent RoPE (only when the attention kernel does not form them) ----
+  if (!fuse_q) {
     umma_gemm::Params gp = {};
     gp.rope_tab = w.rope; gp.n_pos = d.N; gp.rope_half = d.r3 / 2;
     gp.nseg = 1;
@@ -277,7 +313,7 @@ int fast_fwd(Problem& p) {
   }
   // ---- attention ----
   if (tc_attn) {
-    if ((rc = umma_attention(p, w.Qhat, w.K, w.V, w.O))) return rc;
+    if ((rc = umma_attention(p, fuse_q, fuse_q ? w.Qt : w.Qhat, w.GcatT, w.rope, w.K, w.V, w.O))) return rc;
   } else {
     if ((rc = simt_attention_bf16(p, w.Qhat, w.K, w.V, w.O))) return rc;
   }

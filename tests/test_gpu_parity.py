@@ -95,6 +95,11 @@ FAST = [
     dict(B=3, N=128, d_model=256, n_H=8, r=(8, 128, 128), t=(8, 128, 128), causal=True, rope=True),
     dict(B=2, N=77, d_model=64, n_H=2, r=(2, 32, 32), t=(2, 96, 96), causal=True, rope=False),
     dict(B=1, N=1, d_model=64, n_H=2, r=(2, 64, 64), t=(2, 64, 64), causal=True, rope=True),
+    # query rank above 128: per-head queries come from the separate GEMM, not the attention prologue
+    dict(B=2, N=150, d_model=256, n_H=4, r=(4, 256, 64), t=(4, 64, 64), causal=True, rope=True),
+    # no mask: one CTA walks several head pairs; odd head count ends on a single head
+    dict(B=2, N=197, d_model=192, n_H=3, r=(3, 64, 96), t=(3, 96, 96), causal=False, rope=True),
+    dict(B=3, N=260, d_model=384, n_H=12, r=(4, 96, 96), t=(4, 96, 96), causal=False, rope=False),
 ]
 
 
@@ -105,6 +110,18 @@ def test_small_shapes_tensor_core_path(shape):
     got = gpu_fwd(X, wt, w, pos0=3)
     assert Bd.last_path() == 2
     check(got, oracle_fwd(X, wt, w, pos0=3), "bf16", str(shape), scaled=True)
+
+
+def test_fused_and_unfused_query_paths_agree():
+    # the attention kernel forming Qhat in its prologue vs reading it from the query GEMM
+    w = H.custom_workload(dtype="bf16", B=2, N=300, d_model=256, n_H=8, r=(3, 128, 128), t=(3, 64, 128), causal=True,
+                          rope=True, rope_base=500000.0, seed=91)
+    X, wt = H.host_inputs(w)
+    ref = oracle_fwd(X, wt, w, pos0=1000)
+    for flags in (0, 0x400):
+        got = gpu_fwd(X, wt, w, flags=flags, pos0=1000)
+        assert Bd.last_path() == 2
+        check(got, ref, "bf16", f"flags={flags}", scaled=True)
 
 
 def test_tensor_core_path_writes_cache():
