@@ -59,14 +59,29 @@ bool tmap_2d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uin
 }
 
 // ---- weight preparation -------------------------------------------------------------------
-// out[(h*sh + b*sb + c*sc)] = bf16(mult * sum_a U1[h,a] C[a,b,c])
-__global__ void k_head_core_bf16(const bf16* __restrict__ C, const bf16* __restrict__ U1, bf16* __restrict__ out,
-                                 int nH, int r1, int rb, int rc, long sh, long sb, long sc, float mult) {
-  long total = (long)nH * rb * rc;
-  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
-    int c = (int)(i % rc);
-    int b = (int)((i / rc) % rb);
-    int h = (int)(i / ((long)rc * rb));
+// One launch for everything that depends on the weights and positions only:
+//   blocks [0, g1)        G^T : GcatT[h, c, b] = bf16(mult * sum_a U1[h,a] C[a,b,c])     (C x_1 U1, Definition 2)
+//   blocks [g1, g1+g2)    Gt  : GtP[j, h, c]   = bf16(sum_a Ut1[h,a] Ct[a,j,c])
+//   blocks [g1+g2, ...)   (cos, sin) table for positions pos0 .. pos0 + n_pos - 1
+struct PrepParams {
+  const bf16 *C, *U1, *Ct, *Ut1;
+  bf16 *GcatT, *GtP;
+  float2* rope;
+  int nH, r1, r2, r3, t1, t2, t3;
+  int n_pos, pos0;
+  float mult;
+  double log2_base;
+  int g1, g2, g3;
+};
+
+__device__ __forceinline__ void head_core_part(const bf16* __restrict__ C, const bf16* __restrict__ U1,
+                                               bf16* __restrict__ out, int nH, int r1, int rb, int rc, long sh, long sb,
+                                               long sc, float mult, int block, int nblocks) {
+  const long total = (long)nH * rb * rc;
+  for (long i = block * (long)blockDim.x + threadIdx.x; i < total; i += (long)nblocks * blockDim.x) {
+    const int c = (int)(i % rc);
+    const int b = (int)((i / rc) % rb);
+    const int h = (int)(i / ((long)rc * rb));
     float acc = 0.f;
     for (int a = 0; a < r1; ++a)
       acc = fmaf(__bfloat162float(U1[(long)h * r1 + a]), __bfloat162float(C[((long)a * rb + b) * rc + c]), acc);
@@ -74,10 +89,18 @@ __global__ void k_head_core_bf16(const bf16* __restrict__ C, const bf16* __restr
   }
 }
 
-__global__ void k_rope_table_f(float2* __restrict__ tab, int n_pos, int half, int r, int pos0, double log2_base) {
-  long total = (long)n_pos * half;
-  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x)
-    tab[i] = dec::rope_cos_sin(pos0 + (int)(i / half), (int)(i % half), r, log2_base);
+__global__ void __launch_bounds__(256) k_prefill_prep(const PrepParams p) {
+  const int blk = blockIdx.x;
+  if (blk < p.g1) {
+    head_core_part(p.C, p.U1, p.GcatT, p.nH, p.r1, p.r2, p.r3, (long)p.r3 * p.r2, 1, p.r2, p.mult, blk, p.g1);
+  } else if (blk < p.g1 + p.g2) {
+    head_core_part(p.Ct, p.Ut1, p.GtP, p.nH, p.t1, p.t2, p.t3, p.t3, (long)p.nH * p.t3, 1, 1.f, blk - p.g1, p.g2);
+  } else {
+    const int half = p.r3 / 2;
+    const long total = (long)p.n_pos * half;
+    for (long i = (blk - p.g1 - p.g2) * (long)blockDim.x + threadIdx.x; i < total; i += (long)p.g3 * blockDim.x)
+      p.rope[i] = dec::rope_cos_sin(p.pos0 + (int)(i / half), (int)(i % half), p.r3, p.log2_base);
+  }
 }
 
 int grid_for(long total, int block = 256) {
@@ -267,16 +290,19 @@ int fast_fwd(Problem& p) {
   const float LOG2E = 1.4426950408889634f;
   const bool tc_attn = umma_attention_ok(d) && !(d.flags & 0x200);   // 0x200: bring-up switch, FMA attention
 
-  // ---- weight preparation ----
-  k_head_core_bf16<<<grid_for((long)d.n_H * d.r2 * d.r3), 256, 0, p.stream>>>(
-      (const bf16*)p.C, (const bf16*)p.U1, w.GcatT, d.n_H, d.r1, d.r2, d.r3, (long)d.r3 * d.r2, 1, d.r2, tc_attn ? p.scale * LOG2E : p.scale);
-  TA_LAUNCH_CHECK(p);
-  k_head_core_bf16<<<grid_for((long)d.n_H * d.t2 * d.t3), 256, 0, p.stream>>>(
-      (const bf16*)p.Ct, (const bf16*)p.Ut1, w.GtP, d.n_H, d.t1, d.t2, d.t3, d.t3, (long)d.n_H * d.t3, 1, 1.f);
-  TA_LAUNCH_CHECK(p);
-  if (d.rope) {
-    k_rope_table_f<<<grid_for((long)d.N * (d.r3 / 2)), 256, 0, p.stream>>>(w.rope, d.N, d.r3 / 2, d.r3, d.pos0,
-                                                                          log2((double)d.rope_base));
+  // ---- weight preparation: head-mode core contractions and the RoPE table, one launch ----
+  {
+    PrepParams pp;
+    pp.C = (const bf16*)p.C; pp.U1 = (const bf16*)p.U1; pp.Ct = (const bf16*)p.Ct; pp.Ut1 = (const bf16*)p.Ut1;
+    pp.GcatT = w.GcatT; pp.GtP = w.GtP; pp.rope = w.rope;
+    pp.nH = d.n_H; pp.r1 = d.r1; pp.r2 = d.r2; pp.r3 = d.r3; pp.t1 = d.t1; pp.t2 = d.t2; pp.t3 = d.t3;
+    pp.n_pos = d.N; pp.pos0 = d.pos0;
+    pp.mult = tc_attn ? p.scale * LOG2E : p.scale;
+    pp.log2_base = d.rope ? log2((double)d.rope_base) : 0.0;
+    pp.g1 = grid_for((long)d.n_H * d.r2 * d.r3);
+    pp.g2 = grid_for((long)d.n_H * d.t2 * d.t3);
+    pp.g3 = d.rope ? grid_for((long)d.N * (d.r3 / 2)) : 0;
+    k_prefill_prep<<<pp.g1 + pp.g2 + pp.g3, 256, 0, p.stream>>>(pp);
     TA_LAUNCH_CHECK(p);
   }
 

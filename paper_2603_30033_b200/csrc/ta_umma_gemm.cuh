@@ -25,9 +25,11 @@ constexpr int MAX_BN = 128;
 // Dynamic shared memory of one CTA: the ring is sized for the stage count and tile width of
 // the launch, so that short-K problems (one or two K blocks) leave room for several CTAs
 // per SM and one CTA's epilogue overlaps another's loads and MMAs.
+// The epilogue reuses the ring as a [128][BN + 8] bf16 staging tile, so the ring is never smaller than that.
 __host__ __device__ constexpr size_t smem_bytes(int stages, int bn, int b_mn_major) {
-  return 1024 /*align slack*/ +
-         (size_t)stages * (BM * BK * 2 + (size_t)(b_mn_major ? (bn + 63) / 64 * 64 : bn) * BK * 2);
+  const size_t ring = (size_t)stages * (BM * BK * 2 + (size_t)(b_mn_major ? (bn + 63) / 64 * 64 : bn) * BK * 2);
+  const size_t stage_tile = (size_t)BM * (bn + 8) * 2;
+  return 1024 /*align slack*/ + (ring > stage_tile ? ring : stage_tile);
 }
 // TMEM columns to allocate for a tile width (power of two >= 32).
 __host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : (bn <= 64 ? 64u : 128u); }
@@ -169,43 +171,68 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const bool ok = mbar_wait(&acc_bar, 0, ab);
     tc_fence_after();
     if (ok) {
-      const int nb = p.n_pos > 0 ? row / p.n_pos : 0;
+      const int rloc = q * 32 + lane;
       const int npos = p.n_pos > 0 ? row % p.n_pos : row;
-      for (int ch = 0; ch < p.BN / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
-        tmem_ld_wait();
-        if (row >= p.M) continue;
-        const int col = c0 + ch * 32;
-        if (sg.mode == EP_F32) {
+      if (sg.mode == EP_F32) {
+        for (int ch = 0; ch < p.BN / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
+          tmem_ld_wait();
+          if (row >= p.M) continue;
           float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)blockIdx.z * p.split_stride +
-                                                  (long)row * sg.ld + col);
+                                                  (long)row * sg.ld + c0 + ch * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
                                  __uint_as_float(r[4 * i + 3]));
-        } else {
+        }
+      } else {
+        // bf16 outputs: every thread converts its own accumulator row into a staging tile in shared
+        // memory (the ring is idle once the accumulator is complete; rows padded by 16 bytes keep the
+        // 16-byte stores of a quarter-warp on distinct banks), then each warp writes its 32 rows out
+        // with full-row, coalesced 16-byte stores.
+        const int pitch = (p.BN + 8) * 2;
+        uint8_t* stage = tiles;
+        for (int ch = 0; ch < p.BN / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
+          tmem_ld_wait();
+          const int col = c0 + ch * 32;
           uint32_t o[16];
           if (sg.mode == EP_BF16_ROPE) {
             const int period = 2 * p.rope_half;
             const float2* tab = p.rope_tab + (long)npos * p.rope_half + ((col % period) >> 1);
+            if (row < p.M) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float2 cs = tab[i];
-              const float xe = __uint_as_float(r[2 * i]), xo = __uint_as_float(r[2 * i + 1]);
-              o[i] = pack_bf16(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+              for (int i = 0; i < 16; ++i) {
+                const float2 cs = tab[i];
+                const float xe = __uint_as_float(r[2 * i]), xo = __uint_as_float(r[2 * i + 1]);
+                o[i] = pack_bf16(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+              }
             }
           } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
           }
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)row * sg.ld + col);
+          uint4* sdst = reinterpret_cast<uint4*>(stage + (size_t)rloc * pitch + ch * 64);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-          if (sg.out2) {
-            uint4* d2 = reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)nb * sg.batch2 + (long)npos * sg.ld2 + col);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) d2[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          for (int i = 0; i < 4; ++i) sdst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        }
+        __syncwarp();
+        const int cpr = p.BN / 8;            // 16-byte chunks per row
+        const int rpi = 32 / cpr;            // rows written per warp-wide store
+        const int rsub = lane / cpr, cc = lane % cpr;
+        if (rsub < rpi) {
+          for (int r0 = 0; r0 < 32; r0 += rpi) {
+            const int rr = q * 32 + r0 + rsub;
+            const int grow = m0 + rr;
+            if (grow >= p.M) break;
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)rr * pitch + cc * 16);
+            *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + c0 + cc * 8) = v;
+            if (sg.out2) {
+              const int gb = p.n_pos > 0 ? grow / p.n_pos : 0, gn = p.n_pos > 0 ? grow % p.n_pos : grow;
+              *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)gb * sg.batch2 + (long)gn * sg.ld2 + c0 + cc * 8) = v;
+            }
           }
         }
       }
