@@ -358,7 +358,9 @@ int fast_fwd(Problem& p) {
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
     const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
-    if ((rc = launch_gemm(p, w.Z, d.t2, T, d.t2, &bop, 1, d.d_model, pick_bn(d.d_model), gp))) return rc;
+    // short K (t2) and a wide N: 256-wide tiles halve the number of CTAs and of A-tile reads
+    const int bn = (d.d_model % 256 == 0) ? 256 : pick_bn(d.d_model);
+    if ((rc = launch_gemm(p, w.Z, d.t2, T, d.t2, &bop, 1, d.d_model, bn, gp))) return rc;
   }
   return TA_OK;
 }

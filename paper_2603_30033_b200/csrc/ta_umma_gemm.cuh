@@ -1,6 +1,6 @@
 // C[M, N] = A[M, K] * B[N, K]^T on the 5th-generation tensor cores (tcgen05.mma, bf16 inputs,
 // fp32 accumulation in TMEM), operands streamed by TMA through a shared-memory ring.
-// One CTA computes one 128 x BN output tile:
+// One CTA computes one 128 x BN output tile (BN a multiple of 32, at most 256):
 //   warp 0      TMA producer (one elected lane)
 //   warp 1      TMEM allocation + MMA issue (one elected lane)
 //   warps 2..5  epilogue: TMEM -> registers -> global, one TMEM lane quadrant each
@@ -21,7 +21,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int MAX_STAGES = 4;
 constexpr int THREADS = 192;
-constexpr int MAX_BN = 128;
+constexpr int MAX_BN = 256;
 // Dynamic shared memory of one CTA: the ring is sized for the stage count and tile width of
 // the launch, so that short-K problems (one or two K blocks) leave room for several CTAs
 // per SM and one CTA's epilogue overlaps another's loads and MMAs.
@@ -32,7 +32,7 @@ __host__ __device__ constexpr size_t smem_bytes(int stages, int bn, int b_mn_maj
   return 1024 /*align slack*/ + (ring > stage_tile ? ring : stage_tile);
 }
 // TMEM columns to allocate for a tile width (power of two >= 32).
-__host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : (bn <= 64 ? 64u : 128u); }
+__host__ __device__ constexpr uint32_t tmem_cols(int bn) { return bn <= 32 ? 32u : (bn <= 64 ? 64u : (bn <= 128 ? 128u : 256u)); }
 
 enum { EP_BF16 = 0, EP_BF16_ROPE = 1, EP_F32 = 2 };
 
