@@ -36,6 +36,13 @@ from paper_2603_30033_b200 import workloads as W
 METRIC = "prefill TFLOP/s & decode GB/s vs B200 roofline (fused Tucker attention)"
 KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
 L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on
+# this workload (profiles/).  A value is only listed while the kernel is unchanged since its capture.
+NCU_TRAFFIC_BYTES = {
+    "c4_long_prefill": 17.94e6 + 83.58e6,     # attn::k_attn_prefill, profiles/k_attn_prefill_c4_long_prefill.md
+    "c3_vit_prefill": 29.95e6 + 64.85e6,      # attn::k_attn_prefill, profiles/k_attn_prefill_c3_vit_prefill.md
+    "c5_decode": 1075.01e6 + 4.69e6,          # dec::k_dec_attn<128,128>, profiles/k_dec_attn_c5_decode.md
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -197,7 +204,7 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
     res["roofline"] = {
         "kernel": ("attention (per-head queries + scores + online softmax + PV)" if fused_q
                    else "attention (scores + online softmax + PV)"), "bound": "tensor", "achieved": ach, "peak": peak,
-        "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": None, "kernel_ms": kms_avg,
+        "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": NCU_TRAFFIC_BYTES.get(w.name), "kernel_ms": kms_avg,
         "flops_per_launch": attn_flops, "whole_step_frac_of_peak": (res["value"] / peak) if peak else None,
     }
     res["clocks"] = clocks
@@ -257,7 +264,7 @@ def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sam
     ach = by["cache"] / (kms_avg * 1e-3) / 1e9
     res["roofline"] = {
         "kernel": "decode attention over the latent KV cache", "bound": "hbm", "achieved": ach,
-        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
         "kernel_ms": kms_avg, "bytes_per_launch": by["cache"],
         "whole_step_frac_of_peak": res["value"] / peaks["hbm_gbs"],
     }
@@ -358,6 +365,22 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Slowest rank sets the time: element-wise MAX of a list of per-rank floats over the process
+    group (identity without one).  Works with NCCL (device tensors) and gloo (CPU tensors)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_value(work_per_rank, world, ms):
+    """Units all ranks processed (independent replicas: world x the per-rank work) per second."""
+    return world * work_per_rank / (ms * 1e-3)
+
+
 def _cfg(w):
     return {"kind": w.kind, "B": w.B, "N_or_cache_len": w.N, "d_model": w.d_model, "n_H": w.n_H,
             "ranks_qk": list(w.r), "ranks_vo": list(w.t), "causal": w.causal, "rope": w.rope,
@@ -409,16 +432,11 @@ def main():
             gpu_index = local_rank
     res = fn(w, args.steps, args.warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=ClockSampler(gpu_index))
 
-    ms = res["ms_per_step"]
-    e2e_ms = res["e2e"]["ms_per_step"]
-    if dist is not None:
-        t = torch.tensor([ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([res["ms_per_step"], res["e2e"]["ms_per_step"]], dist, "cuda")
     work = res.get("flops_per_step", res.get("bytes_per_step"))
     div = 1e12 if w.kind == "prefill" else 1e9
-    value = world * work / (ms * 1e-3) / div
-    e2e_value = world * work / (e2e_ms * 1e-3) / div
+    value = whole_job_value(work, world, ms) / div
+    e2e_value = whole_job_value(work, world, e2e_ms) / div
 
     others = []
     if not args.no_others and world == 1:
