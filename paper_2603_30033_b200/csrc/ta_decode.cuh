@@ -57,6 +57,53 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Block-wide scan over the tile counts of all sequences.  Thread t owns the sequences
+// [lo, hi) = [t * chunk, (t + 1) * chunk); returns the total number of tiles and sets `excl` to the
+// number of tiles before sequence `lo`.  wtot_s needs one slot per warp of the block; contains a
+// __syncthreads.
+__device__ __forceinline__ long block_tile_scan(const int32_t* __restrict__ cache_len, int B, int Lmax, int& lo,
+                                                int& hi, long& excl, long long* wtot_s) {
+  const int nthr = blockDim.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarp = (nthr + 31) >> 5;
+  const int chunk = (B + nthr - 1) / nthr;
+  lo = min(B, tid * chunk);
+  hi = min(B, lo + chunk);
+  long long cnt = 0;
+  for (int b = lo; b < hi; ++b) cnt += tiles_of(clamp_len(cache_len[b], Lmax));
+  long long incl = cnt;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const long long v = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += v;
+  }
+  if (lane == 31) wtot_s[wid] = incl;
+  __syncthreads();
+  long long before = 0, total = 0;
+  for (int w = 0; w < nwarp; ++w) {
+    const long long v = wtot_s[w];
+    if (w < wid) before += v;
+    total += v;
+  }
+  excl = (long)(before + incl - cnt);
+  return (long)total;
+}
+
+// (cos, sin) of pos * theta for a rotation frequency theta given in double precision: the angle is
+// reduced to a fraction of a turn in double (positions of tens of thousands would lose ~1e-3 rad
+// in fp32) and only then handed to the fp32 sincospi.
+__device__ __forceinline__ float2 rope_cos_sin_theta(int pos, double theta) {
+  double turns = (double)pos * theta * 0.15915494309189535;   // angle / (2 pi)
+  turns -= rint(turns);
+  float sn, co;
+  sincospif((float)(2.0 * turns), &sn, &co);
+  return make_float2(co, sn);
+}
+
+// Rotation frequencies theta_i = base^(-2 i / r), i < r / 2 <= 128, computed on the host in double
+// precision and passed to the kernels by value.
+struct RopeFreqs {
+  double theta[128];
+};
+
 // (cos, sin) of pos * base^(-2 i / r).  The angle is formed in double precision (positions of
 // tens of thousands would lose ~1e-3 rad in fp32), reduced to a fraction of a turn in double,
 // and only then handed to the fp32 sincospi.  log2_base = log2(base).
@@ -116,21 +163,27 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
   }
   __syncthreads();
 
-  // ---- this CTA's range of the flat tile list ----
-  long total = 0;
-  for (int b = 0; b < p.B; ++b) total += tiles_of(clamp_len(p.cache_len[b], p.Lmax));
+  // ---- this CTA's range of the flat tile list (block-wide scan over the sequences) ----
+  __shared__ long long wtot_s[THREADS / 32];
+  __shared__ int loc_b;
+  __shared__ long long loc_first;
+  int lo, hi;
+  long excl;
+  const long total = block_tile_scan(p.cache_len, p.B, p.Lmax, lo, hi, excl, wtot_s);
   const long t_begin = cta_first_tile(blockIdx.x, total, gridDim.x);
   const long t_end = cta_first_tile(blockIdx.x + 1, total, gridDim.x);
-  int b0 = 0;
-  long seq_first = 0;   // global index of the first tile of sequence b0
-  if (t_begin < t_end) {
-    while (true) {
-      const long nt = tiles_of(clamp_len(p.cache_len[b0], p.Lmax));
-      if (seq_first + nt > t_begin) break;
-      seq_first += nt;
-      ++b0;
+  {
+    // the thread whose sequences contain tile t_begin publishes that sequence and its first tile
+    long f = excl;
+    for (int b = lo; b < hi; ++b) {
+      const long nt = tiles_of(clamp_len(p.cache_len[b], p.Lmax));
+      if (t_begin >= f && t_begin < f + nt) { loc_b = b; loc_first = f; }
+      f += nt;
     }
   }
+  __syncthreads();
+  const int b0 = (t_begin < t_end) ? loc_b : 0;
+  const long seq_first = (t_begin < t_end) ? (long)loc_first : 0;   // global index of the first tile of sequence b0
 
   if (warp == CONSUMER_WARPS) {
     // ------------------------------- TMA producer -------------------------------
@@ -388,7 +441,7 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
 //   qhat_h  <- qhat_h R(L, r3), stored bf16 [B, nH, r3]
 // The core is read with 16-byte loads that are all issued before anything waits on them:
 // warp w, lane (rg = lane / 4, ch = lane % 4) owns chunk ch of the CTA's 64-byte column range
-// in the core rows q = 8 w + rg + 64 i, for AB = 16 / NQ slices a at a time (NQ = ceil(r2/64)).
+// in the core rows q = 8 w + rg + 64 i, for AB = 8 / NQ slices a at a time (NQ = ceil(r2/64)).
 // part: [splits][Mpad][r2 + r3 + t3] fp32.
 // ---------------------------------------------------------------------------------------
 constexpr int DQ_CW = 32;       // latent key coordinates per CTA
@@ -396,12 +449,12 @@ constexpr int DQ_MAX_R1 = 32;   // head ranks r1, t1 supported by the shared-mem
 constexpr int DQ_MAX_R2 = 256;
 
 template <int NQ>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH, int r1, int r2, int r3, int t3,
            const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
-           const int32_t* __restrict__ cache_len, int rope, double log2_base, int append, unsigned int* err) {
-  constexpr int AB = 16 / NQ;                       // core slices per batch
+           const int32_t* __restrict__ cache_len, int rope, const RopeFreqs freqs, int append, unsigned int* err) {
+  constexpr int AB = 8 / NQ;                        // core slices per batch (8 loads of 16 bytes in flight per thread)
   __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
   __shared__ float k_s[DQ_CW];                      // this CTA's coordinates of the new key (unrotated)
   __shared__ float2 cs_s[DQ_CW / 2];                // (cos, sin) at position L for this CTA's pairs
@@ -450,7 +503,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
   }
   for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
   if (threadIdx.x < DQ_CW / 2) {
-    cs_s[threadIdx.x] = rope ? rope_cos_sin(L, c0 / 2 + threadIdx.x, r3, log2_base) : make_float2(1.f, 0.f);
+    cs_s[threadIdx.x] = rope ? rope_cos_sin_theta(L, freqs.theta[c0 / 2 + threadIdx.x]) : make_float2(1.f, 0.f);
   }
   __syncthreads();
   if (threadIdx.x < DQ_CW / 2) {                    // new key, rotated
@@ -557,11 +610,18 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
       for (long off = (long)threadIdx.x * 128; off < span; off += (long)blockDim.x * 128)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(cbase + ((long)a * t2 + jbeg) * row_bytes + off));
   }
-  long total = 0, first = 0;
-  for (int i = 0; i < B; ++i) {
-    if (i == b) first = total;
-    total += tiles_of(clamp_len(cache_len[i], Lmax));
+  __shared__ long long wtot_s[8];
+  __shared__ long long first_s;
+  int lo, hi;
+  long excl;
+  const long total = block_tile_scan(cache_len, B, Lmax, lo, hi, excl, wtot_s);
+  if (b >= lo && b < hi) {
+    long f = excl;
+    for (int i = lo; i < b; ++i) f += tiles_of(clamp_len(cache_len[i], Lmax));
+    first_s = f;
   }
+  __syncthreads();
+  const long first = (long)first_s;
   const long nt = tiles_of(clamp_len(cache_len[b], Lmax));
   // CTAs i with [first_i, first_{i+1}) intersecting [first, first + nt)
   long i0 = first * grid_attn / total;
@@ -607,34 +667,58 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
     inv_l[h] = 1.f / Lsum;
   }
   __syncthreads();
-  for (int e4 = threadIdx.x; e4 < nH * t3 / 4; e4 += blockDim.x) {
-    const int h = (e4 * 4) / t3;
-    const float4* po = reinterpret_cast<const float4*>(part_o + (i0 + b) * 32 * t3) + e4;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k0 = 0; k0 < np; k0 += 4) {
-      float4 v[4];
-      float wg[4];
+  // merged (not yet normalised) outputs: a thread owns up to 4 float4 of the [nH][t3] block
+  // (nH * t3 / 4 <= 1024 = 4 * blockDim.x for nH <= 32, t3 <= 128); for the usual case of at most four
+  // partials all of its loads are issued before any is used
+  {
+    const int n4 = nH * t3 / 4;
+    const float4* po = reinterpret_cast<const float4*>(part_o + (i0 + b) * 32 * t3);
+    for (int k0 = 0; k0 < np || k0 == 0; k0 += 4) {
+      float4 v[4][4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        wg[u] = (k0 + u < np) ? w_s[(k0 + u) * 32 + h] : 0.f;
-        v[u] = (k0 + u < np) ? po[(long)(k0 + u) * 8 * t3] : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int e = 0; e < 4; ++e) {
+        const int e4 = threadIdx.x + e * 256;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          v[e][u] = (e4 < n4 && k0 + u < np) ? po[(long)(k0 + u) * 8 * t3 + e4] : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (wg[u] != 0.f) {     // a zero weight marks a slot whose bytes are not numbers to be used
-          acc.x += wg[u] * v[u].x; acc.y += wg[u] * v[u].y; acc.z += wg[u] * v[u].z; acc.w += wg[u] * v[u].w;
+      for (int e = 0; e < 4; ++e) {
+        const int e4 = threadIdx.x + e * 256;
+        if (e4 < n4) {
+          const int h = (e4 * 4) / t3;
+          float4 acc = k0 == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : reinterpret_cast<float4*>(o_s)[e4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float wg = (k0 + u < np) ? w_s[(k0 + u) * 32 + h] : 0.f;
+            if (wg != 0.f) {     // a zero weight marks a slot whose bytes are not numbers to be used
+              acc.x += wg * v[e][u].x; acc.y += wg * v[e][u].y; acc.z += wg * v[e][u].z; acc.w += wg * v[e][u].w;
+            }
+          }
+          reinterpret_cast<float4*>(o_s)[e4] = acc;
         }
       }
     }
-    const float il = inv_l[h];
-    reinterpret_cast<float4*>(o_s)[e4] = make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il);
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < t1 * t3; e += blockDim.x) {
-    const int a = e / t3, c = e % t3;
-    float acc = 0.f;
-    for (int h = 0; h < nH; ++h) acc = fmaf(ut1_s[h * t1 + a], o_s[h * t3 + c], acc);
-    u_s[e] = acc;
+  // u[a, c] = sum_h Ut1[h, a] o_h[c] / l_h; a thread owns column c and runs of four slices a
+  {
+    const int ngrp = blockDim.x / t3 > 0 ? blockDim.x / t3 : 1;     // thread groups over the slices
+    const int c = threadIdx.x % t3, grp = threadIdx.x / t3;
+    if (grp < ngrp) {
+      for (int a0 = grp * 4; a0 < t1; a0 += ngrp * 4) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int h = 0; h < nH; ++h) {
+          const float ov = o_s[h * t3 + c] * inv_l[h];
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (a0 + u < t1) acc[u] = fmaf(ut1_s[h * t1 + a0 + u], ov, acc[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (a0 + u < t1) u_s[(a0 + u) * t3 + c] = acc[u];
+      }
+    }
   }
   __syncthreads();
   // z[j]: lane group g = lane / nch of warp w owns output row j = jbeg + (w * rpl + g) + 8 * rpl * jj and
@@ -643,37 +727,54 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
   const int rpl = 32 / nch;                // rows per warp-wide load: 4, 2 or 2
   const int g = lane / nch, ch = lane % nch;
   const uint4* Cq = reinterpret_cast<const uint4*>(Ct);
-  constexpr int PF = 8;
-  for (int jl = warp * rpl + (g < rpl ? g : 0); jl < jn; jl += 8 * rpl) {     // uniform trip count per warp
-    const int j = jbeg + jl;
-    float acc = 0.f;
-    for (int a0 = 0; a0 < t1; a0 += PF) {
-      uint4 v[PF];
+  constexpr int PF = 8, JJ = 2;
+  // (the rows of this CTA were prefetched into L2 at the top, so every batch costs one L2 round trip;
+  // a lane group takes JJ output rows at a time, JJ * PF loads in flight)
+  for (int jl = warp * rpl + (g < rpl ? g : 0); jl < jn; jl += 8 * rpl * JJ) {     // uniform trip count per warp
+    float acc[JJ];
 #pragma unroll
-      for (int u = 0; u < PF; ++u)
-        v[u] = (g < rpl && a0 + u < t1) ? Cq[((long)(a0 + u) * t2 + j) * nch + ch] : make_uint4(0u, 0u, 0u, 0u);
+    for (int jj = 0; jj < JJ; ++jj) acc[jj] = 0.f;
+    for (int a0 = 0; a0 < t1; a0 += PF) {
+      uint4 v[JJ][PF];
+#pragma unroll
+      for (int jj = 0; jj < JJ; ++jj) {
+        const int j = jbeg + jl + jj * 8 * rpl;
+#pragma unroll
+        for (int u = 0; u < PF; ++u)
+          v[jj][u] = (g < rpl && a0 + u < t1 && jl + jj * 8 * rpl < jn) ? Cq[((long)(a0 + u) * t2 + j) * nch + ch]
+                                                                        : make_uint4(0u, 0u, 0u, 0u);
+      }
 #pragma unroll
       for (int u = 0; u < PF; ++u) {
         if (a0 + u < t1) {
           const float4 u0 = reinterpret_cast<const float4*>(u_s + (a0 + u) * t3 + ch * 8)[0];
           const float4 u1 = reinterpret_cast<const float4*>(u_s + (a0 + u) * t3 + ch * 8)[1];
-          const uint32_t wv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-          const float2 k0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[0]));
-          const float2 k1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[1]));
-          const float2 k2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[2]));
-          const float2 k3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[3]));
-          acc = fmaf(u0.x, k0.x, acc); acc = fmaf(u0.y, k0.y, acc); acc = fmaf(u0.z, k1.x, acc); acc = fmaf(u0.w, k1.y, acc);
-          acc = fmaf(u1.x, k2.x, acc); acc = fmaf(u1.y, k2.y, acc); acc = fmaf(u1.z, k3.x, acc); acc = fmaf(u1.w, k3.y, acc);
+#pragma unroll
+          for (int jj = 0; jj < JJ; ++jj) {
+            const uint32_t wv[4] = {v[jj][u].x, v[jj][u].y, v[jj][u].z, v[jj][u].w};
+            const float2 k0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[0]));
+            const float2 k1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[1]));
+            const float2 k2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[2]));
+            const float2 k3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[3]));
+            float t = acc[jj];
+            t = fmaf(u0.x, k0.x, t); t = fmaf(u0.y, k0.y, t); t = fmaf(u0.z, k1.x, t); t = fmaf(u0.w, k1.y, t);
+            t = fmaf(u1.x, k2.x, t); t = fmaf(u1.y, k2.y, t); t = fmaf(u1.z, k3.x, t); t = fmaf(u1.w, k3.y, t);
+            acc[jj] = t;
+          }
         }
       }
     }
     // sum over the nch lanes of the group (groups are aligned to multiples of nch lanes)
-    if (g >= rpl) acc = 0.f;
-    for (int off = 1; off < nch; off <<= 1) {
-      const float t = __shfl_down_sync(0xffffffffu, acc, off);
-      if (ch + off < nch) acc += t;
+#pragma unroll
+    for (int jj = 0; jj < JJ; ++jj) {
+      float t = (g >= rpl) ? 0.f : acc[jj];
+      for (int off = 1; off < nch; off <<= 1) {
+        const float o = __shfl_down_sync(0xffffffffu, t, off);
+        if (ch + off < nch) t += o;
+      }
+      const int jrow = jl + jj * 8 * rpl;
+      if (g < rpl && ch == 0 && jrow < jn) z[(long)b * t2 + jbeg + jrow] = __float2bfloat16_rn(t);
     }
-    if (g < rpl && ch == 0) z[(long)b * t2 + j] = __float2bfloat16_rn(acc);
   }
 }
 

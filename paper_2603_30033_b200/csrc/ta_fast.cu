@@ -70,7 +70,7 @@ struct PrepParams {
   int nH, r1, r2, r3, t1, t2, t3;
   int n_pos, pos0;
   float mult;
-  double log2_base;
+  dec::RopeFreqs freqs;
   int g1, g2, g3;
 };
 
@@ -99,8 +99,17 @@ __global__ void __launch_bounds__(256) k_prefill_prep(const PrepParams p) {
     const int half = p.r3 / 2;
     const long total = (long)p.n_pos * half;
     for (long i = (blk - p.g1 - p.g2) * (long)blockDim.x + threadIdx.x; i < total; i += (long)p.g3 * blockDim.x)
-      p.rope[i] = dec::rope_cos_sin(p.pos0 + (int)(i / half), (int)(i % half), p.r3, p.log2_base);
+      p.rope[i] = dec::rope_cos_sin_theta(p.pos0 + (int)(i / half), p.freqs.theta[i % half]);
   }
+}
+
+// theta_i = base^(-2 i / r3) in double precision, i < r3 / 2 (r3 <= 256 on this path)
+dec::RopeFreqs rope_freqs(const tucker_attn_desc& d) {
+  dec::RopeFreqs f;
+  const int half = d.r3 / 2;
+  for (int i = 0; i < 128; ++i)
+    f.theta[i] = (d.rope && i < half) ? pow((double)d.rope_base, -2.0 * (double)i / (double)d.r3) : 0.0;
+  return f;
 }
 
 int grid_for(long total, int block = 256) {
@@ -298,7 +307,7 @@ int fast_fwd(Problem& p) {
     pp.nH = d.n_H; pp.r1 = d.r1; pp.r2 = d.r2; pp.r3 = d.r3; pp.t1 = d.t1; pp.t2 = d.t2; pp.t3 = d.t3;
     pp.n_pos = d.N; pp.pos0 = d.pos0;
     pp.mult = tc_attn ? p.scale * LOG2E : p.scale;
-    pp.log2_base = d.rope ? log2((double)d.rope_base) : 0.0;
+    pp.freqs = rope_freqs(d);
     pp.g1 = grid_for((long)d.n_H * d.r2 * d.r3);
     pp.g2 = grid_for((long)d.n_H * d.t2 * d.t3);
     pp.g3 = d.rope ? grid_for((long)d.N * (d.r3 / 2)) : 0;
@@ -485,11 +494,11 @@ int fast_decode(Problem& p) {
   // ---- 2: finish, RoPE, append, per-head queries ----
   {
     const dim3 grid(d.B, d.r3 / dec::DQ_CW);
+    const dec::RopeFreqs freqs = rope_freqs(d);
     auto launch = [&](auto kernel) {
       kernel<<<grid, 256, 0, p.stream>>>(w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3,
                                          (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
-                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, log2((double)d.rope_base),
-                                         p.append, p.dev_err);
+                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.dev_err);
     };
     switch ((d.r2 + 63) / 64) {
       case 1: launch(dec::k_dec_qhat<1>); break;
