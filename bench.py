@@ -131,24 +131,28 @@ class Flusher:
             self.buf.fill_(1)
 
 
-def time_steps(torch, Bd, step_fn, steps, warmup, flush, barrier):
+def time_steps(torch, Bd, step_fn, steps, warmup, flush, barrier, profile=False):
     """Runs warm-up, then `steps` timed steps.  Returns (per-step ms list, per-step dominant-kernel
-    ms list, wall interval)."""
+    ms list or None, wall interval).  With profile=True two extra events are recorded around the
+    dominant kernel of every step; that pass is only used for the kernel's own duration, because
+    an event between two kernels keeps their launches from overlapping."""
     for _ in range(warmup):
         flush()
         step_fn()
     torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in kev:      # materialise the handles
-        a.record()
-        b.record()
+    if profile:
+        for a, b in kev:      # materialise the handles
+            a.record()
+            b.record()
     barrier()
     torch.cuda.synchronize()
     t0 = time.time()
     for i in range(steps):
         flush()
-        Bd.set_profile_events(*kev[i])
+        if profile:
+            Bd.set_profile_events(*kev[i])
         ev[i][0].record()
         step_fn()
         ev[i][1].record()
@@ -157,7 +161,7 @@ def time_steps(torch, Bd, step_fn, steps, warmup, flush, barrier):
     t1 = time.time()
     barrier()
     ms = [a.elapsed_time(b) for a, b in ev]
-    kms = [a.elapsed_time(b) for a, b in kev]
+    kms = [a.elapsed_time(b) for a, b in kev] if profile else None
     return ms, kms, (t0, t1)
 
 
@@ -182,8 +186,9 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
     flush = Flusher(torch, needed=in_bytes < 2 * L2_BYTES)
     if sampler:
         sampler.start()
-    ms, kms, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
+    ms, _, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
     clocks = sampler.stop(t0, t1) if sampler else None
+    _, kms, _ = time_steps(torch, Bd, step, min(steps, 10), 1, flush, barrier, profile=True)
     launches = Bd.last_launch_count()
     path = Bd.last_path()
     assert Bd.last_device_error() == 0, "device error word set during the benchmark"
@@ -250,8 +255,9 @@ def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sam
     flush = Flusher(torch, needed=by["total"] < 2 * L2_BYTES)
     if sampler:
         sampler.start()
-    ms, kms, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
+    ms, _, (t0, t1) = time_steps(torch, Bd, step, steps, warmup, flush, barrier)
     clocks = sampler.stop(t0, t1) if sampler else None
+    _, kms, _ = time_steps(torch, Bd, step, min(steps, 10), 1, flush, barrier, profile=True)
     launches, path = Bd.last_launch_count(), Bd.last_path()
     assert Bd.last_device_error() == 0, "device error word set during the benchmark"
     ms_step = sum(ms) / len(ms)

@@ -87,6 +87,7 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ uint64_t s_full[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];

@@ -68,6 +68,35 @@ bool fast_decode_supported(const tucker_attn_desc& d, int32_t Lmax);
 size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
 int fast_decode(Problem& p);
 
+// Programmatic dependent launch.  Every kernel of the tensor-core paths starts with pdl_enter():
+// it waits until the preceding kernels of the stream have completed and their writes are visible,
+// and only then lets the next kernel of the stream be scheduled.  Launched through launch_pdl, a
+// kernel's launch and block scheduling therefore overlap the tail of its predecessor, while nothing
+// (global memory, TMEM) is touched before the predecessor is done.  Without the launch attribute
+// both instructions are no-ops.
+#if defined(__CUDACC__)
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 #define TA_CUDA_TRY(expr)                          \
   do {                                             \
     cudaError_t _e = (expr);                       \

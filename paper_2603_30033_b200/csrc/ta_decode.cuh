@@ -141,6 +141,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 template <int R3, int T3>
 __global__ void __launch_bounds__(THREADS, 1)
 k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES];
   __shared__ int abort_flag;
@@ -454,6 +455,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
            const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
            const int32_t* __restrict__ cache_len, int rope, const RopeFreqs freqs, int append, unsigned int* err) {
+  pdl_enter();
   constexpr int AB = 8 / NQ;                        // core slices per batch (8 loads of 16 bytes in flight per thread)
   __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
   __shared__ float k_s[DQ_CW];                      // this CTA's coordinates of the new key (unrotated)
@@ -592,6 +594,7 @@ __global__ void __launch_bounds__(256)
 k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ cache_len,
           int B, int Lmax, int nH, int t1, int t2, int t3, int grid_attn, const bf16* __restrict__ Ct,
           const bf16* __restrict__ Ut1, bf16* __restrict__ z) {
+  pdl_enter();
   extern __shared__ __align__(16) float do_smem[];
   float* o_s = do_smem;                    // [32][t3]
   float* w_s = o_s + 32 * t3;              // [MAX_GRID][32]

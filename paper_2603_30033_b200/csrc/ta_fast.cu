@@ -90,6 +90,7 @@ __device__ __forceinline__ void head_core_part(const bf16* __restrict__ C, const
 }
 
 __global__ void __launch_bounds__(256) k_prefill_prep(const PrepParams p) {
+  pdl_enter();
   const int blk = blockIdx.x;
   if (blk < p.g1) {
     head_core_part(p.C, p.U1, p.GcatT, p.nH, p.r1, p.r2, p.r3, (long)p.r3 * p.r2, 1, p.r2, p.mult, blk, p.g1);
@@ -194,8 +195,8 @@ int launch_gemm(Problem& p, const bf16* A, long lda, int M, int K, const BOperan
     attr_set = true;
   }
   dim3 grid(Ntot / BN, (M + 127) / 128, splits);
-  umma_gemm::k_umma_gemm<<<grid, umma_gemm::THREADS, umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major), p.stream>>>(
-      tmA, tmB[0], tmB[1], tmB[2], gp);
+  (void)launch_pdl(umma_gemm::k_umma_gemm, grid, dim3(umma_gemm::THREADS),
+                   umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major), p.stream, tmA, tmB[0], tmB[1], tmB[2], gp);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
 }
@@ -265,7 +266,8 @@ int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const f
   }
   const long items = (long)ap.n_qt * d.B * ap.n_hg;
   prof_begin(p);
-  attn::k_attn_prefill<<<(unsigned)items, attn::THREADS, attn::SMEM_BYTES, p.stream>>>(tmQ, tmG, tmK, tmV, ap);
+  (void)launch_pdl(attn::k_attn_prefill, dim3((unsigned)items), dim3(attn::THREADS), attn::SMEM_BYTES, p.stream, tmQ, tmG,
+                   tmK, tmV, ap);
   prof_end(p);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
@@ -311,7 +313,7 @@ int fast_fwd(Problem& p) {
     pp.g1 = grid_for((long)d.n_H * d.r2 * d.r3);
     pp.g2 = grid_for((long)d.n_H * d.t2 * d.t3);
     pp.g3 = d.rope ? grid_for((long)d.N * (d.r3 / 2)) : 0;
-    k_prefill_prep<<<pp.g1 + pp.g2 + pp.g3, 256, 0, p.stream>>>(pp);
+    (void)launch_pdl(k_prefill_prep, dim3(pp.g1 + pp.g2 + pp.g3), dim3(256), 0, p.stream, pp);
     TA_LAUNCH_CHECK(p);
   }
 
@@ -436,7 +438,7 @@ int launch_dec_attn(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, 
     attr_set = true;
   }
   prof_begin(p);
-  dec::k_dec_attn<R3, T3><<<dp.grid, dec::THREADS, dec::SMEM_BYTES, p.stream>>>(tmK, tmV, dp);
+  (void)launch_pdl(dec::k_dec_attn<R3, T3>, dim3(dp.grid), dim3(dec::THREADS), dec::SMEM_BYTES, p.stream, tmK, tmV, dp);
   prof_end(p);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
@@ -496,9 +498,9 @@ int fast_decode(Problem& p) {
     const dim3 grid(d.B, d.r3 / dec::DQ_CW);
     const dec::RopeFreqs freqs = rope_freqs(d);
     auto launch = [&](auto kernel) {
-      kernel<<<grid, 256, 0, p.stream>>>(w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2, d.r3, d.t3,
-                                         (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
-                                         (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.dev_err);
+      (void)launch_pdl(kernel, grid, dim3(256), 0, p.stream, w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2,
+                       d.r3, d.t3, (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
+                       (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.dev_err);
     };
     switch ((d.r2 + 63) / 64) {
       case 1: launch(dec::k_dec_qhat<1>); break;
@@ -530,9 +532,9 @@ int fast_decode(Problem& p) {
                                        (int)dec::dec_out_smem(32, 32, 128)));
       out_attr_set = true;
     }
-    dec::k_dec_out<<<dim3(d.B, dec::DO_JS), 256, dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream>>>(
-        w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H, d.t1, d.t2, d.t3, dp.grid, (const bf16*)p.Ct,
-        (const bf16*)p.Ut1, w.z);
+    (void)launch_pdl(dec::k_dec_out, dim3(d.B, dec::DO_JS), dim3(256), dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream,
+                     w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H, d.t1, d.t2, d.t3, dp.grid, (const bf16*)p.Ct,
+                     (const bf16*)p.Ut1, w.z);
     TA_LAUNCH_CHECK(p);
   }
   // ---- 5: y = z Ut2^T ----
