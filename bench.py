@@ -228,15 +228,19 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
 def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=None):
     wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
     dw = [_dev(wt[k], w.dtype, torch) for k in KEYS]
+    shared = getattr(w, "shared_kv", False)
+    if shared:
+        dw[7] = dw[3]           # the same device tensor for U3 and Ut3 selects the shared projection
     L, Lmax, B = w.N, w.N + 1, w.B
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     gen = torch.Generator(device="cuda")
     gen.manual_seed(w.seed)
     Kc = torch.empty(B, Lmax, w.r[2], dtype=tdt, device="cuda")
-    Vc = torch.empty(B, Lmax, w.t[2], dtype=tdt, device="cuda")
+    Vc = Kc if shared else torch.empty(B, Lmax, w.t[2], dtype=tdt, device="cuda")
     for b in range(B):      # cache entries ~ N(0,1), drawn on the device one sequence at a time
         Kc[b] = torch.randn(Lmax, w.r[2], generator=gen, device="cuda", dtype=torch.float32).to(tdt)
-        Vc[b] = torch.randn(Lmax, w.t[2], generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+        if not shared:
+            Vc[b] = torch.randn(Lmax, w.t[2], generator=gen, device="cuda", dtype=torch.float32).to(tdt)
     x32 = torch.from_numpy(W.make_decode_x(w))
     x_host = (x32.to(tdt)).contiguous().pin_memory()
     x = x_host.cuda()
@@ -324,6 +328,8 @@ def oracle_sample(w, budget="default"):
     for b in range(nseq):
         k, v = W.decode_cache_rows(w, b, L)
         Kc[b, :L], Vc[b, :L] = W.round_to_storage(k, w.dtype), W.round_to_storage(v, w.dtype)
+    if getattr(w, "shared_kv", False):
+        Vc = Kc                 # one latent cache serves keys and values
     lens = np.full((nseq,), L, dtype=np.int32)
     by = W.decode_bytes(w, B=nseq)
 
@@ -446,7 +452,7 @@ def main():
 
     others = []
     if not args.no_others and world == 1:
-        for name in ("c2", "c3", "c4", "c5"):
+        for name in ("c2", "c3", "c4", "c5", "f1"):
             ow = W.get_workload(name)
             if ow.name == w.name:
                 continue

@@ -98,6 +98,12 @@ TA_API size_t tucker_attn_decode_workspace_bytes(const tucker_attn_desc* desc, i
  *        latent values (the KV cache of Sec. 3.1); other rows are left untouched.
  *   workspace: >= tucker_attn_fwd_workspace_bytes(desc) bytes, 256-byte aligned.
  * All steps, including the weight-only core contraction, run inside the call.
+ *
+ * Shared key / value projection (Sec. 3.1, "L^KV = X U3"): pass the SAME pointer for U3 and Ut3
+ * (then r3 == t3) with rope == 0.  The latent keys are then the latent values; they are projected
+ * once, and Kcache_out may equal Vcache_out (one cache of N r3 entries instead of 2 N r3).  With
+ * latent RoPE the cached keys are rotated and cannot double as values: Kcache_out == Vcache_out is
+ * TA_ERR_INVALID_ARG unless U3 == Ut3, r3 == t3 and rope == 0.
  */
 TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
                     const void* C, const void* U1, const void* U2, const void* U3,
@@ -116,6 +122,10 @@ TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
  *             (the caller increments its lengths); 0: the caches are not modified
  *   y         [B, d_model]                     out
  *   desc->N, desc->pos0, desc->causal are ignored.
+ *
+ * Shared latent cache (Sec. 3.1): Kcache == Vcache is accepted when U3 == Ut3 (same pointer),
+ * r3 == t3 and rope == 0; the step then reads every cached row once (half the bytes) and appends
+ * one row.  Any other call with Kcache == Vcache is TA_ERR_INVALID_ARG.
  */
 TA_API int tucker_attn_decode(const tucker_attn_desc* desc, const void* x,
                        const void* C, const void* U1, const void* U2, const void* U3,

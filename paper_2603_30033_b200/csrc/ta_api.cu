@@ -48,6 +48,13 @@ static bool use_fast_decode(const tucker_attn_desc& d, int32_t Lmax) {
   return d.dtype == TA_DTYPE_BF16 && !(d.flags & TA_FLAG_FORCE_GENERIC) && fast_decode_supported(d, Lmax);
 }
 
+// Shared key / value projection (Sec. 3.1, L^KV = X U3): the caller passes the SAME factor for U3 and Ut3.
+// Without RoPE the latent keys are then the latent values, so one projection and one cache serve both.
+// (With latent RoPE the cached keys are rotated and cannot double as values.)
+static bool shared_kv_weights(const tucker_attn_desc& d, const void* U3, const void* Ut3) {
+  return U3 == Ut3 && d.r3 == d.t3 && !d.rope;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace ta
@@ -74,6 +81,7 @@ int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X, const void* C, 
   if (!X || !C || !U1 || !U2 || !U3 || !Ct || !Ut1 || !Ut2 || !Ut3 || !Y || !workspace) return TA_ERR_INVALID_ARG;
   if ((Kcache_out == nullptr) != (Vcache_out == nullptr)) return TA_ERR_INVALID_ARG;
   if (Kcache_out && Lmax < desc->N) return TA_ERR_INVALID_ARG;
+  if (Kcache_out && Kcache_out == Vcache_out && !shared_kv_weights(*desc, U3, Ut3)) return TA_ERR_INVALID_ARG;
   const void* ptrs[] = {X, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, Y};
   for (const void* q : ptrs)
     if (!aligned16(q)) return TA_ERR_INVALID_ARG;
@@ -89,6 +97,7 @@ int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X, const void* C, 
   p.X = X; p.C = C; p.U1 = U1; p.U2 = U2; p.U3 = U3; p.Ct = Ct; p.Ut1 = Ut1; p.Ut2 = Ut2; p.Ut3 = Ut3;
   p.Y = Y; p.Kc = Kcache_out; p.Vc = Vcache_out; p.Lmax = Lmax;
   p.cache_len = nullptr; p.append = 0;
+  p.shared_kv = (shared_kv_weights(*desc, U3, Ut3) && Kcache_out == Vcache_out) ? 1 : 0;
   p.ws = static_cast<char*>(workspace); p.ws_bytes = workspace_bytes;
   p.stream = static_cast<cudaStream_t>(cuda_stream);
   p.dev_err = device_error_ptr();
@@ -108,6 +117,7 @@ int tucker_attn_decode(const tucker_attn_desc* desc, const void* x, const void* 
   if (!desc_ok(desc, true)) return TA_ERR_INVALID_ARG;
   if (!x || !C || !U1 || !U2 || !U3 || !Ct || !Ut1 || !Ut2 || !Ut3 || !y || !workspace) return TA_ERR_INVALID_ARG;
   if (!Kcache || !Vcache || !cache_len || Lmax <= 0) return TA_ERR_INVALID_ARG;
+  if (Kcache == Vcache && !shared_kv_weights(*desc, U3, Ut3)) return TA_ERR_INVALID_ARG;
   const void* ptrs[] = {x, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, y, Kcache, Vcache};
   for (const void* q : ptrs)
     if (!aligned16(q)) return TA_ERR_INVALID_ARG;
@@ -122,6 +132,7 @@ int tucker_attn_decode(const tucker_attn_desc* desc, const void* x, const void* 
   p.X = x; p.C = C; p.U1 = U1; p.U2 = U2; p.U3 = U3; p.Ct = Ct; p.Ut1 = Ut1; p.Ut2 = Ut2; p.Ut3 = Ut3;
   p.Y = y; p.Kc = Kcache; p.Vc = Vcache; p.Lmax = Lmax;
   p.cache_len = cache_len; p.append = append ? 1 : 0;
+  p.shared_kv = (Kcache == Vcache) ? 1 : 0;
   p.ws = static_cast<char*>(workspace); p.ws_bytes = workspace_bytes;
   p.stream = static_cast<cudaStream_t>(cuda_stream);
   p.dev_err = device_error_ptr();

@@ -23,6 +23,7 @@ struct Problem {
   int32_t Lmax;
   const int32_t* cache_len; // decode only (device)
   int32_t append;           // decode only
+  int shared_kv;            // one latent cache / one projection serves keys and values (U3 == Ut3, no RoPE)
   char* ws;                 // workspace base (256-byte aligned)
   size_t ws_bytes;
   cudaStream_t stream;

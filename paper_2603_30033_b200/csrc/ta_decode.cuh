@@ -36,6 +36,7 @@ constexpr int MAX_GRID = 160;           // partial weights table in the merge ke
 
 struct Params {
   int B, nH, Lmax, grid;
+  int shared_kv;       // 1: the value cache IS the key cache (one latent cache L^KV, Sec. 3.1): each tile is loaded once
   const int32_t* cache_len;
   const bf16* qhat;    // [B, nH, R3] rotated, scaled by softmax scale * log2 e
   const bf16* knew;    // [B, R3] rotated new key
@@ -204,12 +205,13 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
         if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&full_bar[s], (uint32_t)((KSUB + VSUB) * SUB_BYTES));
+        mbar_expect_tx(&full_bar[s], (uint32_t)((KSUB + (p.shared_kv ? 0 : VSUB)) * SUB_BYTES));
         uint8_t* kt = tiles + (size_t)s * STAGE_BYTES;
         uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
         const int row = (int)(t - first) * TK;
         for (int kk = 0; kk < KSUB; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, b);
-        for (int kk = 0; kk < VSUB; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, b);
+        if (!p.shared_kv)
+          for (int kk = 0; kk < VSUB; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, b);
       }
     }
   } else if (t_begin < t_end) {
@@ -253,7 +255,7 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         uint8_t* kt = tiles + (size_t)s * STAGE_BYTES;
-        uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
+        uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;   // shared latent cache: the K tile is the V tile
         const int k0 = (int)(t - first) * TK;
         const bool last_tile = (k0 + TK > L);        // contains the new token (index L) and possibly invalid rows
         if (last_tile) {
@@ -454,7 +456,8 @@ __global__ void __launch_bounds__(256, 2)
 k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH, int r1, int r2, int r3, int t3,
            const bf16* __restrict__ C, const bf16* __restrict__ U1, float mult, bf16* __restrict__ qhat,
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
-           const int32_t* __restrict__ cache_len, int rope, const RopeFreqs freqs, int append, unsigned int* err) {
+           const int32_t* __restrict__ cache_len, int rope, const RopeFreqs freqs, int append, int shared_kv,
+           unsigned int* err) {
   pdl_enter();
   constexpr int AB = 8 / NQ;                        // core slices per batch (8 loads of 16 bytes in flight per thread)
   __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
@@ -501,7 +504,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + r2 + r3 + c];
     const bf16 vv = __float2bfloat16_rn(acc);
     vnew[(long)b * t3 + c] = vv;
-    if (append) Vc[((long)b * Lmax + L) * t3 + c] = vv;
+    if (append && !shared_kv) Vc[((long)b * Lmax + L) * t3 + c] = vv;   // shared cache: the key row written below is the value row
   }
   for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
   if (threadIdx.x < DQ_CW / 2) {

@@ -326,7 +326,9 @@ int fast_fwd(Problem& p) {
     const int kmode = d.rope ? umma_gemm::EP_BF16_ROPE : umma_gemm::EP_BF16;
     const int bn = common_bn(d.r2, d.r3, d.t3);
     if (!bn) return TA_ERR_UNSUPPORTED_SHAPE;
-    gp.nseg = 3;
+    // shared key / value projection: K is V, two segments instead of three
+    const int nseg = p.shared_kv ? 2 : 3;
+    gp.nseg = nseg;
     gp.seg[0] = seg(0, d.r2, umma_gemm::EP_BF16, w.Qt, d.r2);
     gp.seg[1] = seg(d.r2, d.r3, kmode, w.K, d.r3);
     gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_BF16, w.V, d.t3);
@@ -336,8 +338,10 @@ int fast_fwd(Problem& p) {
       gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
     }
     const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
-    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, T, d.d_model, bops, 3, d.r2 + d.r3 + d.t3, bn, gp))) return rc;
+    const int ntot = d.r2 + d.r3 + (p.shared_kv ? 0 : d.t3);
+    if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, T, d.d_model, bops, 3, ntot, bn, gp))) return rc;
   }
+  const bf16* Vlat = p.shared_kv ? w.K : w.V;   // latent values
   const bool fuse_q = tc_attn && attention_fuses_qhat(d);
   // ---- per-head queries with latent RoPE (only when the attention kernel does not form them) ----
   if (!fuse_q) {
@@ -350,9 +354,9 @@ int fast_fwd(Problem& p) {
   }
   // ---- attention ----
   if (tc_attn) {
-    if ((rc = umma_attention(p, fuse_q, fuse_q ? w.Qt : w.Qhat, w.GcatT, w.rope, w.K, w.V, w.O))) return rc;
+    if ((rc = umma_attention(p, fuse_q, fuse_q ? w.Qt : w.Qhat, w.GcatT, w.rope, w.K, Vlat, w.O))) return rc;
   } else {
-    if ((rc = simt_attention_bf16(p, w.Qhat, w.K, w.V, w.O))) return rc;
+    if ((rc = simt_attention_bf16(p, w.Qhat, w.K, Vlat, w.O))) return rc;
   }
   // ---- output side ----
   {
@@ -500,7 +504,7 @@ int fast_decode(Problem& p) {
     auto launch = [&](auto kernel) {
       (void)launch_pdl(kernel, grid, dim3(256), 0, p.stream, w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2,
                        d.r3, d.t3, (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
-                       (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.dev_err);
+                       (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.shared_kv, p.dev_err);
     };
     switch ((d.r2 + 63) / 64) {
       case 1: launch(dec::k_dec_qhat<1>); break;
@@ -517,6 +521,7 @@ int fast_decode(Problem& p) {
     if (!tmap_3d(&tmV, p.Vc, d.t3, p.Lmax, d.B, d.t3, (uint64_t)p.Lmax * d.t3, 64, 128)) return TA_ERR_CUDA;
     dec::Params dp;
     dp.B = d.B; dp.nH = d.n_H; dp.Lmax = p.Lmax; dp.grid = decode_grid();
+    dp.shared_kv = p.shared_kv;
     dp.cache_len = p.cache_len; dp.qhat = w.qhat; dp.knew = w.knew; dp.vnew = w.vnew;
     dp.part_o = w.part_o; dp.part_ml = w.part_ml; dp.err = p.dev_err;
     if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);

@@ -43,6 +43,7 @@ class Workload:
     rope_base: float
     dtype: str                # "fp32" | "bf16"  (storage type; accumulation is fp32 on the GPU)
     seed: int
+    shared_kv: bool = False   # one latent cache serves keys and values (Ut3 := U3; needs rope == False)
 
     def asdict(self):
         return asdict(self)
@@ -60,6 +61,9 @@ WORKLOADS = {
                  True, True, 500000.0, "bf16", 1003),
         Workload("c5_decode", "decode", 64, 32768, 4096, 32, (8, 128, 128), (8, 128, 128),
                  True, True, 500000.0, "bf16", 1004),
+        # the decode shape with the paper's shared key / value down-projection (one latent cache, no RoPE)
+        Workload("f1_decode_shared_kv", "decode", 64, 32768, 4096, 32, (8, 128, 128), (8, 128, 128),
+                 True, False, 500000.0, "bf16", 1005, True),
     ]
 }
 
@@ -107,7 +111,7 @@ def make_weights(w: Workload, core_std: float | None = None, core_gain: float = 
     d, nH, s = w.d_model, w.n_H, w.seed
     std_c = core_std if core_std is not None else (r2 * r3) ** -0.25
     std_ct = core_std if core_std is not None else (t2 * t3) ** -0.25
-    return {
+    wts = {
         "U1": orthonormal_factor(_rng(s, 1), nH, r1),
         "U2": orthonormal_factor(_rng(s, 2), d, r2),
         "U3": orthonormal_factor(_rng(s, 3), d, r3),
@@ -117,6 +121,9 @@ def make_weights(w: Workload, core_std: float | None = None, core_gain: float = 
         "Ut3": orthonormal_factor(_rng(s, 7), d, t3),
         "Ct": _rng(s, 8).standard_normal((t1, t2, t3)) * std_ct,
     }
+    if getattr(w, "shared_kv", False):
+        wts["Ut3"] = wts["U3"]          # shared key / value down-projection
+    return wts
 
 
 def make_X(w: Workload, B: int | None = None, N: int | None = None) -> np.ndarray:
@@ -213,11 +220,12 @@ def decode_bytes(w: Workload, B: int | None = None, L: int | None = None) -> dic
     t1, t2, t3 = w.t
     d, nH = w.d_model, w.n_H
     e = 2 if w.dtype == "bf16" else 4
+    shared = getattr(w, "shared_kv", False)
     by = {
-        "cache": B * L * (r3 + t3) * e,
-        "weights": (r1 * r2 * r3 + t1 * t2 * t3 + nH * (r1 + t1) + d * (r2 + r3 + t2 + t3)) * e,
+        "cache": B * L * (r3 if shared else r3 + t3) * e,
+        "weights": (r1 * r2 * r3 + t1 * t2 * t3 + nH * (r1 + t1) + d * (r2 + r3 + t2 + (0 if shared else t3))) * e,
         "xy": 2 * B * d * e,
-        "append": B * (r3 + t3) * e,
+        "append": B * (r3 if shared else r3 + t3) * e,
     }
     by["total"] = sum(by.values())
     return by

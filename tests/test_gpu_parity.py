@@ -261,6 +261,80 @@ def test_decode_tensor_core_path(case, append):
         assert np.array_equal(Kh[b], Kc[b].astype(np.float32)) and np.array_equal(Vh[b], Vc[b].astype(np.float32))
 
 
+# --------------------------------------------------------------------------------------
+# shared key / value projection and cache (Sec. 3.1: K, V replaced by L^KV = X U3), no RoPE
+# --------------------------------------------------------------------------------------
+
+def _shared_weights(w):
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    wt["Ut3"] = wt["U3"]
+    return wt
+
+
+@pytest.mark.parametrize("dtype,shape,path", [
+    ("bf16", dict(d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128)), 2),
+    ("bf16", dict(d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 64)), 2),
+    ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
+])
+def test_decode_shared_latent_cache(dtype, shape, path):
+    import torch
+    w = H.custom_workload(kind="decode", dtype=dtype, rope=False, seed=61, **shape)
+    wt = _shared_weights(w)
+    lens = [0, 1, 127, 128, 300, 650]
+    Lmax = 700
+    x, Kc, _, cache_len = W.make_decode_state(w, B=len(lens), L=max(lens), Lmax=Lmax, cache_len=lens)
+    x, Kc = (W.round_to_storage(a, dtype) for a in (x, Kc))
+    ref, ref_k, ref_v = O.tucker_attn_decode(x, *[wt[k] for k in H.WEIGHT_KEYS], Kc, Kc, cache_len, rope=False)
+    np.testing.assert_allclose(ref_k, ref_v)            # one row serves as key and value
+    dw = H.weights_to_device(wt, dtype)
+    dw[7] = dw[3]                                        # the same device tensor for U3 and Ut3
+    Kd = H.to_device(Kc, dtype)
+    y = Bd.tucker_attn_decode(H.to_device(x, dtype), *dw, Kd, Kd, torch.from_numpy(cache_len).cuda(), n_H=w.n_H,
+                              rope=False, append=True)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == path
+    check(y.float().cpu().numpy().astype(np.float64), ref, dtype, f"shared decode {shape}", scaled=True)
+    Kh = Kd.float().cpu().numpy()
+    tol = 1e-5 if dtype == "fp32" else 3e-2
+    for b, L in enumerate(lens):
+        assert np.abs(Kh[b, L] - ref_k[b]).max() < tol
+        assert np.array_equal(Kh[b, :L], Kc[b, :L].astype(np.float32))
+
+
+def test_prefill_shared_projection_and_cache():
+    import torch
+    w = H.custom_workload(dtype="bf16", B=2, N=200, d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128), causal=True,
+                          rope=False, seed=63)
+    wt = _shared_weights(w)
+    X = W.round_to_storage(W.make_X(w), w.dtype)
+    ref, parts = O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=True, rope=False, return_parts=True)
+    dw = H.weights_to_device(wt, w.dtype)
+    dw[7] = dw[3]
+    cache = torch.full((2, 210, 128), 7.0, device="cuda", dtype=torch.bfloat16)
+    Y = Bd.tucker_attn_fwd(H.to_device(X, w.dtype), *dw, n_H=w.n_H, causal=True, rope=False, Kcache=cache, Vcache=cache)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == 2
+    check(Y.float().cpu().numpy().astype(np.float64), ref, "bf16", "shared prefill", scaled=True)
+    for b in range(2):
+        assert np.abs(cache[b, :200].float().cpu().numpy() - parts[b]["K"]).max() < 3e-2
+    assert (cache[:, 200:] == 7.0).all()
+
+
+def test_aliased_caches_need_shared_weights_and_no_rope():
+    import torch
+    w = H.custom_workload(kind="decode", dtype="bf16", d_model=256, n_H=8, r=(4, 64, 64), t=(4, 64, 64), rope=True, seed=65)
+    wt = _shared_weights(w)
+    dw = H.weights_to_device(wt, "bf16")
+    dw[7] = dw[3]
+    Kd = torch.zeros(2, 16, 64, device="cuda", dtype=torch.bfloat16)
+    x = torch.zeros(2, 256, device="cuda", dtype=torch.bfloat16)
+    ld = torch.zeros(2, dtype=torch.int32, device="cuda")
+    with pytest.raises(Bd.TuckerAttnError) as e:      # latent RoPE: rotated keys cannot double as values
+        Bd.tucker_attn_decode(x, *dw, Kd, Kd, ld, n_H=8, rope=True)
+    assert e.value.status == -1
+    dw2 = H.weights_to_device(wt, "bf16")             # distinct U3 / Ut3 tensors: not a shared projection
+    with pytest.raises(Bd.TuckerAttnError):
+        Bd.tucker_attn_decode(x, *dw2, Kd, Kd, ld, n_H=8, rope=False)
+
+
 def test_decode_garbage_beyond_cache_len_is_ignored():
     # slots at and after cache_len hold NaN / Inf bit patterns: they must not leak into the result
     import torch
