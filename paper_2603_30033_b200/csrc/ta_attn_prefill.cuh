@@ -10,7 +10,8 @@
 //   main loop  both heads use the same latent K / V tiles, so every tile is loaded once and
 //              serves two score tiles; the two softmax warpgroups ping-pong so that the tensor
 //              core works on one head while the other head's scores are being exponentiated
-//   epilogue   O_i / l written as bf16
+//   epilogue   O_i / l as bf16 into the head's idle Qhat tile, then out by a TMA tensor store that
+//              completes in the background while the warpgroup starts on the next head pair
 // In the unfused mode (query rank r2 > 128: the Qt tile would not fit) Qhat is read from
 // global memory instead and a CTA handles a single head pair.
 //
@@ -54,7 +55,7 @@ struct Params {
   int n_hg;          // head-pair groups = ceil(n_hp / hp_per_item)
   int fused;         // 1: tmQ is the map of Qt [B, N, r2] and Qhat is formed in the prologue
   const float2* rope;   // [N][r3/2] (cos, sin) for rows of this call, or nullptr (fused mode only)
-  bf16* O;           // [B, N, nH, t3]
+  bf16* O;           // [B, N, nH, t3] (written through the tensor map tmO)
   unsigned int* err;
 };
 
@@ -86,11 +87,13 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint
 
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
-               const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
+               const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const __grid_constant__ CUtensorMap tmO, const Params p) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ uint64_t s_full[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];
+  __shared__ uint64_t o_staged[2], stage_free[2];   // output rows are in shared memory / the output store has read them
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -128,6 +131,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       mbar_init(&o_full[i], 1);
       mbar_init(&qh_done[i], 1);
       mbar_init(&qh_ready[i], 4);   // one arrival per softmax warp
+      mbar_init(&o_staged[i], 4);
+      mbar_init(&stage_free[i], 1);
     }
     fence_barrier_init();
   }
@@ -281,6 +286,16 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const int g = hp - hp_begin;
       const int h0 = hp * 2;
       if (i == 1 && (h0 + 1) >= p.nH) break;   // odd head count: the last pair has one head
+      if (g > 0) {
+        // the previous pair's output store must have finished reading this head's Qhat tile
+        if (q == 0 && lane == 0) {
+          tma_store_wait_read();
+          mbar_arrive(&stage_free[i]);
+        }
+        ok = mbar_wait(&stage_free[i], (uint32_t)((g - 1) & 1), ab);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
       if (p.fused) {
         // ---- prologue: Qhat row from TMEM, latent RoPE, bf16, swizzled K-major store ----
         ok = mbar_wait(&qh_done[i], (uint32_t)(g & 1), ab);
@@ -406,26 +421,37 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      // ---- epilogue: normalised row -> this head's Qhat tile (free now: every MMA of the pair is
+      // complete) in the 128-byte-swizzled layout, then one TMA store per 64-column block; rows
+      // beyond N and columns beyond t3 are clipped by the tensor map ----
       const float inv = 1.f / l;
-      bf16* dst = p.O + (((long)b * p.N + row) * p.nH + (h0 + i)) * p.t3;
       for (int ch = 0; ch < p.t3 / 32; ++ch) {
         uint32_t o[32];
         tmem_ld32(tm_o[i] + lane_addr + ch * 32, o);
         tmem_ld_wait();
-        if (row < p.N) {
-          uint4* d4 = reinterpret_cast<uint4*>(dst + ch * 32);
+        uint8_t* dst = q_tile[i] + (ch >> 1) * SUB_BYTES + rloc * 128;
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint32_t w[4];
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-              w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
-            d4[v] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
+          for (int e = 0; e < 4; ++e)
+            w[e] = pack_bf16(__uint_as_float(o[8 * v + 2 * e]) * inv, __uint_as_float(o[8 * v + 2 * e + 1]) * inv);
+          const int chunk = (ch & 1) * 4 + v;
+          *reinterpret_cast<uint4*>(dst + ((chunk ^ (rloc & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_staged[i]);
+      if (q == 0 && lane == 0) {
+        if (mbar_wait(&o_staged[i], (uint32_t)(g & 1), ab)) {      // all four warps' rows are in shared memory
+          for (int kk = 0; kk < vsub; ++kk) tma_store_4d(&tmO, q_tile[i] + kk * SUB_BYTES, kk * 64, h0 + i, q0, b);
+          tma_store_commit();
         }
       }
       tc_fence_before();   // the next head pair's MMAs overwrite S_i / O_i after these reads
     }
+    if (q == 0 && lane == 0) tma_store_wait_all();   // the stores read shared memory: finish before the CTA may exit
   }
   tc_fence_before();
   __syncthreads();

@@ -36,13 +36,13 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 tensor of up to 3 dims; dims[0] is innermost (contiguous); strides in elements for dims 1..rank-1.
+// bf16 tensor of up to 4 dims; dims[0] is innermost (contiguous); strides in elements for dims 1..rank-1.
 bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_elems,
                const uint32_t* box, CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
-  cuuint64_t gdim[3], gstr[2];
-  cuuint32_t bx[3], es[3];
+  cuuint64_t gdim[4], gstr[3];
+  cuuint32_t bx[4], es[4];
   for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
   for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_elems[i] * 2;
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
@@ -238,7 +238,14 @@ int head_pairs_per_item(const tucker_attn_desc& d, int n_qt, int n_hp) {
 int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const float2* rope, const bf16* K,
                    const bf16* V, bf16* O) {
   const tucker_attn_desc& d = p.d;
-  CUtensorMap tmQ, tmG, tmK, tmV;
+  CUtensorMap tmQ, tmG, tmK, tmV, tmO;
+  {
+    // O [B, N, nH, t3] as a 4-D tensor (t3, head, row, sequence); one store box = 64 columns x 128 rows of one head
+    const uint64_t dims[4] = {(uint64_t)d.t3, (uint64_t)d.n_H, (uint64_t)d.N, (uint64_t)d.B};
+    const uint64_t str[3] = {(uint64_t)d.t3, (uint64_t)d.n_H * d.t3, (uint64_t)d.N * d.n_H * d.t3};
+    const uint32_t box[4] = {64, 1, 128, 1};
+    if (!make_tmap(&tmO, O, 4, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return TA_ERR_CUDA;
+  }
   if (fused) {
     if (!tmap_3d(&tmQ, Q, d.r2, d.N, d.B, d.r2, (uint64_t)d.N * d.r2, 64, 128)) return TA_ERR_CUDA;
     if (!tmap_2d(&tmG, G, (uint64_t)d.r2, (uint64_t)d.n_H * d.r3, (uint64_t)d.r2, 64, (uint32_t)d.r3)) return TA_ERR_CUDA;
@@ -267,7 +274,7 @@ int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const f
   const long items = (long)ap.n_qt * d.B * ap.n_hg;
   prof_begin(p);
   (void)launch_pdl(attn::k_attn_prefill, dim3((unsigned)items), dim3(attn::THREADS), attn::SMEM_BYTES, p.stream, tmQ, tmG,
-                   tmK, tmV, ap);
+                   tmK, tmV, tmO, ap);
   prof_end(p);
   TA_LAUNCH_CHECK(p);
   return TA_OK;
