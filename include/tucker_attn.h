@@ -80,7 +80,11 @@ typedef struct {
 } tucker_attn_desc;
 
 enum {
-  TA_FLAG_FORCE_GENERIC = 1   /* run the shape-generic FMA kernels even where a tensor-core path exists */
+  TA_FLAG_FORCE_GENERIC = 1,          /* run the shape-generic FMA kernels even where a tensor-core path exists */
+  /* Alternative routes through the bf16 tensor-core prefill path; same results within rounding, kept so that
+   * the routes can be checked against each other: */
+  TA_FLAG_FMA_ATTENTION = 0x200,      /* tensor-core GEMMs, but the attention itself on the FMA kernel */
+  TA_FLAG_SEPARATE_QUERIES = 0x400    /* per-head queries from a separate GEMM instead of the attention prologue */
 };
 
 /* Bytes of scratch the corresponding call needs for this descriptor (0 on invalid descriptor). */

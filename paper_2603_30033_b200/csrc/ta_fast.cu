@@ -123,7 +123,7 @@ bool umma_attention_ok(const tucker_attn_desc& d) { return d.r3 <= 128 && d.t3 <
 // The per-head queries are formed inside the attention kernel when the Qt tile fits next to the
 // other tiles in shared memory.
 bool attention_fuses_qhat(const tucker_attn_desc& d) {
-  return umma_attention_ok(d) && d.r2 <= 128 && !(d.flags & (0x200 | 0x400));   // 0x200: FMA attention, 0x400: unfused (bring-up switches)
+  return umma_attention_ok(d) && d.r2 <= 128 && !(d.flags & (TA_FLAG_FMA_ATTENTION | TA_FLAG_SEPARATE_QUERIES));
 }
 
 // ---- workspace ----------------------------------------------------------------------------
@@ -306,7 +306,7 @@ int fast_fwd(Problem& p) {
   carve_fast(d, p.ws, &w);
   const int T = d.B * d.N;
   const float LOG2E = 1.4426950408889634f;
-  const bool tc_attn = umma_attention_ok(d) && !(d.flags & 0x200);   // 0x200: bring-up switch, FMA attention
+  const bool tc_attn = umma_attention_ok(d) && !(d.flags & TA_FLAG_FMA_ATTENTION);
 
   // ---- weight preparation: head-mode core contractions and the RoPE table, one launch ----
   {
