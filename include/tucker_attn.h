@@ -84,7 +84,8 @@ enum {
   /* Alternative routes through the bf16 tensor-core prefill path; same results within rounding, kept so that
    * the routes can be checked against each other: */
   TA_FLAG_FMA_ATTENTION = 0x200,      /* tensor-core GEMMs, but the attention itself on the FMA kernel */
-  TA_FLAG_SEPARATE_QUERIES = 0x400    /* per-head queries from a separate GEMM instead of the attention prologue */
+  TA_FLAG_SEPARATE_QUERIES = 0x400,   /* per-head queries from a separate GEMM instead of the attention prologue */
+  TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x800 /* Z and Y from two GEMM launches instead of the fused output kernel */
 };
 
 /* Bytes of scratch the corresponding call needs for this descriptor (0 on invalid descriptor). */

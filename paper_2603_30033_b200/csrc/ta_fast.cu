@@ -12,6 +12,7 @@
 #include "ta_umma_gemm.cuh"
 #include "ta_attn_prefill.cuh"
 #include "ta_decode.cuh"
+#include "ta_zy_fused.cuh"
 
 #include <math.h>
 
@@ -366,23 +367,44 @@ int fast_fwd(Problem& p) {
     if ((rc = simt_attention_bf16(p, w.Qhat, w.K, Vlat, w.O))) return rc;
   }
   // ---- output side ----
-  {
-    umma_gemm::Params gp = {};
-    gp.n_pos = d.N;
-    gp.nseg = 1;
-    gp.seg[0] = seg(0, d.t2, umma_gemm::EP_BF16, w.Z, d.t2);
-    const BOperand bop = {w.GtP, (long)d.n_H * d.t3, d.t2};
-    if ((rc = launch_gemm(p, w.O, (long)d.n_H * d.t3, T, d.n_H * d.t3, &bop, 1, d.t2, pick_bn(d.t2), gp))) return rc;
-  }
-  {
-    umma_gemm::Params gp = {};
-    gp.n_pos = d.N;
-    gp.nseg = 1;
-    gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
-    const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
-    // short K (t2) and a wide N: 256-wide tiles halve the number of CTAs and of A-tile reads
-    const int bn = (d.d_model % 256 == 0) ? 256 : pick_bn(d.d_model);
-    if ((rc = launch_gemm(p, w.Z, d.t2, T, d.t2, &bop, 1, d.d_model, bn, gp))) return rc;
+  if (d.t2 <= 128 && d.d_model % zy::BN2 == 0 && !(d.flags & TA_FLAG_SEPARATE_OUTPUT_GEMMS)) {
+    // one kernel: Z = O Gt^T stays on chip and feeds Y = Z Ut2^T
+    const int K1 = d.n_H * d.t3;
+    CUtensorMap tmO, tmG, tmU;
+    if (!tmap_2d(&tmO, w.O, (uint64_t)K1, (uint64_t)T, (uint64_t)K1, 64, 128)) return TA_ERR_CUDA;
+    if (!tmap_2d(&tmG, w.GtP, (uint64_t)K1, (uint64_t)d.t2, (uint64_t)K1, 64, (uint32_t)d.t2)) return TA_ERR_CUDA;
+    if (!tmap_2d(&tmU, p.Ut2, (uint64_t)d.t2, (uint64_t)d.d_model, (uint64_t)d.t2, 64, 128)) return TA_ERR_CUDA;
+    zy::Params zp;
+    zp.M = T; zp.K1 = K1; zp.t2 = d.t2; zp.d = d.d_model; zp.stages = zy::MAX_STAGES;
+    zp.Y = (bf16*)p.Y; zp.err = p.dev_err;
+    static bool attr_set = false;
+    if (!attr_set) {
+      TA_CUDA_TRY(cudaFuncSetAttribute(zy::k_zy_fused, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)zy::smem_bytes(zy::MAX_STAGES)));
+      attr_set = true;
+    }
+    (void)launch_pdl(zy::k_zy_fused, dim3((T + 127) / 128), dim3(zy::THREADS), zy::smem_bytes(zp.stages), p.stream, tmO, tmG,
+                     tmU, zp);
+    TA_LAUNCH_CHECK(p);
+  } else {
+    {
+      umma_gemm::Params gp = {};
+      gp.n_pos = d.N;
+      gp.nseg = 1;
+      gp.seg[0] = seg(0, d.t2, umma_gemm::EP_BF16, w.Z, d.t2);
+      const BOperand bop = {w.GtP, (long)d.n_H * d.t3, d.t2};
+      if ((rc = launch_gemm(p, w.O, (long)d.n_H * d.t3, T, d.n_H * d.t3, &bop, 1, d.t2, pick_bn(d.t2), gp))) return rc;
+    }
+    {
+      umma_gemm::Params gp = {};
+      gp.n_pos = d.N;
+      gp.nseg = 1;
+      gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
+      const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
+      // short K (t2) and a wide N: 256-wide tiles halve the number of CTAs and of A-tile reads
+      const int bn = (d.d_model % 256 == 0) ? 256 : pick_bn(d.d_model);
+      if ((rc = launch_gemm(p, w.Z, d.t2, T, d.t2, &bop, 1, d.d_model, bn, gp))) return rc;
+    }
   }
   return TA_OK;
 }

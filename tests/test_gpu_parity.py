@@ -122,7 +122,7 @@ def test_fused_and_unfused_query_paths_agree():
                           rope=True, rope_base=500000.0, seed=91)
     X, wt = H.host_inputs(w)
     ref = oracle_fwd(X, wt, w, pos0=1000)
-    for flags in (0, Bd.TA_FLAG_SEPARATE_QUERIES, Bd.TA_FLAG_FMA_ATTENTION):
+    for flags in (0, Bd.TA_FLAG_SEPARATE_QUERIES, Bd.TA_FLAG_FMA_ATTENTION, Bd.TA_FLAG_SEPARATE_OUTPUT_GEMMS):
         got = gpu_fwd(X, wt, w, flags=flags, pos0=1000)
         assert Bd.last_path() == 2
         check(got, ref, "bf16", f"flags={flags}", scaled=True)
