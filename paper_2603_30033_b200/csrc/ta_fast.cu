@@ -75,14 +75,20 @@ struct PrepParams {
   int g1, g2, g3;
 };
 
+// out[h*sh + b*sb + c*sc] = bf16(mult * sum_a U1[h,a] C[a,b,c]).  The flat loop index walks the OUTPUT in
+// memory order (the index with unit stride innermost), so the stores are coalesced; the reads of the
+// small core tensor are strided instead and served by the caches.
 __device__ __forceinline__ void head_core_part(const bf16* __restrict__ C, const bf16* __restrict__ U1,
                                                bf16* __restrict__ out, int nH, int r1, int rb, int rc, long sh, long sb,
                                                long sc, float mult, int block, int nblocks) {
   const long total = (long)nH * rb * rc;
+  const bool b_inner = (sb == 1);         // which of b / c is contiguous in the output
+  const int n_in = b_inner ? rb : rc, n_out = b_inner ? rc : rb;
   for (long i = block * (long)blockDim.x + threadIdx.x; i < total; i += (long)nblocks * blockDim.x) {
-    const int c = (int)(i % rc);
-    const int b = (int)((i / rc) % rb);
-    const int h = (int)(i / ((long)rc * rb));
+    const int x_in = (int)(i % n_in);
+    const int x_out = (int)((i / n_in) % n_out);
+    const int h = (int)(i / ((long)n_in * n_out));
+    const int b = b_inner ? x_in : x_out, c = b_inner ? x_out : x_in;
     float acc = 0.f;
     for (int a = 0; a < r1; ++a)
       acc = fmaf(__bfloat162float(U1[(long)h * r1 + a]), __bfloat162float(C[((long)a * rb + b) * rc + c]), acc);
