@@ -1,6 +1,7 @@
 // C[M, N] = A[M, K] * B[N, K]^T on the 5th-generation tensor cores (tcgen05.mma, bf16 inputs,
 // fp32 accumulation in TMEM), operands streamed by TMA through a shared-memory ring.
-// One CTA computes one 128 x BN output tile (BN a multiple of 32, at most 256):
+// One CTA computes `ncb` adjacent 128 x BN output tiles of the same 128 rows (BN a multiple of 32, at
+// most 256; ncb accumulators side by side in TMEM), so that the A tile is loaded once for all of them:
 //   warp 0      TMA producer (one elected lane)
 //   warp 1      TMEM allocation + MMA issue (one elected lane)
 //   warps 2..5  epilogue: TMEM -> registers -> global, one TMEM lane quadrant each
@@ -26,8 +27,8 @@ constexpr int MAX_BN = 256;
 // the launch, so that short-K problems (one or two K blocks) leave room for several CTAs
 // per SM and one CTA's epilogue overlaps another's loads and MMAs.
 // The epilogue reuses the ring as a [128][BN + 8] bf16 staging tile, so the ring is never smaller than that.
-__host__ __device__ constexpr size_t smem_bytes(int stages, int bn, int b_mn_major) {
-  const size_t ring = (size_t)stages * (BM * BK * 2 + (size_t)(b_mn_major ? (bn + 63) / 64 * 64 : bn) * BK * 2);
+__host__ __device__ constexpr size_t smem_bytes(int stages, int bn, int b_mn_major, int ncb = 1) {
+  const size_t ring = (size_t)stages * (BM * BK * 2 + (size_t)ncb * (b_mn_major ? (bn + 63) / 64 * 64 : bn) * BK * 2);
   const size_t stage_tile = (size_t)BM * (bn + 8) * 2;
   return 1024 /*align slack*/ + (ring > stage_tile ? ring : stage_tile);
 }
@@ -50,6 +51,7 @@ struct Seg {
 
 struct Params {
   int M, K, BN, nseg;
+  int ncb;                 // column blocks (accumulators) per CTA: 1, or nseg when every segment is one block wide
   int stages;              // ring depth, 1..MAX_STAGES
   int b_mn_major;          // 1: B is given as [K, N] with N contiguous (no transpose needed)
   Seg seg[3];
@@ -76,22 +78,29 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int n_bbox = (p.BN + 63) / 64;
   const uint32_t a_bytes = BM * BK * 2;
   const uint32_t b_bytes = p.b_mn_major ? (uint32_t)n_bbox * (64 * BK * 2) : (uint32_t)p.BN * BK * 2;
-  auto a_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + b_bytes); };
-  auto b_tile = [&](int s) { return tiles + (size_t)s * (a_bytes + b_bytes) + a_bytes; };
+  const int ncb = p.ncb;
+  const uint32_t stage_sz = a_bytes + (uint32_t)ncb * b_bytes;
+  auto a_tile = [&](int s) { return tiles + (size_t)s * stage_sz; };
+  auto b_tile = [&](int s, int cb) { return tiles + (size_t)s * stage_sz + a_bytes + (size_t)cb * b_bytes; };
   const int STAGES = p.stages;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.BN;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.BN * ncb;
   const int num_kb_all = (p.K + BK - 1) / BK;
   const int kb_begin = p.kb_per_split > 0 ? (int)blockIdx.z * p.kb_per_split : 0;
   const int num_kb = p.kb_per_split > 0 ? min(p.kb_per_split, num_kb_all - kb_begin) : num_kb_all;
   Abort ab{&abort_flag, p.err};
-  // segment of this tile's columns, and where they sit in their B tensor map
-  int si = 0;
-  while (si + 1 < p.nseg && n0 >= p.seg[si + 1].n_begin) ++si;
-  const int bn0 = n0 - p.seg[si].n_begin + p.seg[si].b_n_off;
-  const CUtensorMap* tmB = p.seg[si].bmap == 0 ? &tmB0 : (p.seg[si].bmap == 1 ? &tmB1 : &tmB2);
-  const uint32_t ncols_tmem = tmem_cols(p.BN);
+  // segment of column block cb, and where its columns sit in their B tensor map
+  auto seg_of = [&](int cb) {
+    const int nb = n0 + cb * p.BN;
+    int si = 0;
+    while (si + 1 < p.nseg && nb >= p.seg[si + 1].n_begin) ++si;
+    return si;
+  };
+  auto bmap_of = [&](int si) { return p.seg[si].bmap == 0 ? &tmB0 : (p.seg[si].bmap == 1 ? &tmB1 : &tmB2); };
+  const uint32_t acc_cols = tmem_cols(p.BN);                 // columns of one accumulator
+  uint32_t ncols_tmem = acc_cols;                            // allocation: power of two >= ncb accumulators
+  while (ncols_tmem < (uint32_t)ncb * acc_cols) ncols_tmem *= 2;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -114,19 +123,24 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 0) {
     if (elect_one()) {
       tma_prefetch_desc(&tmA);
-      tma_prefetch_desc(tmB);
+      tma_prefetch_desc(bmap_of(seg_of(0)));
       for (int kb = 0; kb < num_kb; ++kb) {
         const int s = kb % STAGES;
         const uint32_t ph = (kb / STAGES) & 1;
         if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+        mbar_expect_tx(&full_bar[s], stage_sz);
         const int kx = (kb_begin + kb) * BK;
         tma_load_2d(a_tile(s), &tmA, &full_bar[s], kx, m0);
-        if (!p.b_mn_major) {
-          tma_load_2d(b_tile(s), tmB, &full_bar[s], kx, bn0);
-        } else {
-          for (int j = 0; j < n_bbox; ++j)   // one [64 k-rows x 64 n] box per 64 columns
-            tma_load_2d(b_tile(s) + j * (64 * BK * 2), tmB, &full_bar[s], bn0 + j * 64, kx);
+        for (int cb = 0; cb < ncb; ++cb) {
+          const int si = seg_of(cb);
+          const int bn0 = n0 + cb * p.BN - p.seg[si].n_begin + p.seg[si].b_n_off;
+          const CUtensorMap* tmB = bmap_of(si);
+          if (!p.b_mn_major) {
+            tma_load_2d(b_tile(s, cb), tmB, &full_bar[s], kx, bn0);
+          } else {
+            for (int j = 0; j < n_bbox; ++j)   // one [64 k-rows x 64 n] box per 64 columns
+              tma_load_2d(b_tile(s, cb) + j * (64 * BK * 2), tmB, &full_bar[s], bn0 + j * 64, kx);
+          }
         }
       }
     }
@@ -140,7 +154,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         ok = mbar_wait(&full_bar[s], ph, ab);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(a_tile(s)), b_addr = smem_u32(b_tile(s));
+        const uint32_t a_addr = smem_u32(a_tile(s));
+        for (int cb = 0; cb < ncb; ++cb) {
+        const uint32_t b_addr = smem_u32(b_tile(s, cb));
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k) {
           const uint64_t ad = umma_desc_kmajor_sw128(a_addr + k * 32);
@@ -157,7 +173,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             bd |= (uint64_t)1 << 46;
             bd |= (uint64_t)2 << 61;
           }
-          umma_ss(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_ss(tmem_base + (uint32_t)cb * acc_cols, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+        }
         }
         umma_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
       }
@@ -167,17 +184,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32)
     const int q = warp % 4;
     const int row = m0 + q * 32 + lane;
-    const Seg sg = p.seg[si];
-    const int c0 = n0 - sg.n_begin;       // first column of this tile inside its segment
     const bool ok = mbar_wait(&acc_bar, 0, ab);
     tc_fence_after();
-    if (ok) {
+    if (ok) for (int cb = 0; cb < ncb; ++cb) {
+      const Seg sg = p.seg[seg_of(cb)];
+      const int c0 = n0 + cb * p.BN - sg.n_begin;       // first column of this block inside its segment
+      const uint32_t acc = tmem_base + (uint32_t)cb * acc_cols + ((uint32_t)(q * 32) << 16);
       const int rloc = q * 32 + lane;
       const int npos = p.n_pos > 0 ? row % p.n_pos : row;
       if (sg.mode == EP_F32) {
         for (int ch = 0; ch < p.BN / 32; ++ch) {
           uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
+          tmem_ld32(acc + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
           if (row >= p.M) continue;
           float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)blockIdx.z * p.split_stride +
@@ -196,7 +214,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint8_t* stage = tiles;
         for (int ch = 0; ch < p.BN / 32; ++ch) {
           uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), r);
+          tmem_ld32(acc + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
           const int col = c0 + ch * 32;
           uint32_t o[16];
@@ -236,6 +254,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           }
         }
+        __syncwarp();   // the warp's staging rows are free again before the next block is converted
       }
     }
   }
