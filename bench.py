@@ -33,6 +33,8 @@ import numpy as np
 
 from paper_2603_30033_b200 import workloads as W
 
+LIB_FLAGS = 0   # TA_FLAG_* bits for every library call (set from --flags)
+
 METRIC = "prefill TFLOP/s & decode GB/s vs B200 roofline (fused Tucker attention)"
 KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
 L2_BYTES = 126 * 1024 * 1024
@@ -177,7 +179,7 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
     desc = Bd.make_desc(B=w.B, N=w.N, d_model=w.d_model, n_H=w.n_H, r=w.r, t=w.t, causal=w.causal, rope=w.rope,
                         rope_base=w.rope_base, dtype=Bd.TA_DTYPE_BF16 if w.dtype == "bf16" else Bd.TA_DTYPE_F32)
     ws = Bd.alloc_workspace(Bd.fwd_workspace_bytes(desc), X.device)
-    kw = dict(n_H=w.n_H, causal=w.causal, rope=w.rope, rope_base=w.rope_base, out=Y, workspace=ws)
+    kw = dict(n_H=w.n_H, causal=w.causal, rope=w.rope, rope_base=w.rope_base, out=Y, workspace=ws, flags=LIB_FLAGS)
 
     def step():
         Bd.tucker_attn_fwd(X, *dw, **kw)
@@ -250,7 +252,7 @@ def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sam
     desc = Bd.make_desc(B=B, N=1, d_model=w.d_model, n_H=w.n_H, r=w.r, t=w.t, causal=True, rope=w.rope,
                         rope_base=w.rope_base, dtype=Bd.TA_DTYPE_BF16 if w.dtype == "bf16" else Bd.TA_DTYPE_F32)
     ws = Bd.alloc_workspace(Bd.decode_workspace_bytes(desc, Lmax), x.device)
-    kw = dict(n_H=w.n_H, rope=w.rope, rope_base=w.rope_base, append=True, out=y, workspace=ws)
+    kw = dict(n_H=w.n_H, rope=w.rope, rope_base=w.rope_base, append=True, out=y, workspace=ws, flags=LIB_FLAGS)
 
     def step():
         Bd.tucker_attn_decode(x, *dw, Kc, Vc, lens, **kw)
@@ -409,8 +411,11 @@ def main():
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the secondary workloads")
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="TA_FLAG_* bits passed to the library (route selection)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    global LIB_FLAGS
+    LIB_FLAGS = args.flags
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

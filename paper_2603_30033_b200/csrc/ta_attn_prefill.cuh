@@ -74,17 +74,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
 __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
 
-// MN-major B operand (V tile as loaded: rows = keys, 64-column blocks), 128-byte swizzle.
-__device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint32_t block_pitch_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)(block_pitch_bytes >> 4) << 16;   // leading offset: next 64-column block
-  d |= (uint64_t)(1024u >> 4) << 32;               // stride offset: next group of 8 key rows
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
-
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,

@@ -1,0 +1,485 @@
+// Decode attention over the latent KV cache (Eq. 9) on tcgen05 tensor cores.
+//
+// Same job, same tile split and same partial format as dec::k_dec_attn (the mma.sync kernel), but the
+// two products of a 128-key tile run as UMMA instructions with the KEYS on the M dimension, so that
+// no tensor work is spent on padding the (at most 32) heads up to a 128-row tile:
+//   S^T [128 keys x 32 heads] = K_tile [128 x r3] * Qhat^T          A = K tile as loaded (K-major), B = Qhat (K-major)
+//   O^T [t3 x 32 heads]      += V_tile^T [t3 x 128] * P [128 x 32]  A = V tile as loaded (M-major), B = P (K-major, bf16)
+// The scores of one tile sit in TMEM with one key per lane and one head per column: a softmax thread
+// owns one key and all heads.  The per-head maximum over the keys of a tile is therefore a reduction
+// ACROSS threads (a transposing butterfly of warp shuffles, then four values per head through shared
+// memory); it only moves the reference maximum of a head when that grows by more than 8 (factor 256),
+// so the accumulator in TMEM is rescaled rarely.  P goes back through shared memory (B operands are
+// read from there); the row sums stay in registers per thread and are reduced once per segment.
+//
+// Two softmax warpgroups take alternate tiles, each with its own score buffer, P buffer, output
+// accumulator and online-softmax state, so that the chain scores -> softmax -> P V of one tile overlaps
+// the next tile's; their two states are merged (log-sum-exp weights) when a segment ends, and one
+// partial per (CTA, sequence) is written exactly as the mma.sync kernel writes it.
+//
+//   warp 0       TMA producer: Qhat of the segment's sequence, K / V ring
+//   warp 1       TMEM allocation, MMA issue
+//   warps 4..7   softmax warpgroup 0 (even tiles)     warps 8..11  softmax warpgroup 1 (odd tiles)
+// TMEM columns: S_0 [0,32) S_1 [32,64) O_0 [64,96) O_1 [96,128).
+// Every wait is bounded (Abort): on a timeout the CTA raises the device error word and leaves.
+#pragma once
+
+#include "ta_common.cuh"
+#include "ta_decode.cuh"
+#include "ta_sm100.cuh"
+
+namespace ta {
+namespace decu {
+
+using namespace sm100;
+using dec::clamp_len;
+using dec::tiles_of;
+
+constexpr int TK = 128;                  // keys per tile
+constexpr int THREADS = 384;
+constexpr int STAGES = 3;
+constexpr int SUB_BYTES = 128 * 64 * 2;  // [128 keys x 64] bf16
+constexpr int MAX_SUB = 2;               // r3, t3 <= 128
+constexpr int STAGE_BYTES = 2 * MAX_SUB * SUB_BYTES;   // K tile + V tile
+constexpr int QSUB_BYTES = 32 * 64 * 2;  // [32 heads x 64] bf16 (Qhat and P sub-tiles)
+constexpr int QBUF_BYTES = MAX_SUB * QSUB_BYTES;
+constexpr int PBUF_BYTES = 2 * QSUB_BYTES;             // [32 heads x 128 keys] bf16
+// ring | Qhat (two segments in flight) | P_0 | P_1   (P_0 and P_1 together double as the 16 KB merge buffer)
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 2 * QBUF_BYTES + 2 * PBUF_BYTES;
+constexpr float kRescaleThreshold = 8.f;
+
+struct Params {
+  int B, nH, Lmax, r3, t3;
+  int shared_kv;       // 1: one latent cache L^KV (Sec. 3.1): the K tile is the V tile
+  const int32_t* cache_len;
+  const bf16* knew;    // [B, r3] rotated new key
+  const bf16* vnew;    // [B, t3] new value
+  float* part_o;       // [grid + B][32][t3]
+  float* part_ml;      // [grid + B][32][2]  (max in log2 units, sum)
+  unsigned int* err;
+};
+
+// Walks this CTA's range of the flat tile list, sequence by sequence.
+struct Walk {
+  const int32_t* cache_len;
+  int Lmax;
+  long t_begin, t_end;
+  int b;
+  long first, nt;
+  int L;
+  __device__ void init(const Params& p, long tb, long te, int b0, long first0) {
+    cache_len = p.cache_len; Lmax = p.Lmax; t_begin = tb; t_end = te;
+    b = b0; first = first0;
+    L = clamp_len(cache_len[b], Lmax);
+    nt = tiles_of(L);
+  }
+  __device__ void seek(long t) {
+    while (t >= first + nt) {
+      first += nt;
+      ++b;
+      L = clamp_len(cache_len[b], Lmax);
+      nt = tiles_of(L);
+    }
+  }
+  __device__ bool seg_start(long t) const { return t == t_begin || t == first; }
+  __device__ bool seg_end(long t) const { return t == t_end - 1 || t == first + nt - 1; }
+  __device__ int k0(long t) const { return (int)(t - first) * TK; }
+  __device__ bool last_tile(long t) const { return k0(t) + TK > L; }
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+  return (uint32_t)((chunk >> 3) * SUB_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+// v[j] of every lane -> lane j receives op over the 32 lanes of v[j] (returned in v[0]).
+template <bool IS_MAX>
+__device__ __forceinline__ float transpose_reduce(float (&v)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < off; ++i) {
+      const float send = up ? v[i] : v[i + off];
+      const float keep = up ? v[i + off] : v[i];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, off);
+      v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
+    }
+  }
+  return v[0];
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmQ, const Params p) {
+  pdl_enter();
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], q_full[2], q_empty[2];
+  __shared__ uint64_t s_full[2], p_full[2], o_full[2], o_read[2], patched[2], wg_bar[2], cta_bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ float mx_s[2][4][32];     // per warpgroup, per warp: tile maxima per head, later row sums
+  __shared__ float m_s[2][32];         // per warpgroup: reference maximum per head (segment merge)
+  __shared__ long long wtot_s[THREADS / 32];
+  __shared__ int loc_b;
+  __shared__ long long loc_first;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* ring = smem_raw + (base - smem_u32(smem_raw));
+  uint8_t* qbuf = ring + (size_t)STAGES * STAGE_BYTES;
+  uint8_t* pbuf = qbuf + 2 * QBUF_BYTES;
+  float* obuf = reinterpret_cast<float*>(pbuf);       // merge buffer [32][t3] fp32 (aliases P_0 | P_1)
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  Abort ab{&abort_flag, p.err};
+  const int ksub = (p.r3 + 63) / 64, vsub = (p.t3 + 63) / 64;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&q_full[i], 1);
+      mbar_init(&q_empty[i], 1);
+      mbar_init(&s_full[i], 1);
+      mbar_init(&p_full[i], 4);      // one arrival per softmax warp
+      mbar_init(&o_full[i], 1);
+      mbar_init(&o_read[i], 4);
+      mbar_init(&patched[i], 4);
+      mbar_init(&wg_bar[i], 4);
+    }
+    mbar_init(&cta_bar, 8);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  const uint32_t tm_s[2] = {tmem, tmem + 32};
+  const uint32_t tm_o[2] = {tmem + 64, tmem + 96};
+
+  // ---- this CTA's range of the flat tile list (same split as the mma.sync kernel) ----
+  int lo, hi;
+  long excl;
+  const long total = dec::block_tile_scan(p.cache_len, p.B, p.Lmax, lo, hi, excl, wtot_s);
+  const long t_begin = dec::cta_first_tile(blockIdx.x, total, gridDim.x);
+  const long t_end = dec::cta_first_tile(blockIdx.x + 1, total, gridDim.x);
+  {
+    long f = excl;
+    for (int b = lo; b < hi; ++b) {
+      const long nt = tiles_of(clamp_len(p.cache_len[b], p.Lmax));
+      if (t_begin >= f && t_begin < f + nt) { loc_b = b; loc_first = f; }
+      f += nt;
+    }
+  }
+  __syncthreads();
+  const bool have_work = t_begin < t_end;
+  const int b0 = have_work ? loc_b : 0;
+  const long seq_first = have_work ? (long)loc_first : 0;
+
+  if (warp < 4) {
+   // the producer / MMA warpgroup hands registers to the softmax warpgroups (32 scores, 32 reference
+   // maxima, 32 row sums and a 32-wide scratch per thread)
+   asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+   if (have_work && warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (elect_one()) {
+      tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmQ);
+      Walk w;
+      w.init(p, t_begin, t_end, b0, seq_first);
+      int it = 0, seg = -1;
+      for (long t = t_begin; t < t_end; ++t, ++it) {
+        w.seek(t);
+        if (w.seg_start(t)) {
+          ++seg;
+          const int qb = seg & 1;
+          if (!mbar_wait(&q_empty[qb], ((seg >> 1) & 1) ^ 1, ab)) break;
+          mbar_expect_tx(&q_full[qb], (uint32_t)(ksub * QSUB_BYTES));
+          for (int kk = 0; kk < ksub; ++kk)
+            tma_load_2d(qbuf + qb * QBUF_BYTES + kk * QSUB_BYTES, &tmQ, &q_full[qb], kk * 64, w.b * p.nH);
+        }
+        const int s = it % STAGES;
+        if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, ab)) break;
+        mbar_expect_tx(&full_bar[s], (uint32_t)((ksub + (p.shared_kv ? 0 : vsub)) * SUB_BYTES));
+        uint8_t* kt = ring + (size_t)s * STAGE_BYTES;
+        uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
+        const int row = w.k0(t);
+        for (int kk = 0; kk < ksub; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, w.b);
+        if (!p.shared_kv)
+          for (int kk = 0; kk < vsub; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, w.b);
+      }
+    }
+   } else if (have_work && warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------
+    if (elect_one()) {
+      const uint32_t idesc_qk = umma_idesc_bf16(128, 32);
+      const uint32_t idesc_pv = umma_idesc_bf16(128, 32) | (1u << 15);   // A = V tile is M-major
+      const int ksteps = p.r3 / 16;
+      struct Pending { int it, s, wg, seg; bool first_of_wg; bool valid; };
+      Pending pend = {0, 0, 0, 0, false, false};
+      bool ok = true;
+      auto issue_pv = [&](const Pending& pv) -> bool {
+        const int j = pv.it >> 1;
+        if (!mbar_wait(&p_full[pv.wg], (uint32_t)(j & 1), ab)) return false;
+        // the accumulator of the previous segment must have been read before it is overwritten
+        if (pv.first_of_wg && pv.seg > 0 && !mbar_wait(&o_read[pv.wg], (uint32_t)((pv.seg - 1) & 1), ab)) return false;
+        tc_fence_after();
+        uint8_t* kt = ring + (size_t)pv.s * STAGE_BYTES;
+        const uint32_t va = smem_u32(p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES);
+        const uint32_t pa = smem_u32(pbuf + pv.wg * PBUF_BYTES);
+        for (int ks = 0; ks < TK / 16; ++ks) {
+          const uint32_t poff = (uint32_t)(ks >> 2) * QSUB_BYTES + (uint32_t)(ks & 3) * 32;
+          umma_ss(tm_o[pv.wg], umma_desc_mnmajor_sw128(va + (uint32_t)ks * 2048, SUB_BYTES),
+                  umma_desc_kmajor_sw128(pa + poff), idesc_pv, (pv.first_of_wg && ks == 0) ? 0u : 1u);
+        }
+        umma_commit(&o_full[pv.wg]);
+        umma_commit(&empty_bar[pv.s]);
+        return true;
+      };
+      Walk w;
+      w.init(p, t_begin, t_end, b0, seq_first);
+      int it = 0, seg = -1;
+      int wg_tiles[2] = {0, 0};      // tiles of the current segment issued per warpgroup
+      int n_last[2] = {0, 0};        // patched (last) tiles seen per warpgroup
+      for (long t = t_begin; t < t_end && ok; ++t, ++it) {
+        w.seek(t);
+        const int wg = it & 1, s = it % STAGES;
+        if (w.seg_start(t)) {
+          ++seg;
+          wg_tiles[0] = wg_tiles[1] = 0;
+          if (!(ok = mbar_wait(&q_full[seg & 1], (uint32_t)((seg >> 1) & 1), ab))) break;
+        }
+        if (!(ok = mbar_wait(&full_bar[s], (uint32_t)((it / STAGES) & 1), ab))) break;
+        if (w.last_tile(t)) {
+          // The warpgroup patches this tile only after it has flushed the segments before it, and such a
+          // flush waits for the pending P V: issue that first (normally it follows the next scores).
+          if (pend.valid) {
+            if (!(ok = issue_pv(pend))) break;
+            pend.valid = false;
+          }
+          if (!(ok = mbar_wait(&patched[wg], (uint32_t)(n_last[wg] & 1), ab))) break;
+          ++n_last[wg];
+        }
+        tc_fence_after();
+        {
+          const uint32_t ka = smem_u32(ring + (size_t)s * STAGE_BYTES);
+          const uint32_t qa = smem_u32(qbuf + (seg & 1) * QBUF_BYTES);
+          for (int ks = 0; ks < ksteps; ++ks) {
+            const uint32_t koff = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
+            const uint32_t qoff = (uint32_t)(ks >> 2) * QSUB_BYTES + (uint32_t)(ks & 3) * 32;
+            umma_ss(tm_s[wg], umma_desc_kmajor_sw128(ka + koff), umma_desc_kmajor_sw128(qa + qoff), idesc_qk, ks != 0);
+          }
+          umma_commit(&s_full[wg]);
+          if (w.seg_end(t)) umma_commit(&q_empty[seg & 1]);   // the segment's Qhat buffer is free once these complete
+        }
+        if (pend.valid && !(ok = issue_pv(pend))) break;
+        pend.it = it; pend.s = s; pend.wg = wg; pend.seg = seg; pend.first_of_wg = (wg_tiles[wg] == 0); pend.valid = true;
+        ++wg_tiles[wg];
+      }
+      if (ok && pend.valid) (void)issue_pv(pend);
+    }
+   }
+  } else {
+   asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+   if (have_work) {
+    // ------------------------------- softmax warpgroups --------------------------
+    const int wg = (warp - 4) / 4;
+    const int q = warp % 4;                     // TMEM lane quadrant
+    const int tid = q * 32 + lane;              // key row of a score tile / value coordinate of O^T
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    uint8_t* my_p = pbuf + wg * PBUF_BYTES;
+    // this thread's P element (head h) lives at my_p + p_off + h * 128 + ((p_chunk ^ (h & 7)) << 4)
+    const uint32_t p_off = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(tid & 7) * 2;
+    const int p_chunk = (tid & 63) >> 3;
+    uint32_t wg_phase = 0, cta_phase = 0;
+    bool ok = true;
+    auto wg_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&wg_bar[wg]);
+      bool good = mbar_wait(&wg_bar[wg], wg_phase & 1, ab);
+      ++wg_phase;
+      return __all_sync(0xffffffffu, good);
+    };
+    auto cta_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&cta_bar);
+      bool good = mbar_wait(&cta_bar, cta_phase & 1, ab);
+      ++cta_phase;
+      return __all_sync(0xffffffffu, good);
+    };
+    Walk w;
+    w.init(p, t_begin, t_end, b0, seq_first);
+    int it = 0, seg = -1;
+    int n_mine = 0;            // tiles of the current segment handled by this warpgroup
+    int j_last = 0;            // index (it >> 1) of the latest tile handled by this warpgroup
+    float m_used[32], l_acc[32];
+    float m_lane = -INFINITY;  // m_used[lane]
+    for (long t = t_begin; t < t_end && ok; ++t, ++it) {
+      w.seek(t);
+      if (w.seg_start(t)) {
+        ++seg;
+        n_mine = 0;
+        m_lane = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < 32; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
+      }
+      if ((it & 1) == wg) {
+        const int s = it % STAGES, j = it >> 1;
+        const int k0 = w.k0(t), L = w.L;
+        const bool last_tile = w.last_tile(t);
+        if (last_tile) {
+          // the tile holding the new token: its row comes from the workspace, rows past it are invalid
+          ok = mbar_wait(&full_bar[s], (uint32_t)((it / STAGES) & 1), ab);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          uint8_t* kt = ring + (size_t)s * STAGE_BYTES;
+          uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;
+          const int rnew = L - k0;
+          if (tid == rnew) {
+            const uint4* ks = reinterpret_cast<const uint4*>(p.knew + (long)w.b * p.r3);
+            for (int c = 0; c < p.r3 / 8; ++c) *reinterpret_cast<uint4*>(kt + swz(tid, c)) = ks[c];
+            const uint4* vs = reinterpret_cast<const uint4*>(p.vnew + (long)w.b * p.t3);
+            for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = vs[c];
+          } else if (tid > rnew) {
+            for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&patched[wg]);
+        }
+        ok = mbar_wait(&s_full[wg], (uint32_t)(j & 1), ab);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sr[32];
+        tmem_ld32(tm_s[wg] + lane_addr, sr);
+        tmem_ld_wait();
+        float sc[32];
+        const bool visible = (k0 + tid) <= L;
+#pragma unroll
+        for (int h = 0; h < 32; ++h) sc[h] = visible ? __uint_as_float(sr[h]) : -INFINITY;
+        // ---- maximum per head over the 128 keys of the tile ----
+        float tmp[32];
+#pragma unroll
+        for (int h = 0; h < 32; ++h) tmp[h] = sc[h];
+        mx_s[wg][q][lane] = transpose_reduce<true>(tmp, lane);
+        if (!(ok = wg_sync())) break;
+        const float mt = fmaxf(fmaxf(mx_s[wg][0][lane], mx_s[wg][1][lane]), fmaxf(mx_s[wg][2][lane], mx_s[wg][3][lane]));
+        // every tile holds at least one visible key (the last one holds the new token), so mt is finite
+        const bool need = mt > m_lane + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? mt : m_lane;
+          const float f_lane = need ? ex2(m_lane - m_new) : 1.f;     // exp2(-inf) = 0 on the first tile
+          float fac[32];
+#pragma unroll
+          for (int h = 0; h < 32; ++h) {
+            fac[h] = __shfl_sync(0xffffffffu, f_lane, h);
+            m_used[h] = __shfl_sync(0xffffffffu, m_new, h);
+            l_acc[h] *= fac[h];
+          }
+          m_lane = m_new;
+          if (n_mine > 0) {
+            ok = mbar_wait(&o_full[wg], (uint32_t)(j_last & 1), ab);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t o[32];
+            tmem_ld32(tm_o[wg] + lane_addr, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int h = 0; h < 32; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * fac[h]);
+            tmem_st32(tm_o[wg] + lane_addr, o);
+            tmem_st_wait();
+          }
+        }
+        // (mx_s is written again only after the next s_full wait of this group, and the MMA issuer
+        // issues those scores after it saw all four warps' arrivals on p_full of this tile, i.e. after
+        // every warp's reads above.)
+        // ---- p = exp2(s - m), bf16, into the P operand; row sums per thread ----
+#pragma unroll
+        for (int h = 0; h < 32; ++h) {
+          const float pv = ex2(sc[h] - m_used[h]);
+          l_acc[h] += pv;
+          const __nv_bfloat16 pb = __float2bfloat16_rn(pv);
+          *reinterpret_cast<__nv_bfloat16*>(my_p + p_off + h * 128 + ((p_chunk ^ (h & 7)) << 4)) = pb;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[wg]);
+        ++n_mine;
+        j_last = j;
+      }
+      if (w.seg_end(t)) {
+        // ---- segment done: merge the two warpgroups' states, write the partial of (CTA, sequence) ----
+        float o[32];
+        if (n_mine > 0) {
+          ok = mbar_wait(&o_full[wg], (uint32_t)(j_last & 1), ab);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t orr[32];
+          tmem_ld32(tm_o[wg] + lane_addr, orr);
+          tmem_ld_wait();
+#pragma unroll
+          for (int h = 0; h < 32; ++h) o[h] = __uint_as_float(orr[h]);
+        } else {
+#pragma unroll
+          for (int h = 0; h < 32; ++h) o[h] = 0.f;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&o_read[wg]);
+        float tmp[32];
+#pragma unroll
+        for (int h = 0; h < 32; ++h) tmp[h] = l_acc[h];
+        mx_s[wg][q][lane] = transpose_reduce<false>(tmp, lane);    // row sums over this warp's 32 keys
+        if (q == 0) m_s[wg][lane] = m_lane;
+        if (!(ok = cta_sync())) break;
+        const float ma = m_s[0][lane], mb = m_s[1][lane];
+        const float M = fmaxf(ma, mb);                               // finite: the segment has at least one tile
+        const float wa = (ma == -INFINITY) ? 0.f : ex2(ma - M), wb = (mb == -INFINITY) ? 0.f : ex2(mb - M);
+        const float Ltot = (mx_s[0][0][lane] + mx_s[0][1][lane] + mx_s[0][2][lane] + mx_s[0][3][lane]) * wa +
+                           (mx_s[1][0][lane] + mx_s[1][1][lane] + mx_s[1][2][lane] + mx_s[1][3][lane]) * wb;
+        const float w_own = wg == 0 ? wa : wb;
+        const long slot = (long)blockIdx.x + w.b;
+        if (wg == 1 && tid < p.t3) {      // warp-uniform: t3 is a multiple of 32
+#pragma unroll
+          for (int h = 0; h < 32; ++h) obuf[h * p.t3 + tid] = o[h] * __shfl_sync(0xffffffffu, w_own, h);
+        }
+        if (!(ok = cta_sync())) break;
+        if (wg == 0) {
+          float* dst = p.part_o + slot * 32 * p.t3;
+#pragma unroll
+          for (int h = 0; h < 32; ++h) {
+            const float wh = __shfl_sync(0xffffffffu, w_own, h);
+            if (tid < p.t3) dst[h * p.t3 + tid] = o[h] * wh + obuf[h * p.t3 + tid];
+          }
+          if (q == 0) {
+            float* ml = p.part_ml + slot * 64;
+            ml[lane * 2 + 0] = M;
+            ml[lane * 2 + 1] = Ltot;
+          }
+        }
+        if (!(ok = cta_sync())) break;   // the merge buffer aliases the P operands of the next segment
+      }
+    }
+   }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 128);
+}
+
+}  // namespace decu
+}  // namespace ta

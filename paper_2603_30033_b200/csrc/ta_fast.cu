@@ -12,6 +12,7 @@
 #include "ta_umma_gemm.cuh"
 #include "ta_attn_prefill.cuh"
 #include "ta_decode.cuh"
+#include "ta_decode_umma.cuh"
 #include "ta_zy_fused.cuh"
 
 #include <math.h>
@@ -505,6 +506,28 @@ int launch_dec_attn(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, 
   return TA_OK;
 }
 
+// The tcgen05 form of the cache-streaming kernel (keys on the M dimension, ranks at run time).
+int launch_dec_attn_umma(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const dec::Params& dp, int grid) {
+  const tucker_attn_desc& d = p.d;
+  CUtensorMap tmQ;   // Qhat [B * n_H rows, r3]: one box = 32 rows (all heads of a sequence) x 64 columns
+  if (!tmap_2d(&tmQ, dp.qhat, (uint64_t)d.r3, (uint64_t)d.B * d.n_H, (uint64_t)d.r3, 64, 32)) return TA_ERR_CUDA;
+  decu::Params up;
+  up.B = dp.B; up.nH = dp.nH; up.Lmax = dp.Lmax; up.r3 = d.r3; up.t3 = d.t3; up.shared_kv = dp.shared_kv;
+  up.cache_len = dp.cache_len; up.knew = dp.knew; up.vnew = dp.vnew;
+  up.part_o = dp.part_o; up.part_ml = dp.part_ml; up.err = dp.err;
+  static bool attr_set = false;
+  if (!attr_set) {
+    TA_CUDA_TRY(cudaFuncSetAttribute(decu::k_dec_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)decu::SMEM_BYTES));
+    attr_set = true;
+  }
+  prof_begin(p);
+  (void)launch_pdl(decu::k_dec_attn_umma, dim3(grid), dim3(decu::THREADS), decu::SMEM_BYTES, p.stream, tmK, tmV, tmQ, up);
+  prof_end(p);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
+
 bool dec_rank_ok(int r3, int t3) {
   return (r3 == 128 && t3 == 128) || (r3 == 64 && t3 == 64) || (r3 == 96 && t3 == 96) || (r3 == 128 && t3 == 64) ||
          (r3 == 64 && t3 == 128);
@@ -581,7 +604,8 @@ int fast_decode(Problem& p) {
     dp.shared_kv = p.shared_kv;
     dp.cache_len = p.cache_len; dp.qhat = w.qhat; dp.knew = w.knew; dp.vnew = w.vnew;
     dp.part_o = w.part_o; dp.part_ml = w.part_ml; dp.err = p.dev_err;
-    if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);
+    if (d.flags & TA_FLAG_UMMA_DECODE) rc = launch_dec_attn_umma(p, tmK, tmV, dp, dp.grid);
+    else if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);
     else if (d.r3 == 64 && d.t3 == 64) rc = launch_dec_attn<64, 64>(p, tmK, tmV, dp);
     else if (d.r3 == 96 && d.t3 == 96) rc = launch_dec_attn<96, 96>(p, tmK, tmV, dp);
     else if (d.r3 == 128 && d.t3 == 64) rc = launch_dec_attn<128, 64>(p, tmK, tmV, dp);

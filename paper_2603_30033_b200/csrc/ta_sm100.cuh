@@ -186,6 +186,18 @@ __device__ __forceinline__ uint64_t umma_desc_kmajor_sw128(uint32_t saddr) {
   return d;
 }
 
+// MN-major operand (a tile stored with its M or N index contiguous: rows = K index, 64-element blocks
+// of the M / N index `block_pitch_bytes` apart), 128-byte swizzle; stepping K by 16 rows adds 2048 bytes.
+__device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t saddr, uint32_t block_pitch_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(block_pitch_bytes >> 4) << 16;   // leading offset: next 64-column block
+  d |= (uint64_t)(1024u >> 4) << 32;               // stride offset: next group of 8 key rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 // Instruction descriptor: D fp32, A and B bf16, both K-major, shape M x N (x16).
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);

@@ -244,13 +244,14 @@ DEC_FAST = [
 ]
 
 
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
 @pytest.mark.parametrize("append", [True, False])
 @pytest.mark.parametrize("case", DEC_FAST)
-def test_decode_tensor_core_path(case, append):
+def test_decode_tensor_core_path(case, append, flags):
     case = dict(case)
     lens, Lmax = case.pop("lens"), case.pop("Lmax")
     w = H.custom_workload(kind="decode", dtype="bf16", rope=True, rope_base=500000.0, seed=23, **case)
-    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, len(lens), lens, Lmax, append=append)
+    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, len(lens), lens, Lmax, append=append, flags=flags)
     assert Bd.last_path() == 2
     check(y, ref, "bf16", f"decode {case}", scaled=True)
     Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
