@@ -37,15 +37,16 @@ using dec::tiles_of;
 
 constexpr int TK = 128;                  // keys per tile
 constexpr int THREADS = 384;
-constexpr int STAGES = 3;
+constexpr int MAX_STAGES = 6;
 constexpr int SUB_BYTES = 128 * 64 * 2;  // [128 keys x 64] bf16
 constexpr int MAX_SUB = 2;               // r3, t3 <= 128
 constexpr int STAGE_BYTES = 2 * MAX_SUB * SUB_BYTES;   // K tile + V tile
 constexpr int QSUB_BYTES = 32 * 64 * 2;  // [32 heads x 64] bf16 (Qhat and P sub-tiles)
 constexpr int QBUF_BYTES = MAX_SUB * QSUB_BYTES;
 constexpr int PBUF_BYTES = 2 * QSUB_BYTES;             // [32 heads x 128 keys] bf16
+constexpr int RING_BYTES = 3 * STAGE_BYTES;            // three K + V stages, or six K-only stages (shared cache)
 // ring | Qhat (two segments in flight) | P_0 | P_1   (P_0 and P_1 together double as the 16 KB merge buffer)
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + 2 * QBUF_BYTES + 2 * PBUF_BYTES;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)RING_BYTES + 2 * QBUF_BYTES + 2 * PBUF_BYTES;
 constexpr float kRescaleThreshold = 8.f;
 
 struct Params {
@@ -118,11 +119,17 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmQ, const Params p) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], q_full[2], q_empty[2];
-  __shared__ uint64_t s_full[2], p_full[2], o_full[2], o_read[2], patched[2], wg_bar[2], cta_bar;
+  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], q_full[2], q_empty[2];
+  __shared__ uint64_t s_full[2], s_free[2], p_full[2], o_full[2], o_read[2], patched[2], wg_bar[2], cta_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float mx_s[2][4][32];     // per warpgroup, per warp: tile maxima per head, later row sums
+  // Exchange area of the softmax warpgroups.  Per tile: the four warps' maxima per head, as bf16 (the
+  // reference maximum only has to be the same for all threads and close to the true one), double-
+  // buffered by tile parity because a warp may start its next tile while another still reads this
+  // one's.  Per segment flush: the four warps' row sums per head, fp32, in the same bytes.
+  __shared__ __align__(16) unsigned char xch_raw[2 * 4 * 32 * 4];
+  auto mxh = reinterpret_cast<__nv_bfloat16 (*)[2][4][32]>(xch_raw);   // [wg][tile parity][warp][head]
+  auto sum_s = reinterpret_cast<float (*)[4][32]>(xch_raw);            // [wg][warp][head]
   __shared__ float m_s[2][32];         // per warpgroup: reference maximum per head (segment merge)
   __shared__ long long wtot_s[THREADS / 32];
   __shared__ int loc_b;
@@ -130,7 +137,12 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* ring = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* qbuf = ring + (size_t)STAGES * STAGE_BYTES;
+  uint8_t* qbuf = ring + (size_t)RING_BYTES;
+  // With one shared latent cache a stage holds a K tile only: twice the stages, and the scores may
+  // run two tiles ahead of the P V products instead of one.
+  const int STAGES = p.shared_kv ? 6 : 3;
+  const int stage_bytes = p.shared_kv ? MAX_SUB * SUB_BYTES : STAGE_BYTES;
+  const int ahead = p.shared_kv ? 2 : 1;
   uint8_t* pbuf = qbuf + 2 * QBUF_BYTES;
   float* obuf = reinterpret_cast<float*>(pbuf);       // merge buffer [32][t3] fp32 (aliases P_0 | P_1)
 
@@ -140,7 +152,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < MAX_STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
@@ -148,6 +160,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mbar_init(&q_full[i], 1);
       mbar_init(&q_empty[i], 1);
       mbar_init(&s_full[i], 1);
+      mbar_init(&s_free[i], 4);      // the scores of a tile are in the warpgroup's registers
       mbar_init(&p_full[i], 4);      // one arrival per softmax warp
       mbar_init(&o_full[i], 1);
       mbar_init(&o_read[i], 4);
@@ -211,7 +224,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int s = it % STAGES;
         if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, ab)) break;
         mbar_expect_tx(&full_bar[s], (uint32_t)((ksub + (p.shared_kv ? 0 : vsub)) * SUB_BYTES));
-        uint8_t* kt = ring + (size_t)s * STAGE_BYTES;
+        uint8_t* kt = ring + (size_t)s * stage_bytes;
         uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
         const int row = w.k0(t);
         for (int kk = 0; kk < ksub; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, w.b);
@@ -222,71 +235,103 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
    } else if (have_work && warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (elect_one()) {
+      // This one thread issues 16 small MMAs per tile, so its own instruction stream is the critical
+      // resource: descriptors are formed once per operand and stepped by constants, the K loops are
+      // unrolled, and the (at most three) tiles between score issue and P V issue sit in registers.
       const uint32_t idesc_qk = umma_idesc_bf16(128, 32);
       const uint32_t idesc_pv = umma_idesc_bf16(128, 32) | (1u << 15);   // A = V tile is M-major
       const int ksteps = p.r3 / 16;
-      struct Pending { int it, s, wg, seg; bool first_of_wg; bool valid; };
-      Pending pend = {0, 0, 0, 0, false, false};
+      const uint64_t dq0 = umma_desc_kmajor_sw128(smem_u32(qbuf));
+      const uint64_t dp0 = umma_desc_kmajor_sw128(smem_u32(pbuf));
+      const uint64_t dk0 = umma_desc_kmajor_sw128(smem_u32(ring));
+      const uint64_t dv0 = umma_desc_mnmajor_sw128(smem_u32(ring) + (p.shared_kv ? 0u : (uint32_t)(MAX_SUB * SUB_BYTES)), SUB_BYTES);
+      const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);          // descriptor address fields count 16 bytes
+      // tile state packed in one word: it << 8 | stage << 4 | first_of_wg << 1 | (seg > 0)
+      uint32_t pq0 = 0, pq1 = 0, pq2 = 0;   // pending P V products, oldest first
+      int n_pend = 0;
+      int pv_seg0 = 0, pv_seg1 = 0, pv_seg2 = 0;
       bool ok = true;
-      auto issue_pv = [&](const Pending& pv) -> bool {
-        const int j = pv.it >> 1;
-        if (!mbar_wait(&p_full[pv.wg], (uint32_t)(j & 1), ab)) return false;
+      auto issue_pv = [&](uint32_t code, int sg) -> bool {
+        const int it = (int)(code >> 8), st = (int)((code >> 4) & 15), wg = it & 1;
+        const bool first_of_wg = (code & 2u) != 0;
+        if (!mbar_wait(&p_full[wg], (uint32_t)((it >> 1) & 1), ab)) return false;
         // the accumulator of the previous segment must have been read before it is overwritten
-        if (pv.first_of_wg && pv.seg > 0 && !mbar_wait(&o_read[pv.wg], (uint32_t)((pv.seg - 1) & 1), ab)) return false;
+        if (first_of_wg && sg > 0 && !mbar_wait(&o_read[wg], (uint32_t)((sg - 1) & 1), ab)) return false;
         tc_fence_after();
-        uint8_t* kt = ring + (size_t)pv.s * STAGE_BYTES;
-        const uint32_t va = smem_u32(p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES);
-        const uint32_t pa = smem_u32(pbuf + pv.wg * PBUF_BYTES);
-        for (int ks = 0; ks < TK / 16; ++ks) {
-          const uint32_t poff = (uint32_t)(ks >> 2) * QSUB_BYTES + (uint32_t)(ks & 3) * 32;
-          umma_ss(tm_o[pv.wg], umma_desc_mnmajor_sw128(va + (uint32_t)ks * 2048, SUB_BYTES),
-                  umma_desc_kmajor_sw128(pa + poff), idesc_pv, (pv.first_of_wg && ks == 0) ? 0u : 1u);
-        }
-        umma_commit(&o_full[pv.wg]);
-        umma_commit(&empty_bar[pv.s]);
+        const uint64_t dv = dv0 + stage_step * (uint64_t)st;
+        const uint64_t dp = dp0 + (uint64_t)(wg * (PBUF_BYTES >> 4));
+        const uint32_t d = tmem + 64u + (uint32_t)wg * 32u;
+        umma_ss(d, dv, dp, idesc_pv, first_of_wg ? 0u : 1u);
+#pragma unroll
+        for (int ks = 1; ks < TK / 16; ++ks)
+          umma_ss(d, dv + (uint64_t)(ks * 128), dp + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_pv, 1u);
+        umma_commit(&o_full[wg]);
+        umma_commit(&empty_bar[st]);
         return true;
+      };
+      auto pop_pv = [&]() -> bool {
+        const bool good = issue_pv(pq0, pv_seg0);
+        pq0 = pq1; pq1 = pq2; pv_seg0 = pv_seg1; pv_seg1 = pv_seg2;
+        --n_pend;
+        return good;
       };
       Walk w;
       w.init(p, t_begin, t_end, b0, seq_first);
-      int it = 0, seg = -1;
-      int wg_tiles[2] = {0, 0};      // tiles of the current segment issued per warpgroup
-      int n_last[2] = {0, 0};        // patched (last) tiles seen per warpgroup
-      for (long t = t_begin; t < t_end && ok; ++t, ++it) {
+      const int n_tiles = (int)(t_end - t_begin);
+      int seg = -1;
+      int st = 0;                    // ring stage of the next score tile, and the parity of its round
+      uint32_t st_par = 0;
+      int wg_tiles0 = 0, wg_tiles1 = 0;   // tiles of the current segment issued per warpgroup
+      int n_last0 = 0, n_last1 = 0;       // patched (last) tiles seen per warpgroup
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        // ---- keep the scores `ahead` tiles in front of the P V products ----
+        while (n_pend > ahead && ok) ok = pop_pv();
+        if (!ok) break;
+        const long t = t_begin + it;
         w.seek(t);
-        const int wg = it & 1, s = it % STAGES;
+        const int wg = it & 1, j = it >> 1;
         if (w.seg_start(t)) {
           ++seg;
-          wg_tiles[0] = wg_tiles[1] = 0;
+          wg_tiles0 = wg_tiles1 = 0;
           if (!(ok = mbar_wait(&q_full[seg & 1], (uint32_t)((seg >> 1) & 1), ab))) break;
         }
-        if (!(ok = mbar_wait(&full_bar[s], (uint32_t)((it / STAGES) & 1), ab))) break;
+        if (!(ok = mbar_wait(&full_bar[st], st_par, ab))) break;
         if (w.last_tile(t)) {
           // The warpgroup patches this tile only after it has flushed the segments before it, and such a
-          // flush waits for the pending P V: issue that first (normally it follows the next scores).
-          if (pend.valid) {
-            if (!(ok = issue_pv(pend))) break;
-            pend.valid = false;
-          }
-          if (!(ok = mbar_wait(&patched[wg], (uint32_t)(n_last[wg] & 1), ab))) break;
-          ++n_last[wg];
+          // flush waits for every P V issued so far: issue the pending ones first.
+          while (n_pend > 0 && ok) ok = pop_pv();
+          if (!ok) break;
+          int& nl = wg ? n_last1 : n_last0;
+          if (!(ok = mbar_wait(&patched[wg], (uint32_t)(nl & 1), ab))) break;
+          ++nl;
         }
+        // the warpgroup has taken the scores of its previous tile out of this buffer
+        if (j > 0 && !(ok = mbar_wait(&s_free[wg], (uint32_t)((j - 1) & 1), ab))) break;
         tc_fence_after();
         {
-          const uint32_t ka = smem_u32(ring + (size_t)s * STAGE_BYTES);
-          const uint32_t qa = smem_u32(qbuf + (seg & 1) * QBUF_BYTES);
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const uint32_t koff = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
-            const uint32_t qoff = (uint32_t)(ks >> 2) * QSUB_BYTES + (uint32_t)(ks & 3) * 32;
-            umma_ss(tm_s[wg], umma_desc_kmajor_sw128(ka + koff), umma_desc_kmajor_sw128(qa + qoff), idesc_qk, ks != 0);
-          }
+          const uint64_t dk = dk0 + stage_step * (uint64_t)st;
+          const uint64_t dq = dq0 + (uint64_t)((seg & 1) * (QBUF_BYTES >> 4));
+          const uint32_t d = tmem + (uint32_t)wg * 32u;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            if (ks < ksteps)
+              umma_ss(d, dk + (uint64_t)((ks >> 2) * (SUB_BYTES >> 4) + (ks & 3) * 2),
+                      dq + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_qk, ks != 0 ? 1u : 0u);
           umma_commit(&s_full[wg]);
           if (w.seg_end(t)) umma_commit(&q_empty[seg & 1]);   // the segment's Qhat buffer is free once these complete
         }
-        if (pend.valid && !(ok = issue_pv(pend))) break;
-        pend.it = it; pend.s = s; pend.wg = wg; pend.seg = seg; pend.first_of_wg = (wg_tiles[wg] == 0); pend.valid = true;
-        ++wg_tiles[wg];
+        {
+          int& wt = wg ? wg_tiles1 : wg_tiles0;
+          const uint32_t code = ((uint32_t)it << 8) | ((uint32_t)st << 4) | (wt == 0 ? 2u : 0u);
+          if (n_pend == 0) { pq0 = code; pv_seg0 = seg; }
+          else if (n_pend == 1) { pq1 = code; pv_seg1 = seg; }
+          else { pq2 = code; pv_seg2 = seg; }
+          ++n_pend;
+          ++wt;
+        }
+        if (++st == STAGES) { st = 0; st_par ^= 1u; }
       }
-      if (ok && pend.valid) (void)issue_pv(pend);
+      while (ok && n_pend > 0) ok = pop_pv();
     }
    }
   } else {
@@ -342,7 +387,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           ok = mbar_wait(&full_bar[s], (uint32_t)((it / STAGES) & 1), ab);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          uint8_t* kt = ring + (size_t)s * STAGE_BYTES;
+          uint8_t* kt = ring + (size_t)s * stage_bytes;
           uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;
           const int rnew = L - k0;
           if (tid == rnew) {
@@ -364,6 +409,9 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         uint32_t sr[32];
         tmem_ld32(tm_s[wg] + lane_addr, sr);
         tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_free[wg]);     // the next scores may overwrite the buffer
         float sc[32];
         const bool visible = (k0 + tid) <= L;
 #pragma unroll
@@ -372,9 +420,10 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         float tmp[32];
 #pragma unroll
         for (int h = 0; h < 32; ++h) tmp[h] = sc[h];
-        mx_s[wg][q][lane] = transpose_reduce<true>(tmp, lane);
+        mxh[wg][j & 1][q][lane] = __float2bfloat16_rn(transpose_reduce<true>(tmp, lane));
         if (!(ok = wg_sync())) break;
-        const float mt = fmaxf(fmaxf(mx_s[wg][0][lane], mx_s[wg][1][lane]), fmaxf(mx_s[wg][2][lane], mx_s[wg][3][lane]));
+        const float mt = fmaxf(fmaxf(__bfloat162float(mxh[wg][j & 1][0][lane]), __bfloat162float(mxh[wg][j & 1][1][lane])),
+                               fmaxf(__bfloat162float(mxh[wg][j & 1][2][lane]), __bfloat162float(mxh[wg][j & 1][3][lane])));
         // every tile holds at least one visible key (the last one holds the new token), so mt is finite
         const bool need = mt > m_lane + kRescaleThreshold;
         if (__any_sync(0xffffffffu, need)) {
@@ -402,10 +451,15 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             tmem_st_wait();
           }
         }
-        // (mx_s is written again only after the next s_full wait of this group, and the MMA issuer
-        // issues those scores after it saw all four warps' arrivals on p_full of this tile, i.e. after
-        // every warp's reads above.)
+        // (This parity's exchange buffer is written again two tiles on, after the group's sync of the
+        // tile in between, which every warp reaches only after its reads above.)
         // ---- p = exp2(s - m), bf16, into the P operand; row sums per thread ----
+        if (j > 0) {
+          // the P V of this group's previous tile must have finished reading the P buffer
+          ok = mbar_wait(&o_full[wg], (uint32_t)((j - 1) & 1), ab);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
 #pragma unroll
         for (int h = 0; h < 32; ++h) {
           const float pv = ex2(sc[h] - m_used[h]);
@@ -443,14 +497,14 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         float tmp[32];
 #pragma unroll
         for (int h = 0; h < 32; ++h) tmp[h] = l_acc[h];
-        mx_s[wg][q][lane] = transpose_reduce<false>(tmp, lane);    // row sums over this warp's 32 keys
+        sum_s[wg][q][lane] = transpose_reduce<false>(tmp, lane);   // row sums over this warp's 32 keys
         if (q == 0) m_s[wg][lane] = m_lane;
         if (!(ok = cta_sync())) break;
         const float ma = m_s[0][lane], mb = m_s[1][lane];
         const float M = fmaxf(ma, mb);                               // finite: the segment has at least one tile
         const float wa = (ma == -INFINITY) ? 0.f : ex2(ma - M), wb = (mb == -INFINITY) ? 0.f : ex2(mb - M);
-        const float Ltot = (mx_s[0][0][lane] + mx_s[0][1][lane] + mx_s[0][2][lane] + mx_s[0][3][lane]) * wa +
-                           (mx_s[1][0][lane] + mx_s[1][1][lane] + mx_s[1][2][lane] + mx_s[1][3][lane]) * wb;
+        const float Ltot = (sum_s[0][0][lane] + sum_s[0][1][lane] + sum_s[0][2][lane] + sum_s[0][3][lane]) * wa +
+                           (sum_s[1][0][lane] + sum_s[1][1][lane] + sum_s[1][2][lane] + sum_s[1][3][lane]) * wb;
         const float w_own = wg == 0 ? wa : wb;
         const long slot = (long)blockIdx.x + w.b;
         if (wg == 1 && tid < p.t3) {      // warp-uniform: t3 is a multiple of 32

@@ -277,7 +277,8 @@ def _shared_weights(w):
     ("bf16", dict(d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 64)), 2),
     ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
 ])
-def test_decode_shared_latent_cache(dtype, shape, path):
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
+def test_decode_shared_latent_cache(dtype, shape, path, flags):
     import torch
     w = H.custom_workload(kind="decode", dtype=dtype, rope=False, seed=61, **shape)
     wt = _shared_weights(w)
@@ -291,7 +292,7 @@ def test_decode_shared_latent_cache(dtype, shape, path):
     dw[7] = dw[3]                                        # the same device tensor for U3 and Ut3
     Kd = H.to_device(Kc, dtype)
     y = Bd.tucker_attn_decode(H.to_device(x, dtype), *dw, Kd, Kd, torch.from_numpy(cache_len).cuda(), n_H=w.n_H,
-                              rope=False, append=True)
+                              rope=False, append=True, flags=flags)
     assert Bd.last_device_error() == 0 and Bd.last_path() == path
     check(y.float().cpu().numpy().astype(np.float64), ref, dtype, f"shared decode {shape}", scaled=True)
     Kh = Kd.float().cpu().numpy()
