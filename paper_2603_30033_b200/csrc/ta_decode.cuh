@@ -142,7 +142,10 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 template <int R3, int T3>
 __global__ void __launch_bounds__(THREADS, 1)
 k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
-  pdl_enter();
+  // The cached rows below cache_len and cache_len itself were final before the preceding kernel (which
+  // forms the queries and appends the new row) began, so the tile split and the first ring loads run
+  // while it finishes; pdl_enter() comes before anything that kernel writes is read.  The new row's
+  // slot may be read half-written: it is replaced from the workspace below in any case.
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES];
   __shared__ int abort_flag;
@@ -214,8 +217,10 @@ k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUte
           for (int kk = 0; kk < VSUB; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, b);
       }
     }
+    pdl_enter();
   } else if (t_begin < t_end) {
     // ------------------------------- consumers ----------------------------------
+    pdl_enter();
     const int mt = warp / 4, kq = warp % 4;
     const int g = lane / 4, tq = lane % 4;
     int b = b0;

@@ -365,6 +365,7 @@ int fast_fwd(Problem& p) {
     const bool one_block_each = d.r2 == bn && d.r3 == bn && d.t3 == bn;
     if (one_block_each && (size_t)T * d.d_model * sizeof(bf16) > l2_bytes() && (T + 127) / 128 >= sm_count() * 4 / 5)
       gp.ncb = nseg;
+    gp.early = 1;   // X and the factors are inputs of the call: only the epilogue needs the preparation kernel's table
     if ((rc = launch_gemm(p, (const bf16*)p.X, d.d_model, T, d.d_model, bops, 3, ntot, bn, gp))) return rc;
   }
   const bf16* Vlat = p.shared_kv ? w.K : w.V;   // latent values
@@ -630,6 +631,7 @@ int fast_decode(Problem& p) {
     gp.nseg = 1;
     gp.seg[0] = seg(0, d.d_model, umma_gemm::EP_BF16, p.Y, d.d_model);
     const BOperand bop = {(const bf16*)p.Ut2, d.t2, d.d_model};
+    gp.early = 2;   // the factor Ut2 is an input of the call; z comes from the preceding kernel
     if ((rc = launch_gemm(p, w.z, d.t2, d.B, d.t2, &bop, 1, d.d_model, pick_bn(d.d_model), gp))) return rc;
   }
   return TA_OK;

@@ -57,6 +57,8 @@ struct Params {
   Seg seg[3];
   const float2* rope_tab;  // [n_pos][rope_half] (cos, sin); EP_BF16_ROPE only
   int n_pos, rope_half;    // row -> position = row % n_pos; RoPE period in columns = 2*rope_half
+  int early;               // 0: everything waits for the preceding kernel; 1: A and B were complete before the
+                           // preceding kernel started, only the epilogue (tables, outputs) waits; 2: B only
   int kb_per_split;        // split-K: 64-wide K blocks per blockIdx.z (0 = no split); EP_F32 outputs only
   long split_stride;       // elements between the partial outputs of consecutive splits
   unsigned int* err;
@@ -65,7 +67,10 @@ struct Params {
 __global__ void __launch_bounds__(THREADS, 2)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const Params p) {
-  pdl_enter();
+  // Operands that were final before the preceding kernel of the stream began may be fetched while that
+  // kernel still runs (Params::early); every thread still passes pdl_enter() before it touches anything
+  // the preceding kernel writes, and before it lets the next kernel be scheduled.
+  if (p.early == 0) pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], acc_bar;
   __shared__ uint32_t tmem_base_slot;
@@ -124,13 +129,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (elect_one()) {
       tma_prefetch_desc(&tmA);
       tma_prefetch_desc(bmap_of(seg_of(0)));
-      for (int kb = 0; kb < num_kb; ++kb) {
+      auto load_b = [&](int kb) {
         const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&full_bar[s], stage_sz);
         const int kx = (kb_begin + kb) * BK;
-        tma_load_2d(a_tile(s), &tmA, &full_bar[s], kx, m0);
         for (int cb = 0; cb < ncb; ++cb) {
           const int si = seg_of(cb);
           const int bn0 = n0 + cb * p.BN - p.seg[si].n_begin + p.seg[si].b_n_off;
@@ -142,8 +143,28 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               tma_load_2d(b_tile(s, cb) + j * (64 * BK * 2), tmB, &full_bar[s], bn0 + j * 64, kx);
           }
         }
+      };
+      int b_ahead = 0;               // K blocks whose B tiles were requested before the wait
+      if (p.early == 2) {
+        b_ahead = num_kb < STAGES ? num_kb : STAGES;
+        for (int kb = 0; kb < b_ahead; ++kb) {
+          mbar_expect_tx(&full_bar[kb], stage_sz);
+          load_b(kb);
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+      }
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (kb >= b_ahead) {
+          if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
+          mbar_expect_tx(&full_bar[s], stage_sz);
+          load_b(kb);
+        }
+        tma_load_2d(a_tile(s), &tmA, &full_bar[s], (kb_begin + kb) * BK, m0);
       }
     }
+    if (p.early) pdl_enter();
   } else if (warp == 1) {
     if (elect_one()) {
       const uint32_t idesc = umma_idesc_bf16(BM, p.BN) | (p.b_mn_major ? (1u << 16) : 0u);
@@ -180,8 +201,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       umma_commit(&acc_bar);          // accumulator complete
     }
+    if (p.early) pdl_enter();
   } else {
     // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32)
+    if (p.early) pdl_enter();
     const int q = warp % 4;
     const int row = m0 + q * 32 + lane;
     const bool ok = mbar_wait(&acc_bar, 0, ab);
