@@ -463,7 +463,6 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
            bf16* __restrict__ knew, bf16* __restrict__ vnew, bf16* __restrict__ Kc, bf16* __restrict__ Vc, int Lmax,
            const int32_t* __restrict__ cache_len, int rope, const RopeFreqs freqs, int append, int shared_kv,
            unsigned int* err) {
-  pdl_enter();
   constexpr int AB = 8 / NQ;                        // core slices per batch (8 loads of 16 bytes in flight per thread)
   __shared__ float qt_s[DQ_MAX_R2];                 // latent query of the new token
   __shared__ float k_s[DQ_CW];                      // this CTA's coordinates of the new key (unrotated)
@@ -494,6 +493,14 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     if (threadIdx.x == 0 && blockIdx.y == 0) atomicOr(err, (unsigned)TA_DEVERR_BAD_CACHE_LEN);
     L = clamp_len(L, Lmax);
   }
+  // Everything above and the two tables below depend on the call's inputs only (core, U1, cache_len)
+  // and runs while the projection GEMM before this kernel finishes; its partial sums are read after
+  // pdl_enter(), and nothing is written before it.
+  for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
+  if (threadIdx.x < DQ_CW / 2) {
+    cs_s[threadIdx.x] = rope ? rope_cos_sin_theta(L, freqs.theta[c0 / 2 + threadIdx.x]) : make_float2(1.f, 0.f);
+  }
+  pdl_enter();
   // split-K sums: all of qt, this CTA's 32 key coordinates, and the value coordinates c with
   // (c / 32) % gridDim.y == blockIdx.y
   const float* prow = part + (long)b * ncol;
@@ -510,10 +517,6 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     const bf16 vv = __float2bfloat16_rn(acc);
     vnew[(long)b * t3 + c] = vv;
     if (append && !shared_kv) Vc[((long)b * Lmax + L) * t3 + c] = vv;   // shared cache: the key row written below is the value row
-  }
-  for (int i = threadIdx.x; i < nH * r1; i += blockDim.x) u1_s[i] = __bfloat162float(U1[i]);
-  if (threadIdx.x < DQ_CW / 2) {
-    cs_s[threadIdx.x] = rope ? rope_cos_sin_theta(L, freqs.theta[c0 / 2 + threadIdx.x]) : make_float2(1.f, 0.f);
   }
   __syncthreads();
   if (threadIdx.x < DQ_CW / 2) {                    // new key, rotated
@@ -602,7 +605,6 @@ __global__ void __launch_bounds__(256)
 k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ cache_len,
           int B, int Lmax, int nH, int t1, int t2, int t3, int grid_attn, const bf16* __restrict__ Ct,
           const bf16* __restrict__ Ut1, bf16* __restrict__ z) {
-  pdl_enter();
   extern __shared__ __align__(16) float do_smem[];
   float* o_s = do_smem;                    // [32][t3]
   float* w_s = o_s + 32 * t3;              // [MAX_GRID][32]
@@ -649,6 +651,9 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
     on_s[k] = cta_first_tile(i, total, grid_attn) != cta_first_tile(i + 1, total, grid_attn);
   }
   __syncthreads();
+  // Up to here only inputs of the call were read (cache_len, Ut1, the prefetch of the output core), while
+  // the attention kernel before this one finishes; its partials are read after pdl_enter().
+  pdl_enter();
   if (threadIdx.x < 32) {
     // log-sum-exp over the partials of head h; four (max, sum) pairs are loaded at a time
     const int h = threadIdx.x;
