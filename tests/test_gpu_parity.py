@@ -410,8 +410,10 @@ def test_sharp_softmax_variant():
     check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2", scaled=True)
 
 
-def test_full_size_decode_sampled():
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
+def test_full_size_decode_sampled(flags):
     # benchmark decode workload: 64 sequences, 32768 cached latent rows each, RoPE at position 32768
+    # (with both forms of the cache-streaming kernel, each in the launch configuration bench.py times)
     import torch
     w = W.get_workload("c5")
     L, Lmax, B = w.N, w.N + 1, w.B
@@ -427,7 +429,7 @@ def test_full_size_decode_sampled():
         Kd[b, :lens[b]] = torch.from_numpy(k).to(torch.bfloat16).cuda()
         Vd[b, :lens[b]] = torch.from_numpy(v).to(torch.bfloat16).cuda()
     y = Bd.tucker_attn_decode(H.to_device(x, w.dtype), *dw, Kd, Vd, torch.from_numpy(lens).cuda(), n_H=w.n_H,
-                              rope=True, rope_base=w.rope_base, append=True)
+                              rope=True, rope_base=w.rope_base, append=True, flags=flags)
     assert Bd.last_device_error() == 0
     y = y.float().cpu().numpy().astype(np.float64)
     sample = [0, 5, 40, 63]
