@@ -76,39 +76,91 @@ struct PrepParams {
   int g1, g2, g3;
 };
 
-// out[h*sh + b*sb + c*sc] = bf16(mult * sum_a U1[h,a] C[a,b,c]).  The flat loop index walks the OUTPUT in
-// memory order (the index with unit stride innermost), so the stores are coalesced; the reads of the
-// small core tensor are strided instead and served by the caches.
-__device__ __forceinline__ void head_core_part(const bf16* __restrict__ C, const bf16* __restrict__ U1,
-                                               bf16* __restrict__ out, int nH, int r1, int rb, int rc, long sh, long sb,
-                                               long sc, float mult, int block, int nblocks) {
-  const long total = (long)nH * rb * rc;
-  const bool b_inner = (sb == 1);         // which of b / c is contiguous in the output
-  const int n_in = b_inner ? rb : rc, n_out = b_inner ? rc : rb;
-  for (long i = block * (long)blockDim.x + threadIdx.x; i < total; i += (long)nblocks * blockDim.x) {
-    const int x_in = (int)(i % n_in);
-    const int x_out = (int)((i / n_in) % n_out);
-    const int h = (int)(i / ((long)n_in * n_out));
-    const int b = b_inner ? x_in : x_out, c = b_inner ? x_out : x_in;
-    float acc = 0.f;
-    for (int a = 0; a < r1; ++a)
-      acc = fmaf(__bfloat162float(U1[(long)h * r1 + a]), __bfloat162float(C[((long)a * rb + b) * rc + c]), acc);
-    out[h * sh + b * sb + c * sc] = __float2bfloat16_rn(acc * mult);
+constexpr int PREP_THREADS = 128;
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+    f[2 * e] = t.x; f[2 * e + 1] = t.y;
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  return make_uint4(sm100::pack_bf16(f[0], f[1]), sm100::pack_bf16(f[2], f[3]), sm100::pack_bf16(f[4], f[5]),
+                    sm100::pack_bf16(f[6], f[7]));
+}
+
+// acc[0..8) = sum_a u[a] * C[a, row, c0 .. c0 + 8): 16-byte loads along the contiguous index of the core,
+// four slices requested before the first is used.
+__device__ __forceinline__ void head_core_8(const bf16* __restrict__ Cbase, long slice_stride, const bf16* __restrict__ u,
+                                            int r1, float (&acc)[8]) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  for (int a0 = 0; a0 < r1; a0 += 4) {
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      v[k] = (a0 + k < r1) ? *reinterpret_cast<const uint4*>(Cbase + (long)(a0 + k) * slice_stride) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (a0 + k < r1) {
+        const float ua = __bfloat162float(u[a0 + k]);
+        float f[8];
+        unpack8(v[k], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(ua, f[e], acc[e]);
+      }
+    }
   }
 }
 
-__global__ void __launch_bounds__(256) k_prefill_prep(const PrepParams p) {
+__global__ void __launch_bounds__(PREP_THREADS) k_prefill_prep(const PrepParams p) {
   pdl_enter();
-  const int blk = blockIdx.x;
+  __shared__ __align__(16) bf16 tile[32][40];     // [c][b], rows padded to 80 bytes (16-byte aligned, conflict-poor)
+  const int blk = blockIdx.x, t = threadIdx.x;
   if (blk < p.g1) {
-    head_core_part(p.C, p.U1, p.GcatT, p.nH, p.r1, p.r2, p.r3, (long)p.r3 * p.r2, 1, p.r2, p.mult, blk, p.g1);
+    // G^T tile: head h, 32 query coordinates b x 32 key coordinates c.  Read along c (contiguous in the
+    // core), transpose through shared memory, write along b (contiguous in GcatT[h, c, b]).
+    const int tc = p.r3 / 32, tb = p.r2 / 32;
+    const int h = blk / (tb * tc), b0 = ((blk / tc) % tb) * 32, c0 = (blk % tc) * 32;
+    {
+      const int bl = t / 4, cc = (t % 4) * 8;
+      float acc[8];
+      head_core_8(p.C + ((long)(b0 + bl) * p.r3 + c0 + cc), (long)p.r2 * p.r3, p.U1 + (long)h * p.r1, p.r1, acc);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) tile[cc + e][bl] = __float2bfloat16_rn(acc[e] * p.mult);
+    }
+    __syncthreads();
+    {
+      const int cl = t / 4, bb = (t % 4) * 8;
+      *reinterpret_cast<uint4*>(p.GcatT + ((long)h * p.r3 + c0 + cl) * p.r2 + b0 + bb) =
+          *reinterpret_cast<const uint4*>(&tile[cl][bb]);
+    }
   } else if (blk < p.g1 + p.g2) {
-    head_core_part(p.Ct, p.Ut1, p.GtP, p.nH, p.t1, p.t2, p.t3, p.t3, (long)p.nH * p.t3, 1, 1.f, blk - p.g1, p.g2);
+    // GtP[j, h, c .. c + 8): the value coordinate c is contiguous in the core and in the output
+    const long i = (long)(blk - p.g1) * PREP_THREADS + t;
+    const int cch = p.t3 / 8;
+    const long total = (long)p.t2 * p.nH * cch;
+    if (i < total) {
+      const int c8 = (int)(i % cch) * 8, h = (int)((i / cch) % p.nH), j = (int)(i / ((long)cch * p.nH));
+      float acc[8];
+      head_core_8(p.Ct + ((long)j * p.t3 + c8), (long)p.t2 * p.t3, p.Ut1 + (long)h * p.t1, p.t1, acc);
+      *reinterpret_cast<uint4*>(p.GtP + ((long)j * p.nH + h) * p.t3 + c8) = pack8(acc);
+    }
   } else {
-    const int half = p.r3 / 2;
-    const long total = (long)p.n_pos * half;
-    for (long i = (blk - p.g1 - p.g2) * (long)blockDim.x + threadIdx.x; i < total; i += (long)p.g3 * blockDim.x)
-      p.rope[i] = dec::rope_cos_sin_theta(p.pos0 + (int)(i / half), p.freqs.theta[i % half]);
+    // (cos, sin) table: four consecutive pairs of one position per thread, two 16-byte stores
+    const int half = p.r3 / 2;                      // a multiple of 16
+    const long i4 = ((long)(blk - p.g1 - p.g2) * PREP_THREADS + t) * 4;
+    if (i4 < (long)p.n_pos * half) {
+      const int pos = p.pos0 + (int)(i4 / half), i0 = (int)(i4 % half);
+      float2 cs[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) cs[e] = dec::rope_cos_sin_theta(pos, p.freqs.theta[i0 + e]);
+      float4* dst = reinterpret_cast<float4*>(p.rope + i4);
+      dst[0] = make_float4(cs[0].x, cs[0].y, cs[1].x, cs[1].y);
+      dst[1] = make_float4(cs[2].x, cs[2].y, cs[3].x, cs[3].y);
+    }
   }
 }
 
@@ -119,12 +171,6 @@ dec::RopeFreqs rope_freqs(const tucker_attn_desc& d) {
   for (int i = 0; i < 128; ++i)
     f.theta[i] = (d.rope && i < half) ? pow((double)d.rope_base, -2.0 * (double)i / (double)d.r3) : 0.0;
   return f;
-}
-
-int grid_for(long total, int block = 256) {
-  long g = (total + block - 1) / block;
-  if (g > 148L * 8) g = 148L * 8;
-  return (int)(g < 1 ? 1 : g);
 }
 
 bool umma_attention_ok(const tucker_attn_desc& d) { return d.r3 <= 128 && d.t3 <= 128; }
@@ -330,10 +376,11 @@ int fast_fwd(Problem& p) {
     pp.n_pos = d.N; pp.pos0 = d.pos0;
     pp.mult = tc_attn ? p.scale * LOG2E : p.scale;
     pp.freqs = rope_freqs(d);
-    pp.g1 = grid_for((long)d.n_H * d.r2 * d.r3);
-    pp.g2 = grid_for((long)d.n_H * d.t2 * d.t3);
-    pp.g3 = d.rope ? grid_for((long)d.N * (d.r3 / 2)) : 0;
-    (void)launch_pdl(k_prefill_prep, dim3(pp.g1 + pp.g2 + pp.g3), dim3(256), 0, p.stream, pp);
+    // one block per 32 x 32 tile of every G_h^T, one thread per 8 outputs of Gt / 4 entries of the table
+    pp.g1 = d.n_H * (d.r2 / 32) * (d.r3 / 32);
+    pp.g2 = (int)(((long)d.n_H * d.t2 * (d.t3 / 8) + PREP_THREADS - 1) / PREP_THREADS);
+    pp.g3 = d.rope ? (int)(((long)d.N * (d.r3 / 2) / 4 + PREP_THREADS - 1) / PREP_THREADS) : 0;
+    (void)launch_pdl(k_prefill_prep, dim3(pp.g1 + pp.g2 + pp.g3), dim3(PREP_THREADS), 0, p.stream, pp);
     TA_LAUNCH_CHECK(p);
   }
 
