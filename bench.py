@@ -403,6 +403,35 @@ def _cfg(w):
 
 # ----------------------------------------------------------------------------------------
 
+def bench_pack(torch, Bd, peaks, steps=10):
+    """Next row f-3: MHA weights of the c2 layer (d = 768, 12 heads) packed as Tucker-attention weights.
+    Bytes that must move: the four [d, d] inputs read, the eight outputs written."""
+    d, n_H = 768, 12
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1100)
+    Ws = [torch.randn(d, d, device="cuda", dtype=torch.bfloat16, generator=g) for _ in range(4)]
+    outs = Bd.tucker_pack_mha(*Ws, n_H=n_H)
+    nbytes = sum(t.numel() * t.element_size() for t in Ws) + sum(t.numel() * t.element_size() for t in outs)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for i in range(steps + 3):
+        flush.fill_(i & 1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        Bd.tucker_pack_mha(*Ws, n_H=n_H, out=outs)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            times.append(e0.elapsed_time(e1))
+    ms = sum(times) / len(times)
+    ach = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": "f3_pack_mha_gpt2", "unit": "GB/s", "value": ach, "ms_per_step": ms, "bytes_per_step": nbytes,
+            "gpu_launches_per_step": 7, "l2": "flushed between steps",
+            "roofline": {"kernel": "weight packers (selector core, copies, transpose)", "bound": "hbm", "achieved": ach,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                         "kernel_ms": ms, "whole_step_frac_of_peak": ach / peaks["hbm_gbs"]}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -466,6 +495,8 @@ def main():
             o = ofn(ow, max(5, min(args.steps, 20)), 3, torch, Bd, barrier, peaks, with_e2e=False)
             o.pop("clocks", None)
             others.append(o)
+        torch.cuda.empty_cache()
+        others.append(bench_pack(torch, Bd, peaks))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

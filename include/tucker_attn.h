@@ -176,6 +176,48 @@ TA_API int tucker_attn_decode_static(const tucker_attn_desc* desc, const void* x
                               const int32_t* cache_len, int32_t append,
                               void* y, void* cuda_stream);
 
+/*
+ * Weight packers: the paper's special cases as Tucker attention (Sec. 2.2; Lemma 1 and
+ * Theorems 1-3 and their proofs).  They write the two cores and six factors that
+ * tucker_attn_fwd / tucker_attn_decode take, so that MHA, GQA / MQA and MLA weights run
+ * through the same kernels.  All pointers are caller-owned device memory, row-major, of the
+ * storage type `dtype` (inputs and outputs alike); asynchronous on `cuda_stream`; no
+ * workspace.  d_H = d_model / n_H (d_model must be a multiple of n_H).  Returns TA_OK,
+ * TA_ERR_INVALID_ARG (null pointer, bad sizes or dtype) or TA_ERR_CUDA.
+ *
+ * tucker_pack_gqa: n_H query heads, n_G <= n_H key / value heads, head i using group
+ * floor(i n_G / n_H) (n_G = 1 is MQA).  Inputs WQ [d, d], WKg [d, n_G d_H], WVg [d, n_G d_H]
+ * (heads are column blocks of width d_H), WO [d, d] (head i = rows i d_H ..).  Outputs,
+ * ranks (n_H, d, n_G d_H) for both tensors:
+ *   C, Ct [n_H, d, n_G d_H] selector cores, U1, Ut1 [n_H, n_H] = I, U2 [d, d] = WQ,
+ *   U3 [d, n_G d_H] = WKg, Ut2 [d, d] = WO^T, Ut3 [d, n_G d_H] = WVg.
+ * tucker_pack_mha: the same with n_G = n_H (WK, WV [d, d]).
+ * The result equals sum_i softmax(X WQ_i (X WK_g(i))^T / sqrt(d_H)) X WV_g(i) WO_i exactly
+ * (Eq. 1); with rope = 1 the latent RoPE acts on the n_G d_H key coordinates as one
+ * rotation over the whole width, which is NOT the per-head RoPE of a trained MHA / GQA model
+ * unless n_G = 1 (the MQA case of App. C.2).
+ *
+ * tucker_pack_mla: MLA without RoPE.  Inputs WDQ [d, dcq], WUQ [dcq, d], WDKV [d, dck],
+ * WUK [dck, d], WDV [d, dck] (pass WDKV again for a shared latent), WUV [dck, d], WO [d, d];
+ * the up-projections are column-split into heads.  Outputs, ranks (n_H, dcq, dck) and
+ * (n_H, d, dck): C [n_H, dcq, dck] with C[i] = WUQ_i WUK_i^T, Ct [n_H, d, dck] with
+ * Ct[i, o, c] = (WUV_i WO_i)[c, o], U1, Ut1 [n_H, n_H] = I, U2 [d, dcq] = WDQ,
+ * U3 [d, dck] = WDKV, Ut2 [d, d] = I, Ut3 [d, dck] = WDV.
+ */
+TA_API int tucker_pack_gqa(int32_t d_model, int32_t n_H, int32_t n_G, int32_t dtype,
+                    const void* WQ, const void* WKg, const void* WVg, const void* WO,
+                    void* C, void* U1, void* U2, void* U3, void* Ct, void* Ut1, void* Ut2, void* Ut3,
+                    void* cuda_stream);
+TA_API int tucker_pack_mha(int32_t d_model, int32_t n_H, int32_t dtype,
+                    const void* WQ, const void* WK, const void* WV, const void* WO,
+                    void* C, void* U1, void* U2, void* U3, void* Ct, void* Ut1, void* Ut2, void* Ut3,
+                    void* cuda_stream);
+TA_API int tucker_pack_mla(int32_t d_model, int32_t n_H, int32_t dcq, int32_t dck, int32_t dtype,
+                    const void* WDQ, const void* WUQ, const void* WDKV, const void* WUK,
+                    const void* WDV, const void* WUV, const void* WO,
+                    void* C, void* U1, void* U2, void* U3, void* Ct, void* Ut1, void* Ut2, void* Ut3,
+                    void* cuda_stream);
+
 /* Human-readable name of a status code (static storage). */
 TA_API const char* tucker_attn_status_string(int status);
 

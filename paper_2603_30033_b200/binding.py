@@ -81,6 +81,12 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_attn_last_launch_count.restype = ctypes.c_int
     lib.tucker_attn_set_profile_events.restype = ctypes.c_int
     lib.tucker_attn_set_profile_events.argtypes = [vp, vp]
+    lib.tucker_pack_gqa.restype = ctypes.c_int
+    lib.tucker_pack_gqa.argtypes = [i32] * 4 + [vp] * 13
+    lib.tucker_pack_mha.restype = ctypes.c_int
+    lib.tucker_pack_mha.argtypes = [i32] * 3 + [vp] * 13
+    lib.tucker_pack_mla.restype = ctypes.c_int
+    lib.tucker_pack_mla.argtypes = [i32] * 5 + [vp] * 16
     _lib = lib
     return lib
 
@@ -267,6 +273,90 @@ def tucker_attn_decode_static(x, C, U1, U2, U3, Ct, Ut1, Ut2, Ut3, Kcache, Vcach
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_attn_decode_static")
     return out
+
+
+_PACK_KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
+
+
+def _pack_outputs(shapes, like, out=None):
+    torch = _torch()
+    if out is None:
+        return [torch.empty(sh, dtype=like.dtype, device=like.device) for sh in shapes]
+    if len(out) != len(shapes):
+        raise ValueError(f"out must hold {len(shapes)} tensors (C, U1, U2, U3, Ct, Ut1, Ut2, Ut3)")
+    for name, t, sh in zip(_PACK_KEYS, out, shapes):
+        _check(t, name, sh, like.dtype, like.device)
+    return list(out)
+
+
+def tucker_pack_gqa(WQ, WKg, WVg, WO, *, n_H: int, n_G: int, out=None):
+    """GQA / MQA (n_G = n_H: MHA) weights as Tucker-attention weights; returns the list
+    [C, U1, U2, U3, Ct, Ut1, Ut2, Ut3] of new device tensors (ranks (n_H, d, n_G d_H))."""
+    torch = _torch()
+    lib = load_library()
+    d = WQ.shape[0]
+    dev, dt = WQ.device, WQ.dtype
+    if d % n_H or not (1 <= n_G <= n_H):
+        raise ValueError("d_model must be a multiple of n_H and 1 <= n_G <= n_H")
+    w = n_G * (d // n_H)
+    _check(WQ, "WQ", (d, d), dt, dev)
+    _check(WKg, "WKg", (d, w), dt, dev)
+    _check(WVg, "WVg", (d, w), dt, dev)
+    _check(WO, "WO", (d, d), dt, dev)
+    outs = _pack_outputs([(n_H, d, w), (n_H, n_H), (d, d), (d, w), (n_H, d, w), (n_H, n_H), (d, d), (d, w)], WQ, out)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_pack_gqa(int(d), int(n_H), int(n_G), _dtype_code(WQ), WQ.data_ptr(), WKg.data_ptr(),
+                                 WVg.data_ptr(), WO.data_ptr(), *[o.data_ptr() for o in outs], _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_pack_gqa")
+    return outs
+
+
+def tucker_pack_mha(WQ, WK, WV, WO, *, n_H: int, out=None):
+    """MHA weights as Tucker-attention weights (ranks (n_H, d, d)); see tucker_pack_gqa."""
+    torch = _torch()
+    lib = load_library()
+    d = WQ.shape[0]
+    dev, dt = WQ.device, WQ.dtype
+    if d % n_H:
+        raise ValueError("d_model must be a multiple of n_H")
+    for name, t in (("WQ", WQ), ("WK", WK), ("WV", WV), ("WO", WO)):
+        _check(t, name, (d, d), dt, dev)
+    outs = _pack_outputs([(n_H, d, d), (n_H, n_H), (d, d), (d, d), (n_H, d, d), (n_H, n_H), (d, d), (d, d)], WQ, out)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_pack_mha(int(d), int(n_H), _dtype_code(WQ), WQ.data_ptr(), WK.data_ptr(), WV.data_ptr(),
+                                 WO.data_ptr(), *[o.data_ptr() for o in outs], _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_pack_mha")
+    return outs
+
+
+def tucker_pack_mla(WDQ, WUQ, WDKV, WUK, WDV, WUV, WO, *, n_H: int, out=None):
+    """MLA (no RoPE) weights as Tucker-attention weights (ranks (n_H, dcq, dck) and
+    (n_H, d, dck)); pass WDKV as WDV for a shared key / value latent."""
+    torch = _torch()
+    lib = load_library()
+    d, dcq = WDQ.shape
+    dck = WDKV.shape[1]
+    dev, dt = WDQ.device, WDQ.dtype
+    if d % n_H:
+        raise ValueError("d_model must be a multiple of n_H")
+    _check(WDQ, "WDQ", (d, dcq), dt, dev)
+    _check(WUQ, "WUQ", (dcq, d), dt, dev)
+    _check(WDKV, "WDKV", (d, dck), dt, dev)
+    _check(WUK, "WUK", (dck, d), dt, dev)
+    _check(WDV, "WDV", (d, dck), dt, dev)
+    _check(WUV, "WUV", (dck, d), dt, dev)
+    _check(WO, "WO", (d, d), dt, dev)
+    outs = _pack_outputs([(n_H, dcq, dck), (n_H, n_H), (d, dcq), (d, dck), (n_H, d, dck), (n_H, n_H), (d, d), (d, dck)],
+                         WDQ, out)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_pack_mla(int(d), int(n_H), int(dcq), int(dck), _dtype_code(WDQ), WDQ.data_ptr(), WUQ.data_ptr(),
+                                 WDKV.data_ptr(), WUK.data_ptr(), WDV.data_ptr(), WUV.data_ptr(), WO.data_ptr(),
+                                 *[o.data_ptr() for o in outs], _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_pack_mla")
+    return outs
 
 
 def last_device_error(device=None) -> int:
