@@ -6,7 +6,8 @@
 // a K-major, 128-byte-swizzled UMMA A operand; phase 2 walks the d / 128 column chunks of Y with two
 // TMEM accumulators, so that the conversion + coalesced store of one chunk overlaps the MMAs of the
 // next.  One TMA ring (uniform stage size) serves both phases, the producer runs ahead across the
-// phase boundary.
+// phase boundary.  The Z tile and the staging tile are idle until phase 1 has ended, so phase 1 uses
+// them as two more ring stages: its O tiles come from HBM, and the bytes in flight per SM set its pace.
 //   warp 0      TMA producer        warp 1   TMEM allocation + MMA issue        warps 2..5  epilogue
 #pragma once
 
@@ -22,8 +23,10 @@ constexpr int THREADS = 192;
 constexpr int BN2 = 128;                         // columns of Y per chunk
 constexpr int SUB_BYTES = 128 * 64 * 2;          // one [128 x 64] bf16 sub-tile
 constexpr int MAX_STAGES = 4;
+constexpr int EXTRA_STAGES = 2;                  // phase 1 only: the Z tile and the staging tile
 constexpr int STAGE_BYTES = 2 * SUB_BYTES;       // phase 1: O tile (16 KB) + G~ tile (<= 16 KB); phase 2: U~2 chunk (<= 32 KB)
 constexpr int STAGING_PITCH = (BN2 + 8) * 2;     // bytes per staged output row
+static_assert(128 * STAGING_PITCH >= STAGE_BYTES, "the staging tile doubles as a ring stage");
 // ring | Z tile (two sub-tiles) | staging tile
 __host__ __device__ constexpr size_t smem_bytes(int stages) {
   return 1024 + (size_t)stages * STAGE_BYTES + 2 * SUB_BYTES + (size_t)128 * STAGING_PITCH;
@@ -43,15 +46,17 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmU, const Params p) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], z_full, z_ready, acc_full[2], acc_empty[2];
+  __shared__ uint64_t full_bar[MAX_STAGES + EXTRA_STAGES], empty_bar[MAX_STAGES + EXTRA_STAGES];
+  __shared__ uint64_t z_full, z_ready, acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* ring = smem_raw + (base - smem_u32(smem_raw));
   const int S = p.stages;
-  uint8_t* z_tile = ring + (size_t)S * STAGE_BYTES;
-  uint8_t* staging = z_tile + 2 * SUB_BYTES;
+  uint8_t* z_tile = ring + (size_t)S * STAGE_BYTES;        // = ring stage S during phase 1
+  uint8_t* staging = z_tile + 2 * SUB_BYTES;               // = ring stage S + 1 during phase 1
+  const int S1 = S + EXTRA_STAGES;                         // ring depth of phase 1
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int m0 = blockIdx.x * 128;
@@ -59,10 +64,12 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
   const int nsub2 = (p.t2 + 63) / 64;       // 64-wide K sub-tiles of phase 2
   const int nchunk = p.d / BN2;
   Abort ab{&abort_flag, p.err};
+  // use count of ring stage s < S at the end of phase 1 (phase 2 continues each stage's barrier phases)
+  auto uses1 = [&](int s) { return nkb1 > s ? (nkb1 - s + S1 - 1) / S1 : 0; };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < MAX_STAGES; ++s) {
+    for (int s = 0; s < MAX_STAGES + EXTRA_STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
@@ -88,18 +95,17 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
   if (warp == 0) {
     if (elect_one()) {
       tma_prefetch_desc(&tmO); tma_prefetch_desc(&tmG); tma_prefetch_desc(&tmU);
-      int it = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
-        const int s = it % S;
-        if (!(ok = mbar_wait(&empty_bar[s], ((it / S) & 1) ^ 1, ab))) break;
+      for (int kb = 0; kb < nkb1 && ok; ++kb) {
+        const int s = kb % S1;
+        if (!(ok = mbar_wait(&empty_bar[s], ((kb / S1) & 1) ^ 1, ab))) break;
         mbar_expect_tx(&full_bar[s], (uint32_t)(SUB_BYTES + p.t2 * 128));
         tma_load_2d(ring + s * STAGE_BYTES, &tmO, &full_bar[s], kb * 64, m0);
         tma_load_2d(ring + s * STAGE_BYTES + SUB_BYTES, &tmG, &full_bar[s], kb * 64, 0);
       }
-      for (int n = 0; n < nchunk && ok; ++n, ++it) {
-        const int s = it % S;
-        if (!(ok = mbar_wait(&empty_bar[s], ((it / S) & 1) ^ 1, ab))) break;
+      for (int n = 0; n < nchunk && ok; ++n) {
+        const int s = n % S;
+        if (!(ok = mbar_wait(&empty_bar[s], ((uses1(s) + n / S) & 1) ^ 1, ab))) break;
         mbar_expect_tx(&full_bar[s], (uint32_t)(nsub2 * SUB_BYTES));
         for (int kk = 0; kk < nsub2; ++kk)
           tma_load_2d(ring + s * STAGE_BYTES + kk * SUB_BYTES, &tmU, &full_bar[s], kk * 64, n * BN2);
@@ -109,12 +115,11 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
     if (elect_one()) {
       const uint32_t idesc1 = umma_idesc_bf16(128, (uint32_t)p.t2);
       const uint32_t idesc2 = umma_idesc_bf16(128, BN2);
-      int it = 0;
       bool ok = true;
       // ---- phase 1: Z = O Gt^T ----
-      for (int kb = 0; kb < nkb1 && ok; ++kb, ++it) {
-        const int s = it % S;
-        if (!(ok = mbar_wait(&full_bar[s], (it / S) & 1, ab))) break;
+      for (int kb = 0; kb < nkb1 && ok; ++kb) {
+        const int s = kb % S1;
+        if (!(ok = mbar_wait(&full_bar[s], (kb / S1) & 1, ab))) break;
         tc_fence_after();
         const uint32_t a_addr = smem_u32(ring + s * STAGE_BYTES), b_addr = a_addr + SUB_BYTES;
         const int nks = min(4, (p.K1 - kb * 64) / 16);
@@ -127,10 +132,10 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
       // ---- phase 2: Y chunks = Z Ut2^T ----
       if (ok) ok = mbar_wait(&z_ready, 0, ab);     // the bf16 Z tile is in shared memory
       const uint32_t z_addr = smem_u32(z_tile);
-      for (int n = 0; n < nchunk && ok; ++n, ++it) {
-        const int s = it % S, buf = n & 1;
+      for (int n = 0; n < nchunk && ok; ++n) {
+        const int s = n % S, buf = n & 1;
         if (!(ok = mbar_wait(&acc_empty[buf], ((n >> 1) & 1) ^ 1, ab))) break;
-        if (!(ok = mbar_wait(&full_bar[s], (it / S) & 1, ab))) break;
+        if (!(ok = mbar_wait(&full_bar[s], (uses1(s) + n / S) & 1, ab))) break;
         tc_fence_after();
         const uint32_t b_addr = smem_u32(ring + s * STAGE_BYTES);
         for (int ks = 0; ks < p.t2 / 16; ++ks) {
