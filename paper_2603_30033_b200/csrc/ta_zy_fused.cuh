@@ -8,7 +8,9 @@
 // next.  One TMA ring (uniform stage size) serves both phases, the producer runs ahead across the
 // phase boundary.  The Z tile and the staging tile are idle until phase 1 has ended, so phase 1 uses
 // them as two more ring stages: its O tiles come from HBM, and the bytes in flight per SM set its pace.
-//   warp 0      TMA producer        warp 1   TMEM allocation + MMA issue        warps 2..5  epilogue
+//   warp 0      TMA producer        warp 1   TMEM allocation + MMA issue        warps 2..9  epilogue
+// (two epilogue warps per TMEM lane quadrant, one per half of a tile's columns: the conversion and store
+// of a chunk is a latency chain per thread, and it, not the tensor core, paces phase 2)
 #pragma once
 
 #include "ta_common.cuh"
@@ -19,7 +21,7 @@ namespace zy {
 
 using namespace sm100;
 
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;
 constexpr int BN2 = 128;                         // columns of Y per chunk
 constexpr int SUB_BYTES = 128 * 64 * 2;          // one [128 x 64] bf16 sub-tile
 constexpr int MAX_STAGES = 4;
@@ -74,10 +76,10 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
       mbar_init(&empty_bar[s], 1);
     }
     mbar_init(&z_full, 1);
-    mbar_init(&z_ready, 4);          // one arrival per epilogue warp
+    mbar_init(&z_ready, 8);          // one arrival per epilogue warp
     for (int u = 0; u < 2; ++u) {
       mbar_init(&acc_full[u], 1);
-      mbar_init(&acc_empty[u], 4);
+      mbar_init(&acc_empty[u], 8);
     }
     fence_barrier_init();
   }
@@ -147,8 +149,9 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
       }
     }
   } else {
-    // epilogue warps: warp w owns TMEM lanes / tile rows [32 (w % 4), 32 (w % 4) + 32)
-    const int q = warp % 4;
+    // epilogue warps: warp w owns TMEM lanes / tile rows [32 (w % 4), 32 (w % 4) + 32) and the column
+    // half hf = (w - 2) / 4 of every tile
+    const int q = warp % 4, hf = (warp - 2) >> 2;
     const int rloc = q * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     bool ok = mbar_wait(&z_full, 0, ab);
@@ -156,7 +159,7 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
     if (ok) {
       tc_fence_after();
       // Z row -> bf16 -> K-major swizzled A tile
-      for (int ch = 0; ch < p.t2 / 32; ++ch) {
+      for (int ch = hf; ch < p.t2 / 32; ch += 2) {
         uint32_t r[32];
         tmem_ld32(tm_z + lane_addr + ch * 32, r);
         tmem_ld_wait();
@@ -181,7 +184,7 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        for (int ch = 0; ch < BN2 / 32; ++ch) {
+        for (int ch = 2 * hf; ch < 2 * hf + 2; ++ch) {
           uint32_t r[32];
           tmem_ld32(tm_y(buf) + lane_addr + ch * 32, r);
           tmem_ld_wait();
@@ -196,9 +199,9 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[buf]);   // the MMA warp may overwrite this accumulator now
-        // the warp writes its 32 rows: 16 lanes x 16 bytes per row, two rows per pass
-        const int rsub = lane / 16, cc = lane % 16;
-        for (int r0 = 0; r0 < 32; r0 += 2) {
+        // the warp writes its half (128 bytes) of its 32 rows: 8 lanes x 16 bytes per row, four rows per pass
+        const int rsub = lane / 8, cc = hf * 8 + lane % 8;
+        for (int r0 = 0; r0 < 32; r0 += 4) {
           const int rr = q * 32 + r0 + rsub;
           const int grow = m0 + rr;
           if (grow < p.M) {
