@@ -21,7 +21,7 @@ using namespace sm100;
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int MAX_STAGES = 4;
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;   // producer warp, MMA warp, eight epilogue warps
 constexpr int MAX_BN = 256;
 // Dynamic shared memory of one CTA: the ring is sized for the stage count and tile width of
 // the launch, so that short-K problems (one or two K blocks) leave room for several CTAs
@@ -203,9 +203,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     if (p.early) pdl_enter();
   } else {
-    // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32)
+    // epilogue: warp w owns TMEM lanes [32*(w%4), 32*(w%4)+32) and every second 32-column chunk of the
+    // tile (two warps per lane quadrant: the conversion / store chain per thread is what takes the time)
     if (p.early) pdl_enter();
-    const int q = warp % 4;
+    const int q = warp % 4, hf = (warp - 2) >> 2;
     const int row = m0 + q * 32 + lane;
     const bool ok = mbar_wait(&acc_bar, 0, ab);
     tc_fence_after();
@@ -216,7 +217,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int rloc = q * 32 + lane;
       const int npos = p.n_pos > 0 ? row % p.n_pos : row;
       if (sg.mode == EP_F32) {
-        for (int ch = 0; ch < p.BN / 32; ++ch) {
+        for (int ch = hf; ch < p.BN / 32; ch += 2) {
           uint32_t r[32];
           tmem_ld32(acc + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
@@ -231,11 +232,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       } else {
         // bf16 outputs: every thread converts its own accumulator row into a staging tile in shared
         // memory (the ring is idle once the accumulator is complete; rows padded by 16 bytes keep the
-        // 16-byte stores of a quarter-warp on distinct banks), then each warp writes its 32 rows out
-        // with full-row, coalesced 16-byte stores.
+        // 16-byte stores of a quarter-warp on distinct banks), then each warp writes the 64-byte row
+        // segments of its chunks out, eight rows per 16-byte store instruction.
         const int pitch = (p.BN + 8) * 2;
         uint8_t* stage = tiles;
-        for (int ch = 0; ch < p.BN / 32; ++ch) {
+        for (int ch = hf; ch < p.BN / 32; ch += 2) {
           uint32_t r[32];
           tmem_ld32(acc + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
@@ -261,19 +262,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int i = 0; i < 4; ++i) sdst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
         }
         __syncwarp();
-        const int cpr = p.BN / 8;            // 16-byte chunks per row
-        const int rpi = 32 / cpr;            // rows written per warp-wide store
-        const int rsub = lane / cpr, cc = lane % cpr;
-        if (rsub < rpi) {
-          for (int r0 = 0; r0 < 32; r0 += rpi) {
+        const int rsub = lane / 4, cc = lane % 4;
+        for (int ch = hf; ch < p.BN / 32; ch += 2) {
+          for (int r0 = 0; r0 < 32; r0 += 8) {
             const int rr = q * 32 + r0 + rsub;
             const int grow = m0 + rr;
-            if (grow >= p.M) break;
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)rr * pitch + cc * 16);
-            *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + c0 + cc * 8) = v;
+            if (grow >= p.M) continue;
+            const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)rr * pitch + ch * 64 + cc * 16);
+            const int col = c0 + ch * 32 + cc * 8;
+            *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + col) = v;
             if (sg.out2) {
               const int gb = p.n_pos > 0 ? grow / p.n_pos : 0, gn = p.n_pos > 0 ? grow % p.n_pos : grow;
-              *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)gb * sg.batch2 + (long)gn * sg.ld2 + c0 + cc * 8) = v;
+              *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)gb * sg.batch2 + (long)gn * sg.ld2 + col) = v;
             }
           }
         }
