@@ -8,8 +8,8 @@
 //     U2 = W^DQ, U3 = W^DKV, C[i] = W^UQ_i (W^UK_i)^T
 //     Ut3 = W^DV (W^DKV again for a shared latent), Ut2 = I_d, Ct[i, o, c] = (W^UV_i W^O_i)[c, o]
 //
-// These run once per set of weights, not per token: plain kernels, one thread per output element
-// (or per 32 x 32 tile for the transposes and the two small per-head products).
+// These run once per set of weights, not per token: plain kernels, one thread per output element or
+// 16-byte vector (32 x 32 tiles for the transpose); the GQA / MHA packing is a single launch.
 #include "ta_common.cuh"
 
 namespace ta {
@@ -59,30 +59,6 @@ __global__ void k_transpose(const T* __restrict__ src, T* __restrict__ dst, int 
   }
 }
 
-// Selector core of Lemma 1 / Theorem 2, written to two tensors (pre- and post-softmax core are equal):
-// C[i, n, m] over [n_H, d, n_G d_H].  A thread writes 16 bytes of a row at a time when the row width allows
-// it (VEC elements; VEC = 1 otherwise); a row holds at most one 1.
-template <typename T, int VEC>
-__global__ void k_selector_core(T* __restrict__ C, T* __restrict__ Ct, int nH, int nG, int d, int dH) {
-  const long w = (long)nG * dH, wv = w / VEC, total = (long)nH * d * wv;
-  for (long idx = blockIdx.x * (long)blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
-    const int m0 = (int)(idx % wv) * VEC, n = (int)((idx / wv) % d), i = (int)(idx / (wv * d));
-    const int g = (int)(((long)i * nG) / nH);
-    const int m_one = (n / dH == i) ? g * dH + n % dH : -1;      // column of this row's 1, if the row has one
-    T v[VEC];
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) v[e] = cvt<T>(m0 + e == m_one ? 1.f : 0.f);
-    const long off = ((long)i * d + n) * w + m0;
-    if (VEC == 1) {
-      C[off] = v[0];
-      Ct[off] = v[0];
-    } else {
-      *reinterpret_cast<uint4*>(C + off) = *reinterpret_cast<const uint4*>(v);
-      *reinterpret_cast<uint4*>(Ct + off) = *reinterpret_cast<const uint4*>(v);
-    }
-  }
-}
-
 // MLA pre-softmax core: C[i, q, k] = sum_l WUQ[q, i dH + l] WUK[k, i dH + l]   (WUQ [dcq, d], WUK [dck, d])
 template <typename T>
 __global__ void k_mla_core(const T* __restrict__ WUQ, const T* __restrict__ WUK, T* __restrict__ C, int nH, int dcq,
@@ -113,6 +89,90 @@ __global__ void k_mla_core_out(const T* __restrict__ WUV, const T* __restrict__ 
   }
 }
 
+// One launch for the whole GQA / MHA packing: consecutive block ranges do the selector cores, the two
+// identities, the three copies and the transpose (this runs once per set of weights, but seven launches
+// of a few microseconds each were most of its time).
+template <typename T>
+struct GqaPack {
+  const T *WQ, *WKg, *WVg, *WO;
+  T *C, *U1, *U2, *U3, *Ct, *Ut1, *Ut2, *Ut3;
+  int nH, nG, d, dH;
+  int b_core, b_id, b_copy;      // blocks of the core part, of one identity, of one copy; then the transpose tiles
+};
+
+template <typename T, int VEC>
+__device__ __forceinline__ void selector_core_part(T* __restrict__ C, T* __restrict__ Ct, int nH, int nG, int d, int dH,
+                                                   int blk, int nblk) {
+  const long w = (long)nG * dH, wv = w / VEC, total = (long)nH * d * wv;
+  for (long idx = blk * (long)blockDim.x + threadIdx.x; idx < total; idx += (long)nblk * blockDim.x) {
+    const int m0 = (int)(idx % wv) * VEC, n = (int)((idx / wv) % d), i = (int)(idx / (wv * d));
+    const int g = (int)(((long)i * nG) / nH);
+    const int m_one = (n / dH == i) ? g * dH + n % dH : -1;
+    T v[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) v[e] = cvt<T>(m0 + e == m_one ? 1.f : 0.f);
+    const long off = ((long)i * d + n) * w + m0;
+    if (VEC == 1) {
+      C[off] = v[0];
+      Ct[off] = v[0];
+    } else {
+      *reinterpret_cast<uint4*>(C + off) = *reinterpret_cast<const uint4*>(v);
+      *reinterpret_cast<uint4*>(Ct + off) = *reinterpret_cast<const uint4*>(v);
+    }
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void copy_part(const T* __restrict__ src, T* __restrict__ dst, long n, int blk, int nblk) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const bool vec_ok = (n % VEC == 0) && ((uintptr_t)src % 16 == 0) && ((uintptr_t)dst % 16 == 0);
+  if (vec_ok) {
+    const uint4* s4 = reinterpret_cast<const uint4*>(src);
+    uint4* d4 = reinterpret_cast<uint4*>(dst);
+    for (long i = blk * (long)blockDim.x + threadIdx.x; i < n / VEC; i += (long)nblk * blockDim.x) d4[i] = s4[i];
+  } else {
+    for (long i = blk * (long)blockDim.x + threadIdx.x; i < n; i += (long)nblk * blockDim.x) dst[i] = src[i];
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void identity_part(T* __restrict__ dst, int n, int blk, int nblk) {
+  for (long i = blk * (long)blockDim.x + threadIdx.x; i < (long)n * n; i += (long)nblk * blockDim.x)
+    dst[i] = cvt<T>((i / n) == (i % n) ? 1.f : 0.f);
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) k_pack_gqa(const GqaPack<T> p) {
+  __shared__ float tile[32][33];
+  int blk = blockIdx.x;
+  const long w = (long)p.nG * p.dH;
+  if (blk < p.b_core) { selector_core_part<T, VEC>(p.C, p.Ct, p.nH, p.nG, p.d, p.dH, blk, p.b_core); return; }
+  blk -= p.b_core;
+  if (blk < 2 * p.b_id) { identity_part<T>(blk < p.b_id ? p.U1 : p.Ut1, p.nH, blk % p.b_id, p.b_id); return; }
+  blk -= 2 * p.b_id;
+  if (blk < 3 * p.b_copy) {
+    const int which = blk / p.b_copy, b = blk % p.b_copy;
+    if (which == 0) copy_part<T>(p.WQ, p.U2, (long)p.d * p.d, b, p.b_copy);
+    else if (which == 1) copy_part<T>(p.WKg, p.U3, (long)p.d * w, b, p.b_copy);
+    else copy_part<T>(p.WVg, p.Ut3, (long)p.d * w, b, p.b_copy);
+    return;
+  }
+  blk -= 3 * p.b_copy;
+  // Ut2 = WO^T: one 32 x 32 tile per block (thread (x, y) = (t % 32, t / 32), eight rows per pass)
+  const int tiles_x = (p.d + 31) / 32;
+  const int c0 = (blk % tiles_x) * 32, r0 = (blk / tiles_x) * 32;
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+  for (int k = ty; k < 32; k += 8) {
+    const int r = r0 + k, c = c0 + tx;
+    if (r < p.d && c < p.d) tile[k][tx] = ldf(p.WO + (long)r * p.d + c);
+  }
+  __syncthreads();
+  for (int k = ty; k < 32; k += 8) {
+    const int c = c0 + k, r = r0 + tx;
+    if (r < p.d && c < p.d) p.Ut2[(long)c * p.d + r] = cvt<T>(tile[tx][k]);
+  }
+}
+
 int blocks_for(long n) {
   long g = (n + 255) / 256;
   if (g > 148L * 16) g = 148L * 16;
@@ -128,14 +188,17 @@ int pack_gqa_t(int d, int nH, int nG, const void* WQ, const void* WKg, const voi
   const long w = (long)nG * dH;
   constexpr int VEC = 16 / (int)sizeof(T);
   const bool vec_ok = (w % VEC == 0) && ((uintptr_t)C % 16 == 0) && ((uintptr_t)Ct % 16 == 0);
-  if (vec_ok) k_selector_core<T, VEC><<<blocks_for((long)nH * d * w / VEC), 256, 0, st>>>((T*)C, (T*)Ct, nH, nG, d, dH);
-  else k_selector_core<T, 1><<<blocks_for((long)nH * d * w), 256, 0, st>>>((T*)C, (T*)Ct, nH, nG, d, dH);
-  k_identity<T><<<blocks_for((long)nH * nH), 256, 0, st>>>((T*)U1, nH);
-  k_identity<T><<<blocks_for((long)nH * nH), 256, 0, st>>>((T*)Ut1, nH);
-  k_copy<T><<<blocks_for((long)d * d), 256, 0, st>>>((const T*)WQ, (T*)U2, (long)d * d);
-  k_copy<T><<<blocks_for((long)d * w), 256, 0, st>>>((const T*)WKg, (T*)U3, (long)d * w);
-  k_copy<T><<<blocks_for((long)d * w), 256, 0, st>>>((const T*)WVg, (T*)Ut3, (long)d * w);
-  k_transpose<T><<<dim3((d + 31) / 32, (d + 31) / 32), dim3(32, 8), 0, st>>>((const T*)WO, (T*)Ut2, d, d);
+  GqaPack<T> p;
+  p.WQ = (const T*)WQ; p.WKg = (const T*)WKg; p.WVg = (const T*)WVg; p.WO = (const T*)WO;
+  p.C = (T*)C; p.U1 = (T*)U1; p.U2 = (T*)U2; p.U3 = (T*)U3; p.Ct = (T*)Ct; p.Ut1 = (T*)Ut1; p.Ut2 = (T*)Ut2; p.Ut3 = (T*)Ut3;
+  p.nH = nH; p.nG = nG; p.d = d; p.dH = dH;
+  p.b_core = blocks_for((long)nH * d * w / (vec_ok ? VEC : 1));
+  p.b_id = blocks_for((long)nH * nH);
+  p.b_copy = blocks_for((long)d * d / VEC);
+  const int tiles = ((d + 31) / 32) * ((d + 31) / 32);
+  const int grid = p.b_core + 2 * p.b_id + 3 * p.b_copy + tiles;
+  if (vec_ok) k_pack_gqa<T, VEC><<<grid, 256, 0, st>>>(p);
+  else k_pack_gqa<T, 1><<<grid, 256, 0, st>>>(p);
   return launch_ok() ? TA_OK : TA_ERR_CUDA;
 }
 
