@@ -5,22 +5,21 @@
 // no tensor work is spent on padding the (at most 32) heads up to a 128-row tile:
 //   S^T [128 keys x 32 heads] = K_tile [128 x r3] * Qhat^T          A = K tile as loaded (K-major), B = Qhat (K-major)
 //   O^T [t3 x 32 heads]      += V_tile^T [t3 x 128] * P [128 x 32]  A = V tile as loaded (M-major), B = P (K-major, bf16)
-// The scores of one tile sit in TMEM with one key per lane and one head per column: a softmax thread
-// owns one key and all heads.  The per-head maximum over the keys of a tile is therefore a reduction
-// ACROSS threads (a transposing butterfly of warp shuffles, then four values per head through shared
-// memory); it only moves the reference maximum of a head when that grows by more than 8 (factor 256),
-// so the accumulator in TMEM is rescaled rarely.  P goes back through shared memory (B operands are
-// read from there); the row sums stay in registers per thread and are reduced once per segment.
-//
-// Two softmax warpgroups take alternate tiles, each with its own score buffer, P buffer, output
-// accumulator and online-softmax state, so that the chain scores -> softmax -> P V of one tile overlaps
-// the next tile's; their two states are merged (log-sum-exp weights) when a segment ends, and one
-// partial per (CTA, sequence) is written exactly as the mma.sync kernel writes it.
+// The scores of one tile sit in TMEM with one key per lane and one head per column.  Two softmax
+// warpgroups work on EVERY tile, each on 16 of the 32 head columns: a thread owns one key and 16 heads.
+// The per-head maximum over the keys of a tile is a reduction ACROSS threads (a transposing butterfly of
+// warp shuffles, then four values per head through shared memory); it only moves the reference maximum
+// of a head when that grows by more than 8 (factor 256), so the accumulator in TMEM is rescaled rarely.
+// P goes back through shared memory (B operands are read from there); the row sums stay in registers
+// per thread and are reduced once per segment.  Score and P buffers are double-buffered, the output
+// accumulator is single: tile t + 1 is scored and exponentiated while P V of tile t runs, and a segment
+// ends with each warpgroup writing its 16 heads of the partial -- the same partial per (CTA, sequence)
+// that the mma.sync kernel writes.
 //
 //   warp 0       TMA producer: Qhat of the segment's sequence, K / V ring
 //   warp 1       TMEM allocation, MMA issue
-//   warps 4..7   softmax warpgroup 0 (even tiles)     warps 8..11  softmax warpgroup 1 (odd tiles)
-// TMEM columns: S_0 [0,32) S_1 [32,64) O_0 [64,96) O_1 [96,128).
+//   warps 4..7   softmax warpgroup 0 (heads 0..15)     warps 8..11  softmax warpgroup 1 (heads 16..31)
+// TMEM columns: S_0 [0,32) S_1 [32,64) O [64,96).
 // Every wait is bounded (Abort): on a timeout the CTA raises the device error word and leaves.
 #pragma once
 
@@ -45,7 +44,7 @@ constexpr int QSUB_BYTES = 32 * 64 * 2;  // [32 heads x 64] bf16 (Qhat and P sub
 constexpr int QBUF_BYTES = MAX_SUB * QSUB_BYTES;
 constexpr int PBUF_BYTES = 2 * QSUB_BYTES;             // [32 heads x 128 keys] bf16
 constexpr int RING_BYTES = 3 * STAGE_BYTES;            // three K + V stages, or six K-only stages (shared cache)
-// ring | Qhat (two segments in flight) | P_0 | P_1   (P_0 and P_1 together double as the 16 KB merge buffer)
+// ring | Qhat (two segments in flight) | P_0 | P_1
 constexpr size_t SMEM_BYTES = 1024 + (size_t)RING_BYTES + 2 * QBUF_BYTES + 2 * PBUF_BYTES;
 constexpr float kRescaleThreshold = 8.f;
 
@@ -97,11 +96,16 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * SUB_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-// v[j] of every lane -> lane j receives op over the 32 lanes of v[j] (returned in v[0]).
+// v[j] of every lane, j < 16 -> lanes j and j + 16 receive op over the 32 lanes of v[j] (returned in v[0]).
 template <bool IS_MAX>
-__device__ __forceinline__ float transpose_reduce(float (&v)[32], int lane) {
+__device__ __forceinline__ float transpose_reduce16(float (&v)[16], int lane) {
 #pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
+  for (int i = 0; i < 16; ++i) {
+    const float o = __shfl_xor_sync(0xffffffffu, v[i], 16);
+    v[i] = IS_MAX ? fmaxf(v[i], o) : v[i] + o;
+  }
+#pragma unroll
+  for (int off = 8; off >= 1; off >>= 1) {
     const bool up = (lane & off) != 0;
 #pragma unroll
     for (int i = 0; i < off; ++i) {
@@ -120,17 +124,14 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], q_full[2], q_empty[2];
-  __shared__ uint64_t s_full[2], s_free[2], p_full[2], o_full[2], o_read[2], patched[2], wg_bar[2], cta_bar;
+  __shared__ uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_read, patched, wg_bar[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  // Exchange area of the softmax warpgroups.  Per tile: the four warps' maxima per head, as bf16 (the
-  // reference maximum only has to be the same for all threads and close to the true one), double-
-  // buffered by tile parity because a warp may start its next tile while another still reads this
-  // one's.  Per segment flush: the four warps' row sums per head, fp32, in the same bytes.
-  __shared__ __align__(16) unsigned char xch_raw[2 * 4 * 32 * 4];
-  auto mxh = reinterpret_cast<__nv_bfloat16 (*)[2][4][32]>(xch_raw);   // [wg][tile parity][warp][head]
-  auto sum_s = reinterpret_cast<float (*)[4][32]>(xch_raw);            // [wg][warp][head]
-  __shared__ float m_s[2][32];         // per warpgroup: reference maximum per head (segment merge)
+  // per tile: the four warps' maxima per head of each warpgroup, as bf16 (the reference maximum only has
+  // to be the same for all threads and close to the true one), double-buffered by tile parity because a
+  // warp may start the next tile while another still reads this one's; per segment: the warps' row sums
+  __shared__ __nv_bfloat16 mxh[2][2][4][16];      // [wg][tile parity][warp][head]
+  __shared__ float sum_s[2][4][16];               // [wg][warp][head]
   __shared__ long long wtot_s[THREADS / 32];
   __shared__ int loc_b;
   __shared__ long long loc_first;
@@ -138,13 +139,10 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* ring = smem_raw + (base - smem_u32(smem_raw));
   uint8_t* qbuf = ring + (size_t)RING_BYTES;
-  // With one shared latent cache a stage holds a K tile only: twice the stages, and the scores may
-  // run two tiles ahead of the P V products instead of one.
+  uint8_t* pbuf = qbuf + 2 * QBUF_BYTES;
+  // With one shared latent cache a stage holds a K tile only: twice the stages.
   const int STAGES = p.shared_kv ? 6 : 3;
   const int stage_bytes = p.shared_kv ? MAX_SUB * SUB_BYTES : STAGE_BYTES;
-  const int ahead = p.shared_kv ? 2 : 1;
-  uint8_t* pbuf = qbuf + 2 * QBUF_BYTES;
-  float* obuf = reinterpret_cast<float*>(pbuf);       // merge buffer [32][t3] fp32 (aliases P_0 | P_1)
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   Abort ab{&abort_flag, p.err};
@@ -160,14 +158,13 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mbar_init(&q_full[i], 1);
       mbar_init(&q_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&s_free[i], 4);      // the scores of a tile are in the warpgroup's registers
-      mbar_init(&p_full[i], 4);      // one arrival per softmax warp
-      mbar_init(&o_full[i], 1);
-      mbar_init(&o_read[i], 4);
-      mbar_init(&patched[i], 4);
+      mbar_init(&s_free[i], 8);      // the scores are in registers: one arrival per softmax warp
+      mbar_init(&p_full[i], 8);      // P is in shared memory: one arrival per softmax warp
+      mbar_init(&p_free[i], 1);      // the P V product that read this P buffer is complete
       mbar_init(&wg_bar[i], 4);
     }
-    mbar_init(&cta_bar, 8);
+    mbar_init(&o_read, 8);
+    mbar_init(&patched, 4);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -178,8 +175,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_slot;
-  const uint32_t tm_s[2] = {tmem, tmem + 32};
-  const uint32_t tm_o[2] = {tmem + 64, tmem + 96};
+  const uint32_t tm_o = tmem + 64;
 
   // ---- this CTA's range of the flat tile list (same split as the mma.sync kernel) ----
   int lo, hi;
@@ -201,8 +197,6 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const long seq_first = have_work ? (long)loc_first : 0;
 
   if (warp < 4) {
-   // the producer / MMA warpgroup hands registers to the softmax warpgroups (32 scores, 32 reference
-   // maxima, 32 row sums and a 32-wide scratch per thread)
    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
    if (have_work && warp == 0) {
     // ------------------------------- TMA producer -------------------------------
@@ -235,9 +229,9 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
    } else if (have_work && warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (elect_one()) {
-      // This one thread issues 16 small MMAs per tile, so its own instruction stream is the critical
-      // resource: descriptors are formed once per operand and stepped by constants, the K loops are
-      // unrolled, and the (at most three) tiles between score issue and P V issue sit in registers.
+      // This one thread issues 16 small MMAs per tile, so its own instruction stream matters: descriptors
+      // are formed once per operand and stepped by constants, the K loops are unrolled, and the (at most
+      // two) tiles between score issue and P V issue sit in registers.
       const uint32_t idesc_qk = umma_idesc_bf16(128, 32);
       const uint32_t idesc_pv = umma_idesc_bf16(128, 32) | (1u << 15);   // A = V tile is M-major
       const int ksteps = p.r3 / 16;
@@ -246,88 +240,77 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const uint64_t dk0 = umma_desc_kmajor_sw128(smem_u32(ring));
       const uint64_t dv0 = umma_desc_mnmajor_sw128(smem_u32(ring) + (p.shared_kv ? 0u : (uint32_t)(MAX_SUB * SUB_BYTES)), SUB_BYTES);
       const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);          // descriptor address fields count 16 bytes
-      // tile state packed in one word: it << 8 | stage << 4 | first_of_wg << 1 | (seg > 0)
-      uint32_t pq0 = 0, pq1 = 0, pq2 = 0;   // pending P V products, oldest first
-      int n_pend = 0;
-      int pv_seg0 = 0, pv_seg1 = 0, pv_seg2 = 0;
+      // pending P V products, oldest first; a tile's state in one word: it << 8 | stage << 4 | first tile of its segment
+      uint32_t pq0 = 0, pq1 = 0;
+      int pv_seg0 = 0, pv_seg1 = 0, n_pend = 0;
       bool ok = true;
       auto issue_pv = [&](uint32_t code, int sg) -> bool {
-        const int it = (int)(code >> 8), st = (int)((code >> 4) & 15), wg = it & 1;
-        const bool first_of_wg = (code & 2u) != 0;
-        if (!mbar_wait(&p_full[wg], (uint32_t)((it >> 1) & 1), ab)) return false;
+        const int it = (int)(code >> 8), st = (int)((code >> 4) & 15), buf = it & 1;
+        const bool first = (code & 1u) != 0;
+        if (!mbar_wait(&p_full[buf], (uint32_t)((it >> 1) & 1), ab)) return false;
         // the accumulator of the previous segment must have been read before it is overwritten
-        if (first_of_wg && sg > 0 && !mbar_wait(&o_read[wg], (uint32_t)((sg - 1) & 1), ab)) return false;
+        if (first && sg > 0 && !mbar_wait(&o_read, (uint32_t)((sg - 1) & 1), ab)) return false;
         tc_fence_after();
         const uint64_t dv = dv0 + stage_step * (uint64_t)st;
-        const uint64_t dp = dp0 + (uint64_t)(wg * (PBUF_BYTES >> 4));
-        const uint32_t d = tmem + 64u + (uint32_t)wg * 32u;
-        umma_ss(d, dv, dp, idesc_pv, first_of_wg ? 0u : 1u);
+        const uint64_t dp = dp0 + (uint64_t)(buf * (PBUF_BYTES >> 4));
+        umma_ss(tm_o, dv, dp, idesc_pv, first ? 0u : 1u);
 #pragma unroll
         for (int ks = 1; ks < TK / 16; ++ks)
-          umma_ss(d, dv + (uint64_t)(ks * 128), dp + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_pv, 1u);
-        umma_commit(&o_full[wg]);
+          umma_ss(tm_o, dv + (uint64_t)(ks * 128), dp + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_pv, 1u);
+        umma_commit(&p_free[buf]);
         umma_commit(&empty_bar[st]);
         return true;
       };
       auto pop_pv = [&]() -> bool {
         const bool good = issue_pv(pq0, pv_seg0);
-        pq0 = pq1; pq1 = pq2; pv_seg0 = pv_seg1; pv_seg1 = pv_seg2;
+        pq0 = pq1; pv_seg0 = pv_seg1;
         --n_pend;
         return good;
       };
       Walk w;
       w.init(p, t_begin, t_end, b0, seq_first);
       const int n_tiles = (int)(t_end - t_begin);
-      int seg = -1;
-      int st = 0;                    // ring stage of the next score tile, and the parity of its round
+      int seg = -1, st = 0, n_last = 0;
       uint32_t st_par = 0;
-      int wg_tiles0 = 0, wg_tiles1 = 0;   // tiles of the current segment issued per warpgroup
-      int n_last0 = 0, n_last1 = 0;       // patched (last) tiles seen per warpgroup
       for (int it = 0; it < n_tiles && ok; ++it) {
-        // ---- keep the scores `ahead` tiles in front of the P V products ----
-        while (n_pend > ahead && ok) ok = pop_pv();
+        while (n_pend > 1 && ok) ok = pop_pv();      // the scores run one tile ahead of the P V products
         if (!ok) break;
         const long t = t_begin + it;
         w.seek(t);
-        const int wg = it & 1, j = it >> 1;
-        if (w.seg_start(t)) {
+        const int buf = it & 1, j = it >> 1;
+        const bool first = w.seg_start(t);
+        if (first) {
           ++seg;
-          wg_tiles0 = wg_tiles1 = 0;
           if (!(ok = mbar_wait(&q_full[seg & 1], (uint32_t)((seg >> 1) & 1), ab))) break;
         }
         if (!(ok = mbar_wait(&full_bar[st], st_par, ab))) break;
         if (w.last_tile(t)) {
-          // The warpgroup patches this tile only after it has flushed the segments before it, and such a
+          // Warpgroup 0 patches this tile only after it has flushed the segments before it, and such a
           // flush waits for every P V issued so far: issue the pending ones first.
           while (n_pend > 0 && ok) ok = pop_pv();
           if (!ok) break;
-          int& nl = wg ? n_last1 : n_last0;
-          if (!(ok = mbar_wait(&patched[wg], (uint32_t)(nl & 1), ab))) break;
-          ++nl;
+          if (!(ok = mbar_wait(&patched, (uint32_t)(n_last & 1), ab))) break;
+          ++n_last;
         }
-        // the warpgroup has taken the scores of its previous tile out of this buffer
-        if (j > 0 && !(ok = mbar_wait(&s_free[wg], (uint32_t)((j - 1) & 1), ab))) break;
+        // both warpgroups have taken the scores of tile it - 2 out of this buffer
+        if (j > 0 && !(ok = mbar_wait(&s_free[buf], (uint32_t)((j - 1) & 1), ab))) break;
         tc_fence_after();
         {
           const uint64_t dk = dk0 + stage_step * (uint64_t)st;
           const uint64_t dq = dq0 + (uint64_t)((seg & 1) * (QBUF_BYTES >> 4));
-          const uint32_t d = tmem + (uint32_t)wg * 32u;
+          const uint32_t d = tmem + (uint32_t)buf * 32u;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
             if (ks < ksteps)
               umma_ss(d, dk + (uint64_t)((ks >> 2) * (SUB_BYTES >> 4) + (ks & 3) * 2),
                       dq + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_qk, ks != 0 ? 1u : 0u);
-          umma_commit(&s_full[wg]);
+          umma_commit(&s_full[buf]);
           if (w.seg_end(t)) umma_commit(&q_empty[seg & 1]);   // the segment's Qhat buffer is free once these complete
         }
         {
-          int& wt = wg ? wg_tiles1 : wg_tiles0;
-          const uint32_t code = ((uint32_t)it << 8) | ((uint32_t)st << 4) | (wt == 0 ? 2u : 0u);
-          if (n_pend == 0) { pq0 = code; pv_seg0 = seg; }
-          else if (n_pend == 1) { pq1 = code; pv_seg1 = seg; }
-          else { pq2 = code; pv_seg2 = seg; }
+          const uint32_t code = ((uint32_t)it << 8) | ((uint32_t)st << 4) | (first ? 1u : 0u);
+          if (n_pend == 0) { pq0 = code; pv_seg0 = seg; } else { pq1 = code; pv_seg1 = seg; }
           ++n_pend;
-          ++wt;
         }
         if (++st == STAGES) { st = 0; st_par ^= 1u; }
       }
@@ -338,15 +321,15 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
    if (have_work) {
     // ------------------------------- softmax warpgroups --------------------------
-    const int wg = (warp - 4) / 4;
+    const int wg = (warp - 4) / 4;              // heads [16 wg, 16 wg + 16)
     const int q = warp % 4;                     // TMEM lane quadrant
     const int tid = q * 32 + lane;              // key row of a score tile / value coordinate of O^T
+    const int hl = lane & 15;                   // the head (within the group) whose maxima / sums this lane combines
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    uint8_t* my_p = pbuf + wg * PBUF_BYTES;
-    // this thread's P element (head h) lives at my_p + p_off + h * 128 + ((p_chunk ^ (h & 7)) << 4)
-    const uint32_t p_off = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(tid & 7) * 2;
-    const int p_chunk = (tid & 63) >> 3;
-    uint32_t wg_phase = 0, cta_phase = 0;
+    // this thread's P element of head 16 wg + j lives at p_row0 + j * 128 + ((p_chunk ^ (j & 7)) << 4) in a P buffer
+    const uint32_t p_row0 = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(wg * 16) * 128 + (uint32_t)(tid & 7) * 2;
+    const int p_chunk = (tid & 63) >> 3;        // (16 wg + j) & 7 == j & 7
+    uint32_t wg_phase = 0;
     bool ok = true;
     auto wg_sync = [&]() -> bool {
       __syncwarp();
@@ -355,177 +338,139 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       ++wg_phase;
       return __all_sync(0xffffffffu, good);
     };
-    auto cta_sync = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&cta_bar);
-      bool good = mbar_wait(&cta_bar, cta_phase & 1, ab);
-      ++cta_phase;
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      bool good = mbar_wait(bar, parity, ab);
       return __all_sync(0xffffffffu, good);
     };
     Walk w;
     w.init(p, t_begin, t_end, b0, seq_first);
-    int it = 0, seg = -1;
-    int n_mine = 0;            // tiles of the current segment handled by this warpgroup
-    int j_last = 0;            // index (it >> 1) of the latest tile handled by this warpgroup
-    float m_used[32], l_acc[32];
-    float m_lane = -INFINITY;  // m_used[lane]
+    int it = 0, n_seen = 0;    // tiles of the current segment handled so far
+    float m_used[16], l_acc[16];
+    float m_lane = -INFINITY;  // m_used[hl]
     for (long t = t_begin; t < t_end && ok; ++t, ++it) {
       w.seek(t);
       if (w.seg_start(t)) {
-        ++seg;
-        n_mine = 0;
+        n_seen = 0;
         m_lane = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < 32; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
+        for (int h = 0; h < 16; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
       }
-      if ((it & 1) == wg) {
-        const int s = it % STAGES, j = it >> 1;
-        const int k0 = w.k0(t), L = w.L;
-        const bool last_tile = w.last_tile(t);
-        if (last_tile) {
-          // the tile holding the new token: its row comes from the workspace, rows past it are invalid
-          ok = mbar_wait(&full_bar[s], (uint32_t)((it / STAGES) & 1), ab);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          uint8_t* kt = ring + (size_t)s * stage_bytes;
-          uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;
-          const int rnew = L - k0;
-          if (tid == rnew) {
-            const uint4* ks = reinterpret_cast<const uint4*>(p.knew + (long)w.b * p.r3);
-            for (int c = 0; c < p.r3 / 8; ++c) *reinterpret_cast<uint4*>(kt + swz(tid, c)) = ks[c];
-            const uint4* vs = reinterpret_cast<const uint4*>(p.vnew + (long)w.b * p.t3);
-            for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = vs[c];
-          } else if (tid > rnew) {
-            for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&patched[wg]);
+      const int s = it % STAGES, buf = it & 1, j = it >> 1;
+      const int k0 = w.k0(t), L = w.L;
+      if (w.last_tile(t) && wg == 0) {
+        // the tile holding the new token: its row comes from the workspace, rows past it are invalid
+        if (!(ok = wait_all(&full_bar[s], (uint32_t)((it / STAGES) & 1)))) break;
+        uint8_t* kt = ring + (size_t)s * stage_bytes;
+        uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;
+        const int rnew = L - k0;
+        if (tid == rnew) {
+          const uint4* ks = reinterpret_cast<const uint4*>(p.knew + (long)w.b * p.r3);
+          for (int c = 0; c < p.r3 / 8; ++c) *reinterpret_cast<uint4*>(kt + swz(tid, c)) = ks[c];
+          const uint4* vs = reinterpret_cast<const uint4*>(p.vnew + (long)w.b * p.t3);
+          for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = vs[c];
+        } else if (tid > rnew) {
+          for (int c = 0; c < p.t3 / 8; ++c) *reinterpret_cast<uint4*>(vt + swz(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
         }
-        ok = mbar_wait(&s_full[wg], (uint32_t)(j & 1), ab);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&patched);
+      }
+      if (!(ok = wait_all(&s_full[buf], (uint32_t)(j & 1)))) break;
+      tc_fence_after();
+      uint32_t sr[16];
+      tmem_ld16(tmem + (uint32_t)buf * 32u + (uint32_t)wg * 16u + lane_addr, sr);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_free[buf]);       // the scores of tile it + 2 may overwrite the buffer
+      float sc[16];
+      const bool visible = (k0 + tid) <= L;
+#pragma unroll
+      for (int h = 0; h < 16; ++h) sc[h] = visible ? __uint_as_float(sr[h]) : -INFINITY;
+      // ---- maximum per head over the 128 keys of the tile ----
+      {
+        float tmp[16];
+#pragma unroll
+        for (int h = 0; h < 16; ++h) tmp[h] = sc[h];
+        const float wm = transpose_reduce16<true>(tmp, lane);
+        if (lane < 16) mxh[wg][buf][q][lane] = __float2bfloat16_rn(wm);
+      }
+      if (!(ok = wg_sync())) break;
+      const float mt = fmaxf(fmaxf(__bfloat162float(mxh[wg][buf][0][hl]), __bfloat162float(mxh[wg][buf][1][hl])),
+                             fmaxf(__bfloat162float(mxh[wg][buf][2][hl]), __bfloat162float(mxh[wg][buf][3][hl])));
+      // every tile holds at least one visible key (the last one holds the new token), so mt is finite
+      const bool need = mt > m_lane + kRescaleThreshold;
+      if (__any_sync(0xffffffffu, need)) {
+        const float m_new = need ? mt : m_lane;
+        const float f_lane = need ? ex2(m_lane - m_new) : 1.f;     // exp2(-inf) = 0 on the first tile
+        float fac[16];
+#pragma unroll
+        for (int h = 0; h < 16; ++h) {
+          fac[h] = __shfl_sync(0xffffffffu, f_lane, h);
+          m_used[h] = __shfl_sync(0xffffffffu, m_new, h);
+          l_acc[h] *= fac[h];
+        }
+        m_lane = m_new;
+        if (n_seen > 0) {
+          // P V of the previous tile must be complete before its accumulator columns are rescaled
+          if (!(ok = wait_all(&p_free[(it - 1) & 1], (uint32_t)(((it - 1) >> 1) & 1)))) break;
+          tc_fence_after();
+          uint32_t o[16];
+          tmem_ld16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int h = 0; h < 16; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * fac[h]);
+          tmem_st16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
+          tmem_st_wait();
+        }
+      }
+      // the P V product of tile it - 2 must have finished reading this P buffer
+      if (j > 0 && !(ok = wait_all(&p_free[buf], (uint32_t)((j - 1) & 1)))) break;
+      // ---- p = exp2(s - m), bf16, into the P operand; row sums per thread ----
+      {
+        uint8_t* my_p = pbuf + buf * PBUF_BYTES + p_row0;
+#pragma unroll
+        for (int h = 0; h < 16; ++h) {
+          const float pv = ex2(sc[h] - m_used[h]);
+          l_acc[h] += pv;
+          *reinterpret_cast<__nv_bfloat16*>(my_p + h * 128 + ((p_chunk ^ (h & 7)) << 4)) = __float2bfloat16_rn(pv);
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[buf]);
+      ++n_seen;
+      if (w.seg_end(t)) {
+        // ---- segment done: this warpgroup's 16 heads of the partial of (CTA, sequence) ----
+        if (!(ok = wait_all(&p_free[buf], (uint32_t)(j & 1)))) break;      // P V of this tile is complete
         tc_fence_after();
-        uint32_t sr[32];
-        tmem_ld32(tm_s[wg] + lane_addr, sr);
+        uint32_t o[16];
+        tmem_ld16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&s_free[wg]);     // the next scores may overwrite the buffer
-        float sc[32];
-        const bool visible = (k0 + tid) <= L;
+        if (lane == 0) mbar_arrive(&o_read);       // the next segment may overwrite the accumulator
+        {
+          float tmp[16];
 #pragma unroll
-        for (int h = 0; h < 32; ++h) sc[h] = visible ? __uint_as_float(sr[h]) : -INFINITY;
-        // ---- maximum per head over the 128 keys of the tile ----
-        float tmp[32];
-#pragma unroll
-        for (int h = 0; h < 32; ++h) tmp[h] = sc[h];
-        mxh[wg][j & 1][q][lane] = __float2bfloat16_rn(transpose_reduce<true>(tmp, lane));
+          for (int h = 0; h < 16; ++h) tmp[h] = l_acc[h];
+          const float ws = transpose_reduce16<false>(tmp, lane);   // row sums over this warp's 32 keys
+          if (lane < 16) sum_s[wg][q][lane] = ws;
+        }
         if (!(ok = wg_sync())) break;
-        const float mt = fmaxf(fmaxf(__bfloat162float(mxh[wg][j & 1][0][lane]), __bfloat162float(mxh[wg][j & 1][1][lane])),
-                               fmaxf(__bfloat162float(mxh[wg][j & 1][2][lane]), __bfloat162float(mxh[wg][j & 1][3][lane])));
-        // every tile holds at least one visible key (the last one holds the new token), so mt is finite
-        const bool need = mt > m_lane + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          const float m_new = need ? mt : m_lane;
-          const float f_lane = need ? ex2(m_lane - m_new) : 1.f;     // exp2(-inf) = 0 on the first tile
-          float fac[32];
-#pragma unroll
-          for (int h = 0; h < 32; ++h) {
-            fac[h] = __shfl_sync(0xffffffffu, f_lane, h);
-            m_used[h] = __shfl_sync(0xffffffffu, m_new, h);
-            l_acc[h] *= fac[h];
-          }
-          m_lane = m_new;
-          if (n_mine > 0) {
-            ok = mbar_wait(&o_full[wg], (uint32_t)(j_last & 1), ab);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t o[32];
-            tmem_ld32(tm_o[wg] + lane_addr, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int h = 0; h < 32; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * fac[h]);
-            tmem_st32(tm_o[wg] + lane_addr, o);
-            tmem_st_wait();
-          }
-        }
-        // (This parity's exchange buffer is written again two tiles on, after the group's sync of the
-        // tile in between, which every warp reaches only after its reads above.)
-        // ---- p = exp2(s - m), bf16, into the P operand; row sums per thread ----
-        if (j > 0) {
-          // the P V of this group's previous tile must have finished reading the P buffer
-          ok = mbar_wait(&o_full[wg], (uint32_t)((j - 1) & 1), ab);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
-#pragma unroll
-        for (int h = 0; h < 32; ++h) {
-          const float pv = ex2(sc[h] - m_used[h]);
-          l_acc[h] += pv;
-          const __nv_bfloat16 pb = __float2bfloat16_rn(pv);
-          *reinterpret_cast<__nv_bfloat16*>(my_p + p_off + h * 128 + ((p_chunk ^ (h & 7)) << 4)) = pb;
-        }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&p_full[wg]);
-        ++n_mine;
-        j_last = j;
-      }
-      if (w.seg_end(t)) {
-        // ---- segment done: merge the two warpgroups' states, write the partial of (CTA, sequence) ----
-        float o[32];
-        if (n_mine > 0) {
-          ok = mbar_wait(&o_full[wg], (uint32_t)(j_last & 1), ab);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
-          uint32_t orr[32];
-          tmem_ld32(tm_o[wg] + lane_addr, orr);
-          tmem_ld_wait();
-#pragma unroll
-          for (int h = 0; h < 32; ++h) o[h] = __uint_as_float(orr[h]);
-        } else {
-#pragma unroll
-          for (int h = 0; h < 32; ++h) o[h] = 0.f;
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&o_read[wg]);
-        float tmp[32];
-#pragma unroll
-        for (int h = 0; h < 32; ++h) tmp[h] = l_acc[h];
-        sum_s[wg][q][lane] = transpose_reduce<false>(tmp, lane);   // row sums over this warp's 32 keys
-        if (q == 0) m_s[wg][lane] = m_lane;
-        if (!(ok = cta_sync())) break;
-        const float ma = m_s[0][lane], mb = m_s[1][lane];
-        const float M = fmaxf(ma, mb);                               // finite: the segment has at least one tile
-        const float wa = (ma == -INFINITY) ? 0.f : ex2(ma - M), wb = (mb == -INFINITY) ? 0.f : ex2(mb - M);
-        const float Ltot = (sum_s[0][0][lane] + sum_s[0][1][lane] + sum_s[0][2][lane] + sum_s[0][3][lane]) * wa +
-                           (sum_s[1][0][lane] + sum_s[1][1][lane] + sum_s[1][2][lane] + sum_s[1][3][lane]) * wb;
-        const float w_own = wg == 0 ? wa : wb;
         const long slot = (long)blockIdx.x + w.b;
-        if (wg == 1 && tid < p.t3) {      // warp-uniform: t3 is a multiple of 32
-#pragma unroll
-          for (int h = 0; h < 32; ++h) obuf[h * p.t3 + tid] = o[h] * __shfl_sync(0xffffffffu, w_own, h);
+        if (q == 0 && lane < 16) {
+          float* ml = p.part_ml + slot * 64 + (wg * 16 + lane) * 2;
+          ml[0] = m_lane;
+          ml[1] = sum_s[wg][0][lane] + sum_s[wg][1][lane] + sum_s[wg][2][lane] + sum_s[wg][3][lane];
         }
-        if (!(ok = cta_sync())) break;
-        if (wg == 0) {
-          float* dst = p.part_o + slot * 32 * p.t3;
+        if (tid < p.t3) {
+          float* dst = p.part_o + slot * 32 * p.t3 + (long)(wg * 16) * p.t3 + tid;
 #pragma unroll
-          for (int h = 0; h < 32; ++h) {
-            const float wh = __shfl_sync(0xffffffffu, w_own, h);
-            if (tid < p.t3) dst[h * p.t3 + tid] = o[h] * wh + obuf[h * p.t3 + tid];
-          }
-          if (q == 0) {
-            float* ml = p.part_ml + slot * 64;
-            ml[lane * 2 + 0] = M;
-            ml[lane * 2 + 1] = Ltot;
-          }
+          for (int h = 0; h < 16; ++h) dst[h * p.t3] = __uint_as_float(o[h]);
         }
-        if (!(ok = cta_sync())) break;   // the merge buffer aliases the P operands of the next segment
+        if (!(ok = wg_sync())) break;      // sum_s is free again before the next segment's flush writes it
       }
     }
    }
