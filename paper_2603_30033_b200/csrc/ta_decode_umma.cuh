@@ -92,6 +92,12 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// maximum of x over the 32 lanes of the warp, in every lane (one instruction)
+__device__ __forceinline__ float warp_max(float x) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+  return r;
+}
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * SUB_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
@@ -130,7 +136,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   // per tile: the four warps' maxima per head of each warpgroup, as bf16 (the reference maximum only has
   // to be the same for all threads and close to the true one), double-buffered by tile parity because a
   // warp may start the next tile while another still reads this one's; per segment: the warps' row sums
-  __shared__ __nv_bfloat16 mxh[2][2][4][16];      // [wg][tile parity][warp][head]
+  __shared__ __align__(16) __nv_bfloat16 mxh[2][2][4][16];   // [wg][tile parity][warp][head]
   __shared__ float sum_s[2][4][16];               // [wg][warp][head]
   __shared__ long long wtot_s[THREADS / 32];
   __shared__ int loc_b;
@@ -329,6 +335,9 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // this thread's P element of head 16 wg + j lives at p_row0 + j * 128 + ((p_chunk ^ (j & 7)) << 4) in a P buffer
     const uint32_t p_row0 = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(wg * 16) * 128 + (uint32_t)(tid & 7) * 2;
     const int p_chunk = (tid & 63) >> 3;        // (16 wg + j) & 7 == j & 7
+    uint32_t p_sw[8];                           // offset of head row j (mod 8) incl. the 128-byte swizzle
+#pragma unroll
+    for (int e = 0; e < 8; ++e) p_sw[e] = (uint32_t)(e * 128 + ((p_chunk ^ e) << 4));
     uint32_t wg_phase = 0;
     bool ok = true;
     auto wg_sync = [&]() -> bool {
@@ -355,9 +364,11 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
         for (int h = 0; h < 16; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
       }
-      const int s = it % STAGES, buf = it & 1, j = it >> 1;
+      const int buf = it & 1, j = it >> 1;
       const int k0 = w.k0(t), L = w.L;
-      if (w.last_tile(t) && wg == 0) {
+      const bool last_tile = w.last_tile(t);
+      if (last_tile && wg == 0) {
+        const int s = it % STAGES;
         // the tile holding the new token: its row comes from the workspace, rows past it are invalid
         if (!(ok = wait_all(&full_bar[s], (uint32_t)((it / STAGES) & 1)))) break;
         uint8_t* kt = ring + (size_t)s * stage_bytes;
@@ -384,16 +395,22 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_free[buf]);       // the scores of tile it + 2 may overwrite the buffer
       float sc[16];
-      const bool visible = (k0 + tid) <= L;
 #pragma unroll
-      for (int h = 0; h < 16; ++h) sc[h] = visible ? __uint_as_float(sr[h]) : -INFINITY;
-      // ---- maximum per head over the 128 keys of the tile ----
+      for (int h = 0; h < 16; ++h) sc[h] = __uint_as_float(sr[h]);
+      if (last_tile && (k0 + tid) > L) {       // keys past the new token do not exist
+#pragma unroll
+        for (int h = 0; h < 16; ++h) sc[h] = -INFINITY;
+      }
+      // ---- maximum per head over the 128 keys of the tile: one warp-wide max per head, lane 0 publishes ----
       {
-        float tmp[16];
+        uint32_t pk[8];
 #pragma unroll
-        for (int h = 0; h < 16; ++h) tmp[h] = sc[h];
-        const float wm = transpose_reduce16<true>(tmp, lane);
-        if (lane < 16) mxh[wg][buf][q][lane] = __float2bfloat16_rn(wm);
+        for (int h = 0; h < 16; h += 2) pk[h >> 1] = pack_bf16(warp_max(sc[h]), warp_max(sc[h + 1]));
+        if (lane == 0) {
+          uint4* dst = reinterpret_cast<uint4*>(&mxh[wg][buf][q][0]);
+          dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        }
       }
       if (!(ok = wg_sync())) break;
       const float mt = fmaxf(fmaxf(__bfloat162float(mxh[wg][buf][0][hl]), __bfloat162float(mxh[wg][buf][1][hl])),
@@ -433,7 +450,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         for (int h = 0; h < 16; ++h) {
           const float pv = ex2(sc[h] - m_used[h]);
           l_acc[h] += pv;
-          *reinterpret_cast<__nv_bfloat16*>(my_p + h * 128 + ((p_chunk ^ (h & 7)) << 4)) = __float2bfloat16_rn(pv);
+          *reinterpret_cast<__nv_bfloat16*>(my_p + (h >> 3) * 1024 + p_sw[h & 7]) = __float2bfloat16_rn(pv);
         }
       }
       fence_proxy_async_smem();
