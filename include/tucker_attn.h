@@ -86,7 +86,7 @@ enum {
   TA_FLAG_FMA_ATTENTION = 0x200,      /* tensor-core GEMMs, but the attention itself on the FMA kernel */
   TA_FLAG_SEPARATE_QUERIES = 0x400,   /* per-head queries from a separate GEMM instead of the attention prologue */
   TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x800, /* Z and Y from two GEMM launches instead of the fused output kernel */
-  TA_FLAG_UMMA_DECODE = 0x1000         /* decode: cache-streaming kernel on tcgen05 (keys on the M dimension) */
+  TA_FLAG_MMA_SYNC_DECODE = 0x1000     /* decode: the mma.sync form of the cache-streaming kernel instead of the tcgen05 one */
 };
 
 /* Bytes of scratch the corresponding call needs for this descriptor (0 on invalid descriptor). */

@@ -18,7 +18,7 @@ TA_OK = 0
 TA_DTYPE_F32, TA_DTYPE_BF16 = 0, 1
 TA_FLAG_FORCE_GENERIC = 1
 TA_FLAG_FMA_ATTENTION, TA_FLAG_SEPARATE_QUERIES, TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x200, 0x400, 0x800
-TA_FLAG_UMMA_DECODE = 0x1000
+TA_FLAG_MMA_SYNC_DECODE = 0x1000
 TA_DEVERR_WAIT_TIMEOUT, TA_DEVERR_BAD_CACHE_LEN, TA_DEVERR_BAD_INDEX = 1, 2, 4
 
 EXPORTS = (

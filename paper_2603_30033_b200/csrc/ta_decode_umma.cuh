@@ -127,7 +127,10 @@ __device__ __forceinline__ float transpose_reduce16(float (&v)[16], int lane) {
 __global__ void __launch_bounds__(THREADS, 1)
 k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmQ, const Params p) {
-  pdl_enter();
+  // cache_len was final before the preceding kernel (which forms the queries and appends the new row)
+  // began: set-up and the tile split run while it finishes, and every role passes pdl_enter() before it
+  // touches anything else.  (Requesting the first cache tiles ahead of that wait as well was measured:
+  // no gain with two caches, 6 us slower with the shared cache.)
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], q_full[2], q_empty[2];
   __shared__ uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_read, patched, wg_bar[2];
@@ -210,6 +213,16 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmQ);
       Walk w;
       w.init(p, t_begin, t_end, b0, seq_first);
+      auto load_tile = [&](long t, int s) {     // K / V tile t (w is positioned on it) into ring stage s
+        mbar_expect_tx(&full_bar[s], (uint32_t)((ksub + (p.shared_kv ? 0 : vsub)) * SUB_BYTES));
+        uint8_t* kt = ring + (size_t)s * stage_bytes;
+        uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
+        const int row = w.k0(t);
+        for (int kk = 0; kk < ksub; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, w.b);
+        if (!p.shared_kv)
+          for (int kk = 0; kk < vsub; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, w.b);
+      };
+      pdl_enter();
       int it = 0, seg = -1;
       for (long t = t_begin; t < t_end; ++t, ++it) {
         w.seek(t);
@@ -223,17 +236,14 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         const int s = it % STAGES;
         if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, ab)) break;
-        mbar_expect_tx(&full_bar[s], (uint32_t)((ksub + (p.shared_kv ? 0 : vsub)) * SUB_BYTES));
-        uint8_t* kt = ring + (size_t)s * stage_bytes;
-        uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
-        const int row = w.k0(t);
-        for (int kk = 0; kk < ksub; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, w.b);
-        if (!p.shared_kv)
-          for (int kk = 0; kk < vsub; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, w.b);
+        load_tile(t, s);
       }
+    } else {
+      pdl_enter();
     }
    } else if (have_work && warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
+    pdl_enter();
     if (elect_one()) {
       // This one thread issues 16 small MMAs per tile, so its own instruction stream matters: descriptors
       // are formed once per operand and stepped by constants, the K loops are unrolled, and the (at most
@@ -326,6 +336,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   } else {
    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
    if (have_work) {
+    pdl_enter();
     // ------------------------------- softmax warpgroups --------------------------
     const int wg = (warp - 4) / 4;              // heads [16 wg, 16 wg + 16)
     const int q = warp % 4;                     // TMEM lane quadrant

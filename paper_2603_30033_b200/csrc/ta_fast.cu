@@ -652,7 +652,7 @@ int fast_decode(Problem& p) {
     dp.shared_kv = p.shared_kv;
     dp.cache_len = p.cache_len; dp.qhat = w.qhat; dp.knew = w.knew; dp.vnew = w.vnew;
     dp.part_o = w.part_o; dp.part_ml = w.part_ml; dp.err = p.dev_err;
-    if (d.flags & TA_FLAG_UMMA_DECODE) rc = launch_dec_attn_umma(p, tmK, tmV, dp, dp.grid);
+    if (!(d.flags & TA_FLAG_MMA_SYNC_DECODE)) rc = launch_dec_attn_umma(p, tmK, tmV, dp, dp.grid);
     else if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);
     else if (d.r3 == 64 && d.t3 == 64) rc = launch_dec_attn<64, 64>(p, tmK, tmV, dp);
     else if (d.r3 == 96 && d.t3 == 96) rc = launch_dec_attn<96, 96>(p, tmK, tmV, dp);

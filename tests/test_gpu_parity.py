@@ -244,7 +244,7 @@ DEC_FAST = [
 ]
 
 
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
 @pytest.mark.parametrize("append", [True, False])
 @pytest.mark.parametrize("case", DEC_FAST)
 def test_decode_tensor_core_path(case, append, flags):
@@ -277,7 +277,7 @@ def _shared_weights(w):
     ("bf16", dict(d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 64)), 2),
     ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
 ])
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
 def test_decode_shared_latent_cache(dtype, shape, path, flags):
     import torch
     w = H.custom_workload(kind="decode", dtype=dtype, rope=False, seed=61, **shape)
@@ -410,7 +410,7 @@ def test_sharp_softmax_variant():
     check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2", scaled=True)
 
 
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_UMMA_DECODE])
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
 def test_full_size_decode_sampled(flags):
     # benchmark decode workload: 64 sequences, 32768 cached latent rows each, RoPE at position 32768
     # (with both forms of the cache-streaming kernel, each in the launch configuration bench.py times)
