@@ -1,10 +1,13 @@
-// Decode step over the latent KV cache (Eq. 9, "KV Caching"): kernels of the bf16 path.
+// Decode step over the latent KV cache (Eq. 9, "KV Caching"): kernels of the bf16 path -- the query kernel
+// k_dec_qhat, the output kernel k_dec_out, and k_dec_attn, the mma.sync form of the cache-streaming kernel
+// (the tcgen05 form in ta_decode_umma.cuh is the one used unless TA_FLAG_MMA_SYNC_DECODE asks for this one;
+// both share the tile split, the helpers below and the partial format).
 //
 // k_dec_attn streams every sequence's latent K / V cache exactly once.  The cache is cut into
 // tiles of 128 keys; the flat list of tiles of all sequences is divided evenly over the CTAs
 // (one per SM), so that the load is balanced for any mix of cache lengths.  Each CTA walks its
 // tile range, keeps an online-softmax state per sequence segment, and writes one partial
-// (max, sum, unnormalised O for all heads) per segment; k_dec_merge combines the partials of
+// (max, sum, unnormalised O for all heads) per segment; k_dec_out combines the partials of
 // a sequence with log-sum-exp weights and applies the output-side core (Z = sum_h o_h Gt_h^T).
 //
 // All n_H (<= 32) heads share each K / V byte, so the arithmetic is 2 * n_H flop per cached

@@ -598,7 +598,7 @@ size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t) { return carve_
 //   1  split-K GEMM   partial [qt | k | v] = x [U2 | U3 | Ut3]           (factors read in place)
 //   2  k_dec_qhat     finish the projections, latent RoPE, cache append, per-head queries (core
 //                     contracted with the query first; no per-head G_h)
-//   3  k_dec_attn     stream the latent caches once (all heads per tile)
+//   3  k_dec_attn_umma  stream the latent caches once, all heads per tile (tcgen05; k_dec_attn is the mma.sync form)
 //   4  k_dec_out      merge the partials, output-side core -> z
 //   5  GEMM           y = z Ut2^T
 int fast_decode(Problem& p) {
