@@ -44,6 +44,7 @@ NCU_TRAFFIC_BYTES = {
     "c4_long_prefill": 17.91e6 + 78.09e6,     # attn::k_attn_prefill, profiles/k_attn_prefill_c4_long_prefill.md
     "c3_vit_prefill": 34.14e6 + 65.40e6,      # attn::k_attn_prefill, profiles/k_attn_prefill_c3_vit_prefill.md
     "c5_decode": 1075.34e6 + 4.56e6,          # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_c5_decode.md
+    "f1_decode_shared_kv": 538.05e6 + 4.87e6,  # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_f1_decode_shared_kv.md
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
