@@ -5,20 +5,21 @@
 // no tensor work is spent on padding the (at most 32) heads up to a 128-row tile:
 //   S^T [128 keys x 32 heads] = K_tile [128 x r3] * Qhat^T          A = K tile as loaded (K-major), B = Qhat (K-major)
 //   O^T [t3 x 32 heads]      += V_tile^T [t3 x 128] * P [128 x 32]  A = V tile as loaded (M-major), B = P (K-major, bf16)
-// The scores of one tile sit in TMEM with one key per lane and one head per column.  Two softmax
-// warpgroups work on EVERY tile, each on 16 of the 32 head columns: a thread owns one key and 16 heads.
+// The scores of one tile sit in TMEM with one key per lane and one head per column.  NWG softmax
+// warpgroups work on EVERY tile, each on HPW = 32 / NWG of the 32 head columns: a thread owns one key and
+// HPW heads (the per-tile work of a thread is a latency chain, so more, thinner threads finish a tile sooner).
 // The per-head maximum over the keys of a tile is a reduction ACROSS threads (a transposing butterfly of
 // warp shuffles, then four values per head through shared memory); it only moves the reference maximum
 // of a head when that grows by more than 8 (factor 256), so the accumulator in TMEM is rescaled rarely.
 // P goes back through shared memory (B operands are read from there); the row sums stay in registers
 // per thread and are reduced once per segment.  Score and P buffers are double-buffered, the output
 // accumulator is single: tile t + 1 is scored and exponentiated while P V of tile t runs, and a segment
-// ends with each warpgroup writing its 16 heads of the partial -- the same partial per (CTA, sequence)
+// ends with each warpgroup writing its heads of the partial -- the same partial per (CTA, sequence)
 // that the mma.sync kernel writes.
 //
 //   warp 0       TMA producer: Qhat of the segment's sequence, K / V ring
 //   warp 1       TMEM allocation, MMA issue
-//   warps 4..7   softmax warpgroup 0 (heads 0..15)     warps 8..11  softmax warpgroup 1 (heads 16..31)
+//   warps 4 + 4 g .. 7 + 4 g   softmax warpgroup g (heads HPW g .. HPW g + HPW - 1)
 // TMEM columns: S_0 [0,32) S_1 [32,64) O [64,96).
 // Every wait is bounded (Abort): on a timeout the CTA raises the device error word and leaves.
 #pragma once
@@ -35,7 +36,9 @@ using dec::clamp_len;
 using dec::tiles_of;
 
 constexpr int TK = 128;                  // keys per tile
-constexpr int THREADS = 384;
+constexpr int NWG = 2;                    // softmax warpgroups (4 was measured: slower, 138 us against 118 us with the shared cache)
+constexpr int HPW = 32 / NWG;             // head columns per warpgroup
+constexpr int THREADS = 128 + 128 * NWG;
 constexpr int MAX_STAGES = 6;
 constexpr int SUB_BYTES = 128 * 64 * 2;  // [128 keys x 64] bf16
 constexpr int MAX_SUB = 2;               // r3, t3 <= 128
@@ -102,27 +105,22 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * SUB_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-// v[j] of every lane, j < 16 -> lanes j and j + 16 receive op over the 32 lanes of v[j] (returned in v[0]).
-template <bool IS_MAX>
-__device__ __forceinline__ float transpose_reduce16(float (&v)[16], int lane) {
+// sum of x over the 32 lanes of the warp, in every lane
+__device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const float o = __shfl_xor_sync(0xffffffffu, v[i], 16);
-    v[i] = IS_MAX ? fmaxf(v[i], o) : v[i] + o;
-  }
-#pragma unroll
-  for (int off = 8; off >= 1; off >>= 1) {
-    const bool up = (lane & off) != 0;
-#pragma unroll
-    for (int i = 0; i < off; ++i) {
-      const float send = up ? v[i] : v[i + off];
-      const float keep = up ? v[i + off] : v[i];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, off);
-      v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
-    }
-  }
-  return v[0];
+  for (int off = 16; off >= 1; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+  return x;
 }
+
+template <int N> struct TmemCols;
+template <> struct TmemCols<16> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t (&r)[16]) { tmem_ld16(a, r); }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t (&r)[16]) { tmem_st16(a, r); }
+};
+template <> struct TmemCols<8> {
+  static __device__ __forceinline__ void ld(uint32_t a, uint32_t (&r)[8]) { tmem_ld8(a, r); }
+  static __device__ __forceinline__ void st(uint32_t a, const uint32_t (&r)[8]) { tmem_st8(a, r); }
+};
 
 __global__ void __launch_bounds__(THREADS, 1)
 k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -133,14 +131,14 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   // no gain with two caches, 6 us slower with the shared cache.)
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], q_full[2], q_empty[2];
-  __shared__ uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_read, patched, wg_bar[2];
+  __shared__ uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_read, patched, wg_bar[NWG];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   // per tile: the four warps' maxima per head of each warpgroup, as bf16 (the reference maximum only has
   // to be the same for all threads and close to the true one), double-buffered by tile parity because a
   // warp may start the next tile while another still reads this one's; per segment: the warps' row sums
-  __shared__ __align__(16) __nv_bfloat16 mxh[2][2][4][16];   // [wg][tile parity][warp][head]
-  __shared__ float sum_s[2][4][16];               // [wg][warp][head]
+  __shared__ __align__(16) __nv_bfloat16 mxh[NWG][2][4][HPW];   // [wg][tile parity][warp][head]
+  __shared__ float sum_s[NWG][4][HPW];                          // [wg][warp][head]
   __shared__ long long wtot_s[THREADS / 32];
   __shared__ int loc_b;
   __shared__ long long loc_first;
@@ -167,12 +165,12 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mbar_init(&q_full[i], 1);
       mbar_init(&q_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&s_free[i], 8);      // the scores are in registers: one arrival per softmax warp
-      mbar_init(&p_full[i], 8);      // P is in shared memory: one arrival per softmax warp
-      mbar_init(&p_free[i], 1);      // the P V product that read this P buffer is complete
-      mbar_init(&wg_bar[i], 4);
+      mbar_init(&s_free[i], 4 * NWG);   // the scores are in registers: one arrival per softmax warp
+      mbar_init(&p_full[i], 4 * NWG);   // P is in shared memory: one arrival per softmax warp
+      mbar_init(&p_free[i], 1);         // the P V product that read this P buffer is complete
     }
-    mbar_init(&o_read, 8);
+    for (int i = 0; i < NWG; ++i) mbar_init(&wg_bar[i], 4);
+    mbar_init(&o_read, 4 * NWG);
     mbar_init(&patched, 4);
     fence_barrier_init();
   }
@@ -334,18 +332,23 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
    }
   } else {
-   asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+   // setmaxnreg.inc blocks until the registers exist: the request must fit the pool the CTA was launched
+   // with (registers at launch x threads) minus what the first warpgroup keeps.  2 warpgroups: 168 x 384
+   // = 64512 = 128 x 56 + 256 x 224.  4 warpgroups: 96 x 640 = 61440 >= 128 x 56 + 512 x 104 = 60416.
+   static_assert(NWG == 2 || NWG == 4, "register budgets below are written for 2 or 4 softmax warpgroups");
+   if (NWG == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+   else asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
    if (have_work) {
     pdl_enter();
     // ------------------------------- softmax warpgroups --------------------------
-    const int wg = (warp - 4) / 4;              // heads [16 wg, 16 wg + 16)
+    const int wg = (warp - 4) / 4;              // heads [HPW wg, HPW wg + HPW)
     const int q = warp % 4;                     // TMEM lane quadrant
     const int tid = q * 32 + lane;              // key row of a score tile / value coordinate of O^T
-    const int hl = lane & 15;                   // the head (within the group) whose maxima / sums this lane combines
+    const int hl = lane % HPW;                  // the head (within the group) whose maxima this lane combines
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    // this thread's P element of head 16 wg + j lives at p_row0 + j * 128 + ((p_chunk ^ (j & 7)) << 4) in a P buffer
-    const uint32_t p_row0 = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(wg * 16) * 128 + (uint32_t)(tid & 7) * 2;
-    const int p_chunk = (tid & 63) >> 3;        // (16 wg + j) & 7 == j & 7
+    // this thread's P element of head HPW wg + j lives at p_row0 + j * 128 + ((p_chunk ^ (j & 7)) << 4) in a P buffer
+    const uint32_t p_row0 = (uint32_t)(tid >> 6) * QSUB_BYTES + (uint32_t)(wg * HPW) * 128 + (uint32_t)(tid & 7) * 2;
+    const int p_chunk = (tid & 63) >> 3;        // (HPW wg + j) & 7 == j & 7 (HPW is a multiple of 8)
     uint32_t p_sw[8];                           // offset of head row j (mod 8) incl. the 128-byte swizzle
 #pragma unroll
     for (int e = 0; e < 8; ++e) p_sw[e] = (uint32_t)(e * 128 + ((p_chunk ^ e) << 4));
@@ -365,7 +368,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     Walk w;
     w.init(p, t_begin, t_end, b0, seq_first);
     int it = 0, n_seen = 0;    // tiles of the current segment handled so far
-    float m_used[16], l_acc[16];
+    float m_used[HPW], l_acc[HPW];
     float m_lane = -INFINITY;  // m_used[hl]
     for (long t = t_begin; t < t_end && ok; ++t, ++it) {
       w.seek(t);
@@ -373,7 +376,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         n_seen = 0;
         m_lane = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < 16; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
+        for (int h = 0; h < HPW; ++h) { m_used[h] = -INFINITY; l_acc[h] = 0.f; }
       }
       const int buf = it & 1, j = it >> 1;
       const int k0 = w.k0(t), L = w.L;
@@ -399,28 +402,28 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       }
       if (!(ok = wait_all(&s_full[buf], (uint32_t)(j & 1)))) break;
       tc_fence_after();
-      uint32_t sr[16];
-      tmem_ld16(tmem + (uint32_t)buf * 32u + (uint32_t)wg * 16u + lane_addr, sr);
+      uint32_t sr[HPW];
+      TmemCols<HPW>::ld(tmem + (uint32_t)buf * 32u + (uint32_t)(wg * HPW) + lane_addr, sr);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&s_free[buf]);       // the scores of tile it + 2 may overwrite the buffer
-      float sc[16];
+      float sc[HPW];
 #pragma unroll
-      for (int h = 0; h < 16; ++h) sc[h] = __uint_as_float(sr[h]);
+      for (int h = 0; h < HPW; ++h) sc[h] = __uint_as_float(sr[h]);
       if (last_tile && (k0 + tid) > L) {       // keys past the new token do not exist
 #pragma unroll
-        for (int h = 0; h < 16; ++h) sc[h] = -INFINITY;
+        for (int h = 0; h < HPW; ++h) sc[h] = -INFINITY;
       }
       // ---- maximum per head over the 128 keys of the tile: one warp-wide max per head, lane 0 publishes ----
       {
-        uint32_t pk[8];
+        uint32_t pk[HPW / 2];
 #pragma unroll
-        for (int h = 0; h < 16; h += 2) pk[h >> 1] = pack_bf16(warp_max(sc[h]), warp_max(sc[h + 1]));
+        for (int h = 0; h < HPW; h += 2) pk[h >> 1] = pack_bf16(warp_max(sc[h]), warp_max(sc[h + 1]));
         if (lane == 0) {
           uint4* dst = reinterpret_cast<uint4*>(&mxh[wg][buf][q][0]);
-          dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-          dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+#pragma unroll
+          for (int u = 0; u < HPW / 8; ++u) dst[u] = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
         }
       }
       if (!(ok = wg_sync())) break;
@@ -431,9 +434,9 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       if (__any_sync(0xffffffffu, need)) {
         const float m_new = need ? mt : m_lane;
         const float f_lane = need ? ex2(m_lane - m_new) : 1.f;     // exp2(-inf) = 0 on the first tile
-        float fac[16];
+        float fac[HPW];
 #pragma unroll
-        for (int h = 0; h < 16; ++h) {
+        for (int h = 0; h < HPW; ++h) {
           fac[h] = __shfl_sync(0xffffffffu, f_lane, h);
           m_used[h] = __shfl_sync(0xffffffffu, m_new, h);
           l_acc[h] *= fac[h];
@@ -443,12 +446,12 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           // P V of the previous tile must be complete before its accumulator columns are rescaled
           if (!(ok = wait_all(&p_free[(it - 1) & 1], (uint32_t)(((it - 1) >> 1) & 1)))) break;
           tc_fence_after();
-          uint32_t o[16];
-          tmem_ld16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
+          uint32_t o[HPW];
+          TmemCols<HPW>::ld(tm_o + (uint32_t)(wg * HPW) + lane_addr, o);
           tmem_ld_wait();
 #pragma unroll
-          for (int h = 0; h < 16; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * fac[h]);
-          tmem_st16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
+          for (int h = 0; h < HPW; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * fac[h]);
+          TmemCols<HPW>::st(tm_o + (uint32_t)(wg * HPW) + lane_addr, o);
           tmem_st_wait();
         }
       }
@@ -458,7 +461,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       {
         uint8_t* my_p = pbuf + buf * PBUF_BYTES + p_row0;
 #pragma unroll
-        for (int h = 0; h < 16; ++h) {
+        for (int h = 0; h < HPW; ++h) {
           const float pv = ex2(sc[h] - m_used[h]);
           l_acc[h] += pv;
           *reinterpret_cast<__nv_bfloat16*>(my_p + (h >> 3) * 1024 + p_sw[h & 7]) = __float2bfloat16_rn(pv);
@@ -473,30 +476,28 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // ---- segment done: this warpgroup's 16 heads of the partial of (CTA, sequence) ----
         if (!(ok = wait_all(&p_free[buf], (uint32_t)(j & 1)))) break;      // P V of this tile is complete
         tc_fence_after();
-        uint32_t o[16];
-        tmem_ld16(tm_o + (uint32_t)wg * 16u + lane_addr, o);
+        uint32_t o[HPW];
+        TmemCols<HPW>::ld(tm_o + (uint32_t)(wg * HPW) + lane_addr, o);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&o_read);       // the next segment may overwrite the accumulator
-        {
-          float tmp[16];
 #pragma unroll
-          for (int h = 0; h < 16; ++h) tmp[h] = l_acc[h];
-          const float ws = transpose_reduce16<false>(tmp, lane);   // row sums over this warp's 32 keys
-          if (lane < 16) sum_s[wg][q][lane] = ws;
+        for (int h = 0; h < HPW; ++h) {
+          const float ws = warp_sum(l_acc[h]);       // row sums over this warp's 32 keys
+          if (lane == h) sum_s[wg][q][h] = ws;
         }
         if (!(ok = wg_sync())) break;
         const long slot = (long)blockIdx.x + w.b;
-        if (q == 0 && lane < 16) {
-          float* ml = p.part_ml + slot * 64 + (wg * 16 + lane) * 2;
+        if (q == 0 && lane < HPW) {
+          float* ml = p.part_ml + slot * 64 + (wg * HPW + lane) * 2;
           ml[0] = m_lane;
           ml[1] = sum_s[wg][0][lane] + sum_s[wg][1][lane] + sum_s[wg][2][lane] + sum_s[wg][3][lane];
         }
         if (tid < p.t3) {
-          float* dst = p.part_o + slot * 32 * p.t3 + (long)(wg * 16) * p.t3 + tid;
+          float* dst = p.part_o + slot * 32 * p.t3 + (long)(wg * HPW) * p.t3 + tid;
 #pragma unroll
-          for (int h = 0; h < 16; ++h) dst[h * p.t3] = __uint_as_float(o[h]);
+          for (int h = 0; h < HPW; ++h) dst[h * p.t3] = __uint_as_float(o[h]);
         }
         if (!(ok = wg_sync())) break;      // sum_s is free again before the next segment's flush writes it
       }
