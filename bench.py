@@ -41,8 +41,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on
 # this workload (profiles/).  A value is only listed while the kernel is unchanged since its capture.
 NCU_TRAFFIC_BYTES = {
-    "c4_long_prefill": 17.91e6 + 78.09e6,     # attn::k_attn_prefill, profiles/k_attn_prefill_c4_long_prefill.md
-    "c3_vit_prefill": 34.14e6 + 65.40e6,      # attn::k_attn_prefill, profiles/k_attn_prefill_c3_vit_prefill.md
+    "c4_long_prefill": 17.99e6 + 77.25e6,     # attn::k_attn_prefill, profiles/k_attn_prefill_c4_long_prefill.md
+    "c3_vit_prefill": 34.02e6 + 64.90e6,      # attn::k_attn_prefill, profiles/k_attn_prefill_c3_vit_prefill.md
     "c5_decode": 1075.34e6 + 4.56e6,          # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_c5_decode.md
     "f1_decode_shared_kv": 538.05e6 + 4.87e6,  # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_f1_decode_shared_kv.md
 }
