@@ -262,6 +262,30 @@ def test_decode_tensor_core_path(case, append, flags):
         assert np.array_equal(Kh[b], Kc[b].astype(np.float32)) and np.array_equal(Vh[b], Vc[b].astype(np.float32))
 
 
+@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
+def test_decode_growing_scores_exercise_the_rescaling(flags):
+    # Cached keys whose norm grows along the sequence and a pre-softmax core scaled by 8: the running maximum
+    # of most heads rises by far more than the lazy-rescale threshold from tile to tile, so the accumulated
+    # outputs and row sums are rescaled again and again (the random caches of the other tests almost never
+    # move the maximum after the first tile).
+    import torch
+    w = H.custom_workload(kind="decode", dtype="bf16", d_model=256, n_H=32, r=(8, 64, 128), t=(8, 64, 128), rope=True,
+                          rope_base=500000.0, seed=29)
+    lens, Lmax = [1500, 700, 129, 2047], 2048
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    wt["C"] = W.round_to_storage(wt["C"] * 8.0, w.dtype)
+    x, Kc, Vc, cache_len = W.make_decode_state(w, B=len(lens), L=max(lens), Lmax=Lmax, cache_len=lens)
+    ramp = (1.0 + 3.0 * np.arange(Lmax) / Lmax).astype(np.float32)[None, :, None]
+    x, Kc, Vc = (W.round_to_storage(a, w.dtype) for a in (x, Kc * ramp, Vc))
+    ref, _, _ = O.tucker_attn_decode(x, *[wt[k] for k in H.WEIGHT_KEYS], Kc, Vc, cache_len, rope=True,
+                                     rope_base=w.rope_base)
+    y = Bd.tucker_attn_decode(H.to_device(x, w.dtype), *H.weights_to_device(wt, w.dtype), H.to_device(Kc, w.dtype),
+                              H.to_device(Vc, w.dtype), torch.from_numpy(cache_len).cuda(), n_H=w.n_H, rope=True,
+                              rope_base=w.rope_base, append=True, flags=flags)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == 2
+    check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "decode, growing scores", scaled=True)
+
+
 # --------------------------------------------------------------------------------------
 # shared key / value projection and cache (Sec. 3.1: K, V replaced by L^KV = X U3), no RoPE
 # --------------------------------------------------------------------------------------
