@@ -234,6 +234,19 @@ enum {
 };
 TA_API int tucker_attn_last_device_error(void* cuda_stream);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Launches a one-block kernel
+ * in which one thread waits on a barrier that nothing ever signals, with a wait budget of
+ * about `budget_us` microseconds (1 .. 100000), and a second thread waits on another such
+ * barrier with the library's normal budget.  The first wait must give up and set
+ * TA_DEVERR_WAIT_TIMEOUT in the device error word; the second must return at once through
+ * the block's abort flag.  `out` is caller-owned device memory for three int32: what the
+ * two waits returned (0 = gave up) and the second wait's duration in units of 1024 cycles.
+ * Asynchronous on `cuda_stream`; the context stays usable.  Returns TA_OK,
+ * TA_ERR_INVALID_ARG or TA_ERR_CUDA.
+ */
+TA_API int tucker_attn_selftest_wait_timeout(int32_t budget_us, int32_t* out, void* cuda_stream);
+
 /* Which path the last tucker_attn_fwd / tucker_attn_decode call on this thread took:
  * 0 = none yet, 1 = generic FMA kernels, 2 = tensor-core kernels.  Number of kernels that
  * call launched. */

@@ -25,7 +25,8 @@ EXPORTS = (
     "tucker_attn_fwd_workspace_bytes", "tucker_attn_decode_workspace_bytes", "tucker_attn_fwd",
     "tucker_attn_decode", "tucker_attn_status_string", "tucker_attn_last_device_error",
     "tucker_attn_last_path", "tucker_attn_last_launch_count", "tucker_attn_set_profile_events",
-    "tucker_attn_decode_static",
+    "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout",
+    "tucker_pack_gqa", "tucker_pack_mha", "tucker_pack_mla",
 )
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -81,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_attn_last_launch_count.restype = ctypes.c_int
     lib.tucker_attn_set_profile_events.restype = ctypes.c_int
     lib.tucker_attn_set_profile_events.argtypes = [vp, vp]
+    lib.tucker_attn_selftest_wait_timeout.restype = ctypes.c_int
+    lib.tucker_attn_selftest_wait_timeout.argtypes = [i32, vp, vp]
     lib.tucker_pack_gqa.restype = ctypes.c_int
     lib.tucker_pack_gqa.argtypes = [i32] * 4 + [vp] * 13
     lib.tucker_pack_mha.restype = ctypes.c_int
@@ -357,6 +360,19 @@ def tucker_pack_mla(WDQ, WUQ, WDKV, WUK, WDV, WUV, WO, *, n_H: int, out=None):
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_pack_mla")
     return outs
+
+
+def selftest_wait_timeout(budget_us: int = 2000, device=None):
+    """Runs the library's bounded-wait self-test; returns the int32 tensor [first wait returned,
+    second wait returned, second wait's duration / 1024 cycles] (read it after synchronising)."""
+    torch = _torch()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    out = torch.full((3,), -1, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = load_library().tucker_attn_selftest_wait_timeout(int(budget_us), out.data_ptr(), _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_attn_selftest_wait_timeout")
+    return out
 
 
 def last_device_error(device=None) -> int:

@@ -168,6 +168,13 @@ int tucker_attn_last_device_error(void* cuda_stream) {
   return (int)host;
 }
 
+int tucker_attn_selftest_wait_timeout(int32_t budget_us, int32_t* out, void* cuda_stream) {
+  if (budget_us <= 0 || budget_us > 100000 || !out) return TA_ERR_INVALID_ARG;
+  unsigned int* ptr = device_error_ptr();
+  if (!ptr) return TA_ERR_CUDA;
+  return wait_selftest(ptr, budget_us, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int tucker_attn_set_profile_events(void* ev_start, void* ev_stop) {
   if ((ev_start == nullptr) != (ev_stop == nullptr)) return TA_ERR_INVALID_ARG;
   tl_prof_start = static_cast<cudaEvent_t>(ev_start);

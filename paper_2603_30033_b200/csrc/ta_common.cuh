@@ -68,6 +68,7 @@ int fast_fwd(Problem& p);
 bool fast_decode_supported(const tucker_attn_desc& d, int32_t Lmax);
 size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
 int fast_decode(Problem& p);
+int wait_selftest(unsigned int* dev_err, int budget_us, int* out_dev, cudaStream_t stream);
 
 // Programmatic dependent launch.  Every kernel of the tensor-core paths starts with pdl_enter():
 // it waits until the preceding kernels of the stream have completed and their writes are visible,

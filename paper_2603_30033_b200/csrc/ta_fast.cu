@@ -685,3 +685,36 @@ int fast_decode(Problem& p) {
 }
 
 }  // namespace ta
+
+// ---- self-test of the bounded waits -------------------------------------------------------
+namespace ta {
+namespace {
+// One CTA, two warps.  Lane 0 of warp 0 waits on an mbarrier that nothing ever arrives on; its wait gives up
+// after `budget_cycles`, raises the CTA's abort flag and sets the device error word.  Lane 0 of warp 1 waits
+// on a second such barrier with the full budget and must come back through the abort flag.  out[0] / out[1]
+// receive what the two waits returned (0 = gave up), out[2] the cycles the second wait took.
+__global__ void k_wait_selftest(unsigned int* err, long long budget_cycles, int* out) {
+  __shared__ uint64_t bar[2];
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    sm100::mbar_init(&bar[0], 1);
+    sm100::mbar_init(&bar[1], 1);
+    sm100::fence_barrier_init();
+  }
+  __syncthreads();
+  sm100::Abort ab{&abort_flag, err};
+  if (threadIdx.x == 0) out[0] = sm100::mbar_wait(&bar[0], 0, ab, budget_cycles) ? 1 : 0;
+  if (threadIdx.x == 32) {
+    const long long t0 = clock64();
+    out[1] = sm100::mbar_wait(&bar[1], 0, ab) ? 1 : 0;
+    out[2] = (int)((clock64() - t0) >> 10);
+  }
+}
+}  // namespace
+int wait_selftest(unsigned int* dev_err, int budget_us, int* out_dev, cudaStream_t stream) {
+  const long long cycles = (long long)budget_us * 2000LL;      // about 2 GHz
+  k_wait_selftest<<<1, 64, 0, stream>>>(dev_err, cycles, out_dev);
+  return cudaGetLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+}
+}  // namespace ta

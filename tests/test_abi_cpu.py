@@ -20,7 +20,7 @@ def lib():
 
 def test_exports_match_header(lib):
     text = open(os.path.join(ROOT, "include", "tucker_attn.h")).read()
-    declared = re.findall(r"TA_API[^;(]*?\b(tucker_attn_\w+)\s*\(", text)
+    declared = re.findall(r"TA_API[^;(]*?\b(tucker_\w+)\s*\(", text)
     assert sorted(declared) == sorted(Bd.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name

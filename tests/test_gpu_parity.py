@@ -403,6 +403,24 @@ def test_decode_bad_cache_len_is_flagged_not_fatal():
     assert Bd.last_device_error() == 0                                 # cleared by the read
 
 
+def test_a_wait_that_nothing_ends_gives_up_and_is_reported():
+    # The kernels' waits are bounded: one that runs out sets TA_DEVERR_WAIT_TIMEOUT and every other wait of
+    # the block returns through the abort flag.  The library's self-test kernel does exactly that with a
+    # 2 ms budget (a barrier that nothing signals); the context must stay usable afterwards.
+    import torch
+    assert Bd.last_device_error() == 0
+    out = Bd.selftest_wait_timeout(2000)
+    err = Bd.last_device_error()                       # synchronises the stream
+    assert err == Bd.TA_DEVERR_WAIT_TIMEOUT
+    first, second, cycles_k = out.cpu().tolist()
+    assert first == 0 and second == 0                  # both waits gave up ...
+    assert cycles_k < (50_000_000 >> 10)               # ... the second long before its own two-second budget
+    assert Bd.last_device_error() == 0                 # the word is cleared by the read
+    w = W.get_workload("c1")                           # and ordinary calls still work
+    X, wt = H.host_inputs(w)
+    check(gpu_fwd(X, wt, w), oracle_fwd(X, wt, w), "fp32", "c1 after the self-test")
+
+
 # --------------------------------------------------------------------------------------
 # benchmark-sized workloads, sampled
 # --------------------------------------------------------------------------------------
