@@ -25,7 +25,13 @@ into Tucker form (Lemma 1, Theorems 1-3), used to pin the evaluators against eac
 Pins (see tests/test_oracle_pins.py): brute force == fast path; MHA / GQA / MQA / MLA
 reductions; MQA with standard RoPE in d_H == Tucker with latent RoPE when r3 = d_H;
 position-offset invariance; softmax rows sum to one; permutation equivariance; causality;
-decode == last row of prefill; printed parameter / cache sizes of the paper's tables.
+decode == last row of prefill; printed parameter / cache sizes of the paper's tables
+(separated and shared K,V); MLA with RoPE in its key latent (Sec. 3.2.1), written with
+explicit rotation matrices, == the Tucker evaluator with latent RoPE on the MLA embedding and
+== single-head MHA with standard RoPE when there is one head and no up-projection; shared
+latent cache with latent RoPE == the two-cache decode on (rotated, un-rotated) copies; HOSVD:
+exact recovery of an exact-rank tensor, orthonormal factors, the truncation error bound,
+full-rank round trip of MHA weights, spectra == numpy's singular values of the unfoldings.
 Parity unpinned: the paper prints no numeric forward-pass example, so absolute outputs are
 pinned only through these identities.
 """
@@ -84,6 +90,18 @@ def rope_rotate(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
     out[..., 0::2] = xe * c - xo * s
     out[..., 1::2] = xe * s + xo * c
     return out
+
+
+def rope_matrix(pos: float, r: int, base: float) -> np.ndarray:
+    """The dense r x r rotation R(pos, r) itself (row-vector convention x' = x R): 2 x 2 blocks
+    [[cos, sin], [-sin, cos]] on coordinate pairs (2i, 2i+1), angle pos * base**(-2i/r).
+    Written entry by entry so that it shares nothing with rope_rotate."""
+    R = np.zeros((r, r), F64)
+    for i in range(r // 2):
+        a = float(pos) * float(base) ** (-2.0 * i / r)
+        R[2 * i, 2 * i], R[2 * i, 2 * i + 1] = np.cos(a), np.sin(a)
+        R[2 * i + 1, 2 * i], R[2 * i + 1, 2 * i + 1] = -np.sin(a), np.cos(a)
+    return R
 
 
 # ----------------------------------------------------------------------------------------
@@ -387,3 +405,126 @@ def gqa_param_count(d, n_H, n_G) -> int:
 
 def gqa_kv_cache_elems(N, d, n_H, n_G) -> int:
     return 2 * N * n_G * (d // n_H)
+
+
+# ----------------------------------------------------------------------------------------
+# Shared latent cache with latent RoPE (Sec. 3.1, last paragraph, together with Definition 2)
+# ----------------------------------------------------------------------------------------
+
+def tucker_attn_decode_shared_rope(x, C, U1, U2, U3, Ct, Ut1, Ut2, Lc, cache_len, *,
+                                   rope_base=10000.0, scale=None):
+    """Cached decode step with ONE latent cache L^KV = X U3 (Sec. 3.1: keys and values replaced by
+    the shared down-projection, cache size N r3) and latent RoPE (Definition 2).  The paper does
+    not say what the single cache holds when the keys are rotated; reading taken here: the cache
+    holds the UN-rotated latent rows, the value side uses them as they are, and the key of slot n
+    is the cached row times R(n, r3), formed when it is used.  Lc [B, Lmax, r3]; the new token at
+    position L = cache_len[b] attends to slots 0..L-1 and to itself.
+    Returns (y [B, d], l_new [B, r3] un-rotated latent row of the new token)."""
+    x = np.asarray(x, F64)
+    B, d = x.shape
+    U1, U2, U3 = (np.asarray(a, F64) for a in (U1, U2, U3))
+    Ut1, Ut2 = np.asarray(Ut1, F64), np.asarray(Ut2, F64)
+    n_H = U1.shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(d / n_H)
+    G = head_cores(C, U1)
+    Gt = head_cores(Ct, Ut1)
+    y = np.empty((B, d), F64)
+    l_new = np.empty((B, U3.shape[1]), F64)
+    for b in range(B):
+        L = int(cache_len[b])
+        lat = np.concatenate([np.asarray(Lc[b, :L], F64), x[b:b + 1] @ U3], axis=0)   # [L+1, r3] = V
+        K = rope_rotate(lat, np.arange(L + 1), rope_base)
+        qt = x[b:b + 1] @ U2
+        z = np.zeros((1, Ut2.shape[1]), F64)
+        for h in range(n_H):
+            qh = rope_rotate(qt @ G[h], np.array([L]), rope_base)
+            p = softmax_rows((qh @ K.T) * scale)
+            z += (p @ lat) @ Gt[h].T
+        y[b] = (z @ Ut2.T)[0]
+        l_new[b] = lat[L]
+    return y, l_new
+
+
+# ----------------------------------------------------------------------------------------
+# MLA with RoPE in its key latent (Sec. 3.2.1 "Simplified RoPE for MLA"; App. C.2 "MLA - coupled RoPE")
+# ----------------------------------------------------------------------------------------
+
+def mla_latent_rope_reference(X, WDQ, WUQ, WDKV, WUK, WDV, WUV, WO, n_H, *, causal=False,
+                              rope_base=10000.0, pos0=0):
+    """One sequence X [N, d].  Per head i the query-side matrices are fused into
+    WQ_i^MLA = WDQ WUQ_i WUK_i^T  [d, dcK]  (the paper prints W^UV_i for the last factor; the
+    key up-projection transposed is what makes the product land in the key latent), and
+        score_i[m, n] = X_m WQ_i^MLA R(m, dcK) R(n, dcK)^T WDKV^T X_n^T / sqrt(d_H);
+    values and output as in MLA without RoPE: V_i = X WDV WUV_i, out = sum_i P_i V_i WO_i.
+    Rotations are applied as explicit dense matrices, position by position."""
+    X = np.asarray(X, F64)
+    N, d = X.shape
+    d_H = d // n_H
+    dck = WDKV.shape[1]
+    Rm = [rope_matrix(pos0 + m, dck, rope_base) for m in range(N)]
+    Krot = np.stack([(X[n] @ WDKV) @ Rm[n] for n in range(N)])              # [N, dcK]
+    cv = X @ WDV
+    out = np.zeros((N, d), F64)
+    for i in range(n_H):
+        sl = slice(i * d_H, (i + 1) * d_H)
+        WQmla = WDQ @ WUQ[:, sl] @ WUK[:, sl].T                             # [d, dcK]
+        Qrot = np.stack([(X[m] @ WQmla) @ Rm[m] for m in range(N)])
+        S = (Qrot @ Krot.T) / np.sqrt(d_H)
+        if causal:
+            pos = np.arange(N)
+            S = np.where(causal_mask(pos, pos), -np.inf, S)
+        out += softmax_rows(S) @ (cv @ WUV[:, sl]) @ WO[sl, :]
+    return out
+
+
+# ----------------------------------------------------------------------------------------
+# HOSVD initialiser (App. C.1 "MHA to Tucker Attention"; Sec. 2.1 "Informed Compression Across All Modes")
+# ----------------------------------------------------------------------------------------
+
+def mode_unfold(T: np.ndarray, mode: int) -> np.ndarray:
+    """Mat_mode(T): the mode-`mode` fibres of a 3-way tensor as columns, [I_mode, prod of the others]."""
+    ax = mode - 1
+    return np.moveaxis(np.asarray(T, F64), ax, 0).reshape(T.shape[ax], -1)
+
+
+def mode_spectrum(T: np.ndarray, mode: int) -> np.ndarray:
+    """Singular values of Mat_mode(T) divided by the largest (the normalised per-mode spectrum
+    that Sec. 2.1 plots to choose the ranks)."""
+    s = np.linalg.svd(mode_unfold(T, mode), compute_uv=False)
+    return s / s[0]
+
+
+def hosvd(T: np.ndarray, ranks) -> tuple:
+    """Truncated higher-order SVD: factor j = the ranks[j] leading left singular vectors of
+    Mat_j(T); core = T x_1 U1^T x_2 U2^T x_3 U3^T.  Returns (core, [U1, U2, U3], [s1, s2, s3])
+    with s_j all singular values of Mat_j(T).  T is approximated by core x_1 U1 x_2 U2 x_3 U3 with
+    ||T - approx||^2 <= sum_j sum_{k >= ranks[j]} s_j[k]^2."""
+    T = np.asarray(T, F64)
+    Us, svals = [], []
+    for mode in (1, 2, 3):
+        U, s, _ = np.linalg.svd(mode_unfold(T, mode), full_matrices=False)
+        Us.append(U[:, :ranks[mode - 1]])
+        svals.append(s)
+    core = T
+    for mode in (1, 2, 3):
+        core = mode_product(core, Us[mode - 1].T, mode)
+    return core, Us, svals
+
+
+def mha_weight_tensors(WQ, WK, WV, WO, n_H) -> tuple:
+    """The two n_H x d x d tensors of Eqs. 2-3: W[i] = WQ_i WK_i^T and the transposed stack
+    Wt[i] = (WV_i WO_i)^T (mode 2 = output, mode 3 = value)."""
+    d = WQ.shape[0]
+    d_H = d // n_H
+    W = np.stack([WQ[:, i * d_H:(i + 1) * d_H] @ WK[:, i * d_H:(i + 1) * d_H].T for i in range(n_H)])
+    Wt = np.stack([(WV[:, i * d_H:(i + 1) * d_H] @ WO[i * d_H:(i + 1) * d_H, :]).T for i in range(n_H)])
+    return W.astype(F64), Wt.astype(F64)
+
+
+def mha_to_tucker(WQ, WK, WV, WO, n_H, r, t) -> dict:
+    """MHA weights -> Tucker-attention weights by HOSVD of the two weight tensors (App. C.1)."""
+    W, Wt = mha_weight_tensors(np.asarray(WQ, F64), np.asarray(WK, F64), np.asarray(WV, F64), np.asarray(WO, F64), n_H)
+    C, (U1, U2, U3), sv = hosvd(W, r)
+    Ct, (Ut1, Ut2, Ut3), svt = hosvd(Wt, t)
+    return dict(C=C, U1=U1, U2=U2, U3=U3, Ct=Ct, Ut1=Ut1, Ut2=Ut2, Ut3=Ut3, spectra=sv, spectra_t=svt)

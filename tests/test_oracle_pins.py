@@ -391,6 +391,18 @@ def test_printed_sizes():
         "llama_mha_params_M": O.mha_param_count(d) * layers / MB,
         "llama_gqa8_cache_M": O.gqa_kv_cache_elems(N, d, nH, 8) * layers / MB,
     })
+    # Shakespeare ablation table: shared and separated K,V; parameters in 10^6 bytes, caches in 2^20 bytes
+    layers, d, nH, N, MiB = 12, 768, 12, 256, float(1 << 20)
+    for r1, r in ((8, 128), (8, 64), (6, 64), (4, 32)):
+        got[f"shake_tucker_shared_{r1}_{r}_{r}_params_MB"] = O.tucker_param_count(d, nH, r1, r, shared_kv=True) * layers * 2 / MB
+    for r1, r in ((8, 128), (6, 32)):
+        got[f"shake_tucker_sep_{r1}_{r}_{r}_params_MB"] = O.tucker_param_count(d, nH, r1, r) * layers * 2 / MB
+    for r in (128, 64, 32):
+        got[f"shake_tucker_shared_r{r}_cache_MiB"] = O.tucker_kv_cache_elems(N, r, shared_kv=True) * layers * 2 / MiB
+    for r in (128, 64):
+        got[f"shake_tucker_sep_r{r}_cache_MiB"] = O.tucker_kv_cache_elems(N, r) * layers * 2 / MiB
+    got["shake_mha_cache_MiB"] = O.gqa_kv_cache_elems(N, d, nH, nH) * layers * 2 / MiB
+    got["shake_gqa1_cache_MiB"] = O.gqa_kv_cache_elems(N, d, nH, 1) * layers * 2 / MiB
     assert set(got) == set(g)
     for k, (val, tol) in g.items():
         assert abs(got[k] - val) <= tol, (k, got[k], val)
