@@ -57,7 +57,8 @@ typedef enum {
   TA_ERR_UNSUPPORTED_SHAPE = -2,   /* a rank or size outside what the kernels were built for */
   TA_ERR_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < tucker_attn_*_workspace_bytes(...) */
   TA_ERR_CUDA = -4,                /* a CUDA runtime / driver call failed (launch, tensor map) */
-  TA_ERR_DEVICE_TIMEOUT = -5       /* a bounded device-side wait gave up (see tucker_attn_last_device_error) */
+  TA_ERR_DEVICE_TIMEOUT = -5       /* a bounded device-side wait gave up; returned by tucker_attn_sync_status only
+                                      (the launching call itself is asynchronous and has returned TA_OK by then) */
 } tucker_attn_status;
 
 enum { TA_DTYPE_F32 = 0, TA_DTYPE_BF16 = 1 };
@@ -85,8 +86,7 @@ enum {
    * the routes can be checked against each other: */
   TA_FLAG_FMA_ATTENTION = 0x200,      /* tensor-core GEMMs, but the attention itself on the FMA kernel */
   TA_FLAG_SEPARATE_QUERIES = 0x400,   /* per-head queries from a separate GEMM instead of the attention prologue */
-  TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x800, /* Z and Y from two GEMM launches instead of the fused output kernel */
-  TA_FLAG_MMA_SYNC_DECODE = 0x1000     /* decode: the mma.sync form of the cache-streaming kernel instead of the tcgen05 one */
+  TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x800  /* Z and Y from two GEMM launches instead of the fused output kernel */
 };
 
 /* Bytes of scratch the corresponding call needs for this descriptor (0 on invalid descriptor). */
@@ -222,17 +222,37 @@ TA_API int tucker_pack_mla(int32_t d_model, int32_t n_H, int32_t dcq, int32_t dc
 TA_API const char* tucker_attn_status_string(int status);
 
 /*
- * Device error word.  Kernels never trap: a bounded wait that ran out or an index that
- * failed a bounds check sets a bit in a per-device word and the kernel returns.  This call
+ * Device error word.  Kernels never trap: a bounded wait that ran out, an out-of-range cache length or (in
+ * the checking build) an index that failed its bounds check sets a bit in a per-device word and the kernel
+ * carries on without the offending access, or returns.  This call
  * synchronises `cuda_stream`, reads and clears the word of the current device and returns
  * it (0 = clean; otherwise a bit set of TA_DEVERR_*), or a negative status on CUDA errors.
  */
 enum {
   TA_DEVERR_WAIT_TIMEOUT = 1,   /* an mbarrier / flag wait hit its iteration limit */
   TA_DEVERR_BAD_CACHE_LEN = 2,  /* cache_len[b] outside [0, Lmax) */
-  TA_DEVERR_BAD_INDEX = 4       /* an internal bounds check failed */
+  TA_DEVERR_BAD_INDEX = 4       /* a bounds check failed (only in the -DTA_BOUNDS_CHECK build, see tucker_attn_bounds_checked) */
 };
 TA_API int tucker_attn_last_device_error(void* cuda_stream);
+
+/*
+ * The same read, folded into a status code for callers that only want to know whether the work queued so
+ * far went through (no counterpart in the paper).  Synchronises `cuda_stream`, reads and clears the device
+ * error word and returns TA_OK when it was clean, else TA_ERR_DEVICE_TIMEOUT (a bounded wait gave up: results
+ * of the calls since the last read are invalid), TA_ERR_INVALID_ARG (a cache_len entry was out of range and
+ * was clamped) or TA_ERR_CUDA (the read itself failed, or a bounds check of the checking build fired), in
+ * that order of precedence.
+ */
+TA_API int tucker_attn_sync_status(void* cuda_stream);
+
+/*
+ * 1 when this library was compiled with -DTA_BOUNDS_CHECK, 0 otherwise.  In that build the kernels of the
+ * tensor-core paths and of the decode step compare every global index they form for a store (outputs, caches,
+ * workspace regions) and for a load from the workspace with the extent of the tensor addressed, set
+ * TA_DEVERR_BAD_INDEX and skip the access on a failure; nothing traps.  TMA transfers are bounded by their
+ * tensor maps in either build.  The normal build carries no such checks and never sets that bit.
+ */
+TA_API int tucker_attn_bounds_checked(void);
 
 /*
  * Self-test of the bounded waits (no counterpart in the paper).  Launches a one-block kernel

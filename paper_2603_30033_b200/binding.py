@@ -12,20 +12,23 @@ import os
 from typing import Optional
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtucker_attn.so")
+# TUCKER_ATTN_LIB=checked selects the twin built with -DTA_BOUNDS_CHECK (device-side range checks on every
+# global index, reported through the device error word); anything else, or nothing, the normal library.
+LIB_PATH = os.path.join(_HERE, "libtucker_attn_checked.so" if os.environ.get("TUCKER_ATTN_LIB") == "checked"
+                        else "libtucker_attn.so")
 
 TA_OK = 0
 TA_DTYPE_F32, TA_DTYPE_BF16 = 0, 1
 TA_FLAG_FORCE_GENERIC = 1
 TA_FLAG_FMA_ATTENTION, TA_FLAG_SEPARATE_QUERIES, TA_FLAG_SEPARATE_OUTPUT_GEMMS = 0x200, 0x400, 0x800
-TA_FLAG_MMA_SYNC_DECODE = 0x1000
 TA_DEVERR_WAIT_TIMEOUT, TA_DEVERR_BAD_CACHE_LEN, TA_DEVERR_BAD_INDEX = 1, 2, 4
 
 EXPORTS = (
     "tucker_attn_fwd_workspace_bytes", "tucker_attn_decode_workspace_bytes", "tucker_attn_fwd",
     "tucker_attn_decode", "tucker_attn_status_string", "tucker_attn_last_device_error",
     "tucker_attn_last_path", "tucker_attn_last_launch_count", "tucker_attn_set_profile_events",
-    "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout",
+    "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout", "tucker_attn_sync_status",
+    "tucker_attn_bounds_checked",
     "tucker_pack_gqa", "tucker_pack_mha", "tucker_pack_mla",
 )
 TA_STATIC_SCRATCH_BYTES = 16 << 20
@@ -78,6 +81,9 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_attn_status_string.argtypes = [ctypes.c_int]
     lib.tucker_attn_last_device_error.restype = ctypes.c_int
     lib.tucker_attn_last_device_error.argtypes = [vp]
+    lib.tucker_attn_sync_status.restype = ctypes.c_int
+    lib.tucker_attn_sync_status.argtypes = [vp]
+    lib.tucker_attn_bounds_checked.restype = ctypes.c_int
     lib.tucker_attn_last_path.restype = ctypes.c_int
     lib.tucker_attn_last_launch_count.restype = ctypes.c_int
     lib.tucker_attn_set_profile_events.restype = ctypes.c_int
@@ -381,6 +387,20 @@ def last_device_error(device=None) -> int:
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
     with torch.cuda.device(dev):
         return int(load_library().tucker_attn_last_device_error(_stream_ptr(dev)))
+
+
+def sync_status(device=None) -> int:
+    """Synchronises the current stream and folds the device error word into a status code (and clears
+    it): TA_OK, or TA_ERR_DEVICE_TIMEOUT (-5) / TA_ERR_INVALID_ARG (-1) / TA_ERR_CUDA (-4)."""
+    torch = _torch()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    with torch.cuda.device(dev):
+        return int(load_library().tucker_attn_sync_status(_stream_ptr(dev)))
+
+
+def bounds_checked() -> bool:
+    """True when the loaded library was built with -DTA_BOUNDS_CHECK."""
+    return bool(load_library().tucker_attn_bounds_checked())
 
 
 def last_path() -> int:

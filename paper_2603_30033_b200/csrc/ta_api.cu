@@ -14,9 +14,11 @@ static thread_local cudaEvent_t tl_prof_stop = nullptr;
 
 static unsigned int* device_error_ptr() {
   // one address per device; looked up lazily, cached per device ordinal
-  static unsigned int* cache[64] = {nullptr};
+  static unsigned int* cache[kMaxDevices] = {nullptr};
+  static std::mutex m;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(m);
   if (!cache[dev]) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_device_error_word) != cudaSuccess) return nullptr;
@@ -166,6 +168,23 @@ int tucker_attn_last_device_error(void* cuda_stream) {
   if (cudaMemsetAsync(ptr, 0, sizeof(host), s) != cudaSuccess) return TA_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return TA_ERR_CUDA;
   return (int)host;
+}
+
+int tucker_attn_sync_status(void* cuda_stream) {
+  const int word = tucker_attn_last_device_error(cuda_stream);
+  if (word < 0) return word;
+  if (word & TA_DEVERR_WAIT_TIMEOUT) return TA_ERR_DEVICE_TIMEOUT;
+  if (word & TA_DEVERR_BAD_CACHE_LEN) return TA_ERR_INVALID_ARG;
+  if (word & TA_DEVERR_BAD_INDEX) return TA_ERR_CUDA;
+  return TA_OK;
+}
+
+int tucker_attn_bounds_checked(void) {
+#ifdef TA_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 int tucker_attn_selftest_wait_timeout(int32_t budget_us, int32_t* out, void* cuda_stream) {

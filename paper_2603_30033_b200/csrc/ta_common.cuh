@@ -7,6 +7,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "tucker_attn.h"
 
 namespace ta {
@@ -98,6 +100,41 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+
+// Per-device one-time set-up.  A kernel's dynamic shared-memory limit and the device properties are per
+// device, and one process may drive several GPUs, so each is recorded per device ordinal under a mutex.
+constexpr int kMaxDevices = 64;
+struct PerDeviceFlag {
+  std::mutex m;
+  bool done[kMaxDevices] = {};
+};
+// Raises `func`'s dynamic shared-memory limit to `bytes` on the current device, once per device.
+static inline cudaError_t ensure_dynamic_smem(PerDeviceFlag& f, const void* func, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(f.m);
+  if (f.done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) f.done[dev] = true;
+  return e;
+}
+
+// Debug build (-DTA_BOUNDS_CHECK): every global index that the tensor-core kernels and the decode kernels
+// form for a store, and for a load from the workspace, is compared with the extent of the tensor it
+// addresses before it is used.  A failure sets TA_DEVERR_BAD_INDEX in the device error word and the access
+// is skipped; nothing traps.  In the normal build the macro is the constant `true`.
+#if defined(__CUDACC__) && defined(TA_BOUNDS_CHECK)
+__device__ __forceinline__ bool index_in_bounds(unsigned int* err, long first, long count, long extent) {
+  if (first >= 0 && count >= 0 && first + count <= extent) return true;
+  if (err) atomicOr(err, (unsigned)TA_DEVERR_BAD_INDEX);
+  return false;
+}
+#define TA_IDX_OK(err, first, count, extent) ::ta::index_in_bounds((err), (long)(first), (long)(count), (long)(extent))
+#else
+#define TA_IDX_OK(err, first, count, extent) true
+#endif
 
 #define TA_CUDA_TRY(expr)                          \
   do {                                             \

@@ -1,22 +1,12 @@
-// Decode step over the latent KV cache (Eq. 9, "KV Caching"): kernels of the bf16 path -- the query kernel
-// k_dec_qhat, the output kernel k_dec_out, and k_dec_attn, the mma.sync form of the cache-streaming kernel
-// (the tcgen05 form in ta_decode_umma.cuh is the one used unless TA_FLAG_MMA_SYNC_DECODE asks for this one;
-// both share the tile split, the helpers below and the partial format).
+// Decode step over the latent KV cache (Eq. 9, "KV Caching"): the per-sequence kernels of the bf16 path --
+// the query kernel k_dec_qhat and the output kernel k_dec_out -- and what they share with the
+// cache-streaming kernel (ta_decode_umma.cuh): the tile split, the RoPE angle helpers, the partial format.
 //
-// k_dec_attn streams every sequence's latent K / V cache exactly once.  The cache is cut into
-// tiles of 128 keys; the flat list of tiles of all sequences is divided evenly over the CTAs
-// (one per SM), so that the load is balanced for any mix of cache lengths.  Each CTA walks its
-// tile range, keeps an online-softmax state per sequence segment, and writes one partial
-// (max, sum, unnormalised O for all heads) per segment; k_dec_out combines the partials of
-// a sequence with log-sum-exp weights and applies the output-side core (Z = sum_h o_h Gt_h^T).
-//
-// All n_H (<= 32) heads share each K / V byte, so the arithmetic is 2 * n_H flop per cached
-// element -- beyond plain FMA throughput at HBM speed.  The products therefore run on the
-// tensor cores with the heads as the M dimension (two m16 tiles) of mma.sync m16n8k16:
-//   warp (mt, kq), mt = head half, kq = 32-key quarter of the tile
-//   S[16 heads x 32 keys] = Qhat_mt K_q^T ; online softmax with quad shuffles ; O += P V_q
-// K / V tiles arrive by TMA (3-D tensor map, 128-byte swizzle, conflict-free ldmatrix) through
-// a 3-stage ring fed by a dedicated producer warp.
+// The cache is cut into tiles of 128 keys; the flat list of tiles of all sequences is divided evenly
+// over the CTAs of the streaming kernel (one per SM), so that the load is balanced for any mix of
+// cache lengths.  Each of those CTAs keeps an online-softmax state per sequence segment and writes one
+// partial (max, sum, unnormalised O for all heads) per segment; k_dec_out combines the partials of a
+// sequence with log-sum-exp weights and applies the output-side core (Z = sum_h o_h Gt_h^T).
 #pragma once
 
 #include "ta_common.cuh"
@@ -28,13 +18,6 @@ namespace dec {
 using namespace sm100;
 
 constexpr int TK = 128;                 // keys per tile
-constexpr int CONSUMER_WARPS = 8;
-constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
-constexpr int STAGES = 3;
-constexpr int SUB_BYTES = 128 * 64 * 2;
-constexpr int MAX_SUB = 2;              // r3, t3 <= 128
-constexpr int STAGE_BYTES = 2 * MAX_SUB * SUB_BYTES;   // K tile + V tile
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES;
 constexpr int MAX_GRID = 160;           // partial weights table in the merge kernel
 
 struct Params {
@@ -120,325 +103,6 @@ __device__ __forceinline__ float2 rope_cos_sin(int pos, int i, int r, double log
   return make_float2(co, sn);
 }
 
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-      "{%0, %1, %2, %3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-// Byte offset of (row, 16-byte chunk) inside a tile made of [128 x 64] sub-tiles with 128-byte swizzle.
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-  return (uint32_t)((chunk >> 3) * SUB_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
-template <int R3, int T3>
-__global__ void __launch_bounds__(THREADS, 1)
-k_dec_attn(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
-  // The cached rows below cache_len and cache_len itself were final before the preceding kernel (which
-  // forms the queries and appends the new row) began, so the tile split and the first ring loads run
-  // while it finishes; pdl_enter() comes before anything that kernel writes is read.  The new row's
-  // slot may be read half-written: it is replaced from the workspace below in any case.
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES];
-  __shared__ int abort_flag;
-  __shared__ float ml_s[CONSUMER_WARPS][16][2];
-  __shared__ __align__(16) float obuf[32 * T3];
-
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  Abort ab{&abort_flag, p.err};
-  constexpr int KSUB = (R3 + 63) / 64, VSUB = (T3 + 63) / 64;
-
-  if (threadIdx.x == 0) {
-    abort_flag = 0;
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], CONSUMER_WARPS);
-    }
-    fence_barrier_init();
-  }
-  __syncthreads();
-
-  // ---- this CTA's range of the flat tile list (block-wide scan over the sequences) ----
-  __shared__ long long wtot_s[THREADS / 32];
-  __shared__ int loc_b;
-  __shared__ long long loc_first;
-  int lo, hi;
-  long excl;
-  const long total = block_tile_scan(p.cache_len, p.B, p.Lmax, lo, hi, excl, wtot_s);
-  const long t_begin = cta_first_tile(blockIdx.x, total, gridDim.x);
-  const long t_end = cta_first_tile(blockIdx.x + 1, total, gridDim.x);
-  {
-    // the thread whose sequences contain tile t_begin publishes that sequence and its first tile
-    long f = excl;
-    for (int b = lo; b < hi; ++b) {
-      const long nt = tiles_of(clamp_len(p.cache_len[b], p.Lmax));
-      if (t_begin >= f && t_begin < f + nt) { loc_b = b; loc_first = f; }
-      f += nt;
-    }
-  }
-  __syncthreads();
-  const int b0 = (t_begin < t_end) ? loc_b : 0;
-  const long seq_first = (t_begin < t_end) ? (long)loc_first : 0;   // global index of the first tile of sequence b0
-
-  if (warp == CONSUMER_WARPS) {
-    // ------------------------------- TMA producer -------------------------------
-    if (elect_one() && t_begin < t_end) {
-      tma_prefetch_desc(&tmK);
-      tma_prefetch_desc(&tmV);
-      int b = b0;
-      long first = seq_first;
-      long nt = tiles_of(clamp_len(p.cache_len[b], p.Lmax));
-      int it = 0;
-      for (long t = t_begin; t < t_end; ++t, ++it) {
-        while (t >= first + nt) {
-          first += nt;
-          ++b;
-          nt = tiles_of(clamp_len(p.cache_len[b], p.Lmax));
-        }
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1, ab)) break;
-        mbar_expect_tx(&full_bar[s], (uint32_t)((KSUB + (p.shared_kv ? 0 : VSUB)) * SUB_BYTES));
-        uint8_t* kt = tiles + (size_t)s * STAGE_BYTES;
-        uint8_t* vt = kt + MAX_SUB * SUB_BYTES;
-        const int row = (int)(t - first) * TK;
-        for (int kk = 0; kk < KSUB; ++kk) tma_load_3d(kt + kk * SUB_BYTES, &tmK, &full_bar[s], kk * 64, row, b);
-        if (!p.shared_kv)
-          for (int kk = 0; kk < VSUB; ++kk) tma_load_3d(vt + kk * SUB_BYTES, &tmV, &full_bar[s], kk * 64, row, b);
-      }
-    }
-    pdl_enter();
-  } else if (t_begin < t_end) {
-    // ------------------------------- consumers ----------------------------------
-    pdl_enter();
-    const int mt = warp / 4, kq = warp % 4;
-    const int g = lane / 4, tq = lane % 4;
-    int b = b0;
-    long first = seq_first;
-    int it = 0;
-    bool ok = true;
-    long t = t_begin;
-    while (t < t_end && ok) {
-      // ---- one segment: tiles [t, seg_end) of sequence b ----
-      const int L = clamp_len(p.cache_len[b], p.Lmax);
-      const long nt = tiles_of(L);
-      const long seg_end = (first + nt < t_end) ? first + nt : t_end;
-      // Qhat fragments (A operand): rows = heads 16*mt + {g, g+8}
-      uint32_t qa[R3 / 16][4];
-      {
-        const int h_lo = 16 * mt + g, h_hi = h_lo + 8;
-        const bf16* q_lo = p.qhat + ((long)b * p.nH + h_lo) * R3;
-        const bf16* q_hi = p.qhat + ((long)b * p.nH + h_hi) * R3;
-#pragma unroll
-        for (int kb = 0; kb < R3 / 16; ++kb) {
-          const int c = kb * 16 + 2 * tq;
-          qa[kb][0] = h_lo < p.nH ? *reinterpret_cast<const uint32_t*>(q_lo + c) : 0u;
-          qa[kb][1] = h_hi < p.nH ? *reinterpret_cast<const uint32_t*>(q_hi + c) : 0u;
-          qa[kb][2] = h_lo < p.nH ? *reinterpret_cast<const uint32_t*>(q_lo + c + 8) : 0u;
-          qa[kb][3] = h_hi < p.nH ? *reinterpret_cast<const uint32_t*>(q_hi + c + 8) : 0u;
-        }
-      }
-      float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-      float o[T3 / 8][4];
-#pragma unroll
-      for (int n = 0; n < T3 / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-
-      for (; t < seg_end; ++t, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        ok = mbar_wait(&full_bar[s], ph, ab);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        uint8_t* kt = tiles + (size_t)s * STAGE_BYTES;
-        uint8_t* vt = p.shared_kv ? kt : kt + MAX_SUB * SUB_BYTES;   // shared latent cache: the K tile is the V tile
-        const int k0 = (int)(t - first) * TK;
-        const bool last_tile = (k0 + TK > L);        // contains the new token (index L) and possibly invalid rows
-        if (last_tile) {
-          // rows of this warp's quarter: patch the new token's row from the workspace, zero invalid V rows
-          const int rnew = L - k0;
-          for (int rr = 0; rr < 32; ++rr) {
-            const int r = kq * 32 + rr;
-            if (r == rnew) {
-              if (lane * 4 < R3) {
-                const uint2 kv = *reinterpret_cast<const uint2*>(p.knew + (long)b * R3 + lane * 4);
-                *reinterpret_cast<uint2*>(kt + swz(r, lane >> 1) + (lane & 1) * 8) = kv;
-              }
-              if (lane * 4 < T3) {
-                const uint2 vv = *reinterpret_cast<const uint2*>(p.vnew + (long)b * T3 + lane * 4);
-                *reinterpret_cast<uint2*>(vt + swz(r, lane >> 1) + (lane & 1) * 8) = vv;
-              }
-            } else if (r > rnew) {
-              if (lane * 4 < T3) *reinterpret_cast<uint2*>(vt + swz(r, lane >> 1) + (lane & 1) * 8) = make_uint2(0u, 0u);
-            }
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-        }
-        // ---- S = Qhat K^T for this warp's 32 keys ----
-        float sc[4][4];
-#pragma unroll
-        for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
-        const uint32_t kbase = smem_u32(kt), vbase = smem_u32(vt);
-        {
-          const int mi = lane >> 3, rl = lane & 7;
-#pragma unroll
-          for (int kb = 0; kb < R3 / 16; ++kb) {
-#pragma unroll
-            for (int np = 0; np < 2; ++np) {
-              const int row = kq * 32 + (np * 2 + (mi >> 1)) * 8 + rl;
-              const int chunk = kb * 2 + (mi & 1);
-              uint32_t r0, r1, r2, r3;
-              ldsm_x4(kbase + swz(row, chunk), r0, r1, r2, r3);
-              mma_bf16(sc[np * 2], qa[kb], r0, r1);
-              mma_bf16(sc[np * 2 + 1], qa[kb], r2, r3);
-            }
-          }
-        }
-        if (last_tile) {
-#pragma unroll
-          for (int n = 0; n < 4; ++n)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int key = k0 + kq * 32 + n * 8 + 2 * tq + (e & 1);
-              if (key > L) sc[n][e] = -INFINITY;
-            }
-        }
-        // ---- online softmax (rows g and g+8 of this head half) ----
-        float corr[2];
-        uint32_t pa[2][4];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          float mx = -INFINITY;
-#pragma unroll
-          for (int n = 0; n < 4; ++n) mx = fmaxf(mx, fmaxf(sc[n][2 * r], sc[n][2 * r + 1]));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-          const float m_new = fmaxf(m_run[r], mx);
-          const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-          corr[r] = ex2(m_run[r] - m_safe);      // 0 when nothing was visible before
-          m_run[r] = m_new;
-          float rs = 0.f;
-#pragma unroll
-          for (int n = 0; n < 4; ++n) {
-            sc[n][2 * r] = ex2(sc[n][2 * r] - m_safe);
-            sc[n][2 * r + 1] = ex2(sc[n][2 * r + 1] - m_safe);
-            rs += sc[n][2 * r] + sc[n][2 * r + 1];
-          }
-          l_run[r] = l_run[r] * corr[r] + rs;
-        }
-#pragma unroll
-        for (int kb2 = 0; kb2 < 2; ++kb2) {
-          pa[kb2][0] = pack_bf16(sc[2 * kb2][0], sc[2 * kb2][1]);
-          pa[kb2][1] = pack_bf16(sc[2 * kb2][2], sc[2 * kb2][3]);
-          pa[kb2][2] = pack_bf16(sc[2 * kb2 + 1][0], sc[2 * kb2 + 1][1]);
-          pa[kb2][3] = pack_bf16(sc[2 * kb2 + 1][2], sc[2 * kb2 + 1][3]);
-        }
-#pragma unroll
-        for (int n = 0; n < T3 / 8; ++n) {
-          o[n][0] *= corr[0]; o[n][1] *= corr[0];
-          o[n][2] *= corr[1]; o[n][3] *= corr[1];
-        }
-        // ---- O += P V for this warp's 32 keys ----
-        {
-          const int mi = lane >> 3, rl = lane & 7;
-#pragma unroll
-          for (int kb2 = 0; kb2 < 2; ++kb2) {
-            const int row = kq * 32 + kb2 * 16 + (mi & 1) * 8 + rl;
-#pragma unroll
-            for (int n = 0; n < T3 / 8; n += 2) {
-              uint32_t r0, r1, r2, r3;
-              ldsm_x4_t(vbase + swz(row, n + (mi >> 1)), r0, r1, r2, r3);
-              mma_bf16(o[n], pa[kb2], r0, r1);
-              mma_bf16(o[n + 1], pa[kb2], r2, r3);
-            }
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[s]);
-      }
-      if (!ok) break;
-      // ---- segment done: merge the four key-quarter warps of each head half, write the partial ----
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-      }
-      if (tq == 0) {
-        ml_s[warp][g][0] = m_run[0]; ml_s[warp][g][1] = l_run[0];
-      }
-      consumer_sync();
-      // (rows g+8 are exchanged in a second pass to keep the table small)
-      float Mx[2], Ls[2], own[2];
-      {
-        float M = -INFINITY;
-        for (int k = 0; k < 4; ++k) M = fmaxf(M, ml_s[mt * 4 + k][g][0]);
-        const float Ms = (M == -INFINITY) ? 0.f : M;
-        float Lsum = 0.f;
-        for (int k = 0; k < 4; ++k) Lsum += ml_s[mt * 4 + k][g][1] * ex2(ml_s[mt * 4 + k][g][0] - Ms);
-        Mx[0] = M; Ls[0] = Lsum; own[0] = ex2(m_run[0] - Ms);
-      }
-      consumer_sync();
-      if (tq == 0) {
-        ml_s[warp][g][0] = m_run[1]; ml_s[warp][g][1] = l_run[1];
-      }
-      consumer_sync();
-      {
-        float M = -INFINITY;
-        for (int k = 0; k < 4; ++k) M = fmaxf(M, ml_s[mt * 4 + k][g][0]);
-        const float Ms = (M == -INFINITY) ? 0.f : M;
-        float Lsum = 0.f;
-        for (int k = 0; k < 4; ++k) Lsum += ml_s[mt * 4 + k][g][1] * ex2(ml_s[mt * 4 + k][g][0] - Ms);
-        Mx[1] = M; Ls[1] = Lsum; own[1] = ex2(m_run[1] - Ms);
-      }
-      for (int k = 0; k < 4; ++k) {
-        if (kq == k) {
-#pragma unroll
-          for (int n = 0; n < T3 / 8; ++n) {
-            float* r_lo = obuf + (16 * mt + g) * T3 + n * 8 + 2 * tq;
-            float* r_hi = r_lo + 8 * T3;
-            if (k == 0) {
-              r_lo[0] = o[n][0] * own[0]; r_lo[1] = o[n][1] * own[0];
-              r_hi[0] = o[n][2] * own[1]; r_hi[1] = o[n][3] * own[1];
-            } else {
-              r_lo[0] += o[n][0] * own[0]; r_lo[1] += o[n][1] * own[0];
-              r_hi[0] += o[n][2] * own[1]; r_hi[1] += o[n][3] * own[1];
-            }
-          }
-        }
-        consumer_sync();
-      }
-      {
-        const long slot = (long)blockIdx.x + b;
-        float4* dst = reinterpret_cast<float4*>(p.part_o + slot * 32 * T3);
-        const float4* src = reinterpret_cast<const float4*>(obuf);
-        for (int i = threadIdx.x; i < 32 * T3 / 4; i += 256) dst[i] = src[i];
-        if (kq == 0 && tq == 0) {
-          float* ml = p.part_ml + slot * 64;
-          ml[(16 * mt + g) * 2 + 0] = Mx[0]; ml[(16 * mt + g) * 2 + 1] = Ls[0];
-          ml[(16 * mt + g + 8) * 2 + 0] = Mx[1]; ml[(16 * mt + g + 8) * 2 + 1] = Ls[1];
-        }
-      }
-      consumer_sync();
-      // next sequence
-      first += nt;
-      ++b;
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------
 // k_dec_qhat: grid (B, r3 / 32), 256 threads.  CTA (b, y) finishes the new token's latent
 // projections and forms its per-head queries for the 32 latent key coordinates
@@ -507,19 +171,24 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
   // split-K sums: all of qt, this CTA's 32 key coordinates, and the value coordinates c with
   // (c / 32) % gridDim.y == blockIdx.y
   const float* prow = part + (long)b * ncol;
+  const int nB = gridDim.x;                          // sequences
+  // the split-K partials are [splits][rows padded to 128][ncol]: this sequence's row must lie in every split
+  const bool prow_ok = TA_IDX_OK(err, (long)b * ncol, ncol, split_stride) &&
+                       TA_IDX_OK(err, (long)(splits - 1) * split_stride + (long)b * ncol, ncol, (long)splits * split_stride);
   for (int c = threadIdx.x; c < r2 + DQ_CW; c += blockDim.x) {
     const int col = c < r2 ? c : r2 + c0 + (c - r2);
     float acc = 0.f;
-    for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + col];
+    if (prow_ok) for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + col];
     if (c < r2) qt_s[c] = acc; else k_s[c - r2] = acc;
   }
   for (int c = threadIdx.x; c < t3; c += blockDim.x) {
     if ((c / DQ_CW) % gridDim.y != blockIdx.y) continue;
     float acc = 0.f;
-    for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + r2 + r3 + c];
+    if (prow_ok) for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + r2 + r3 + c];
     const bf16 vv = __float2bfloat16_rn(acc);
-    vnew[(long)b * t3 + c] = vv;
-    if (append && !shared_kv) Vc[((long)b * Lmax + L) * t3 + c] = vv;   // shared cache: the key row written below is the value row
+    if (TA_IDX_OK(err, (long)b * t3 + c, 1, (long)nB * t3)) vnew[(long)b * t3 + c] = vv;
+    if (append && !shared_kv && TA_IDX_OK(err, ((long)b * Lmax + L) * t3 + c, 1, (long)nB * Lmax * t3))
+      Vc[((long)b * Lmax + L) * t3 + c] = vv;   // shared cache: the key row written below is the value row
   }
   __syncthreads();
   if (threadIdx.x < DQ_CW / 2) {                    // new key, rotated
@@ -527,8 +196,10 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     const float xe = k_s[2 * i], xo = k_s[2 * i + 1];
     const float2 cs = cs_s[i];
     const __nv_bfloat162 kv = __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
-    *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + c0 + 2 * i) = kv;
-    if (append) *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + c0 + 2 * i) = kv;
+    if (TA_IDX_OK(err, (long)b * r3 + c0 + 2 * i, 2, (long)nB * r3))
+      *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + c0 + 2 * i) = kv;
+    if (append && TA_IDX_OK(err, ((long)b * Lmax + L) * r3 + c0 + 2 * i, 2, (long)nB * Lmax * r3))
+      *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + c0 + 2 * i) = kv;
   }
   // ---- w[a, c0 + .] for batches of AB slices ----
   for (int a0 = 0; a0 < r1; a0 += AB) {
@@ -583,8 +254,9 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     }
     xe *= mult; xo *= mult;
     const float2 cs = cs_s[cp];
-    *reinterpret_cast<__nv_bfloat162*>(qhat + ((long)b * nH + h) * r3 + c0 + 2 * cp) =
-        __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+    if (TA_IDX_OK(err, ((long)b * nH + h) * r3 + c0 + 2 * cp, 2, (long)nB * nH * r3))
+      *reinterpret_cast<__nv_bfloat162*>(qhat + ((long)b * nH + h) * r3 + c0 + 2 * cp) =
+          __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
   }
 }
 
@@ -607,7 +279,7 @@ __host__ __device__ inline size_t dec_out_smem(int nH, int t1, int t3) {
 __global__ void __launch_bounds__(256)
 k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, const int32_t* __restrict__ cache_len,
           int B, int Lmax, int nH, int t1, int t2, int t3, int grid_attn, const bf16* __restrict__ Ct,
-          const bf16* __restrict__ Ut1, bf16* __restrict__ z) {
+          const bf16* __restrict__ Ut1, bf16* __restrict__ z, unsigned int* err) {
   extern __shared__ __align__(16) float do_smem[];
   float* o_s = do_smem;                    // [32][t3]
   float* w_s = o_s + 32 * t3;              // [MAX_GRID][32]
@@ -645,7 +317,9 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
   while (cta_first_tile(i0 + 1, total, grid_attn) <= first) ++i0;
   long i1 = i0;
   while (i1 + 1 < grid_attn && cta_first_tile(i1 + 1, total, grid_attn) < first + nt) ++i1;
-  const int np = (int)(i1 - i0 + 1);
+  int np = (int)(i1 - i0 + 1);
+  // this sequence's partials occupy the slots i0 + b .. i1 + b of the grid_attn + B that exist
+  if (!TA_IDX_OK(err, i0 + b, np, (long)grid_attn + B)) np = 0;
   for (int i = threadIdx.x; i < nH * t1; i += blockDim.x) ut1_s[i] = __bfloat162float(Ut1[i]);
   // which of the np candidate CTAs wrote a partial for this sequence (a CTA whose tile range is
   // empty wrote nothing: its slot holds stale bytes that must not be used as numbers)
@@ -792,7 +466,8 @@ k_dec_out(const float* __restrict__ part_o, const float* __restrict__ part_ml, c
         if (ch + off < nch) t += o;
       }
       const int jrow = jl + jj * 8 * rpl;
-      if (g < rpl && ch == 0 && jrow < jn) z[(long)b * t2 + jbeg + jrow] = __float2bfloat16_rn(t);
+      if (g < rpl && ch == 0 && jrow < jn && TA_IDX_OK(err, (long)b * t2 + jbeg + jrow, 1, (long)B * t2))
+        z[(long)b * t2 + jbeg + jrow] = __float2bfloat16_rn(t);
     }
   }
 }

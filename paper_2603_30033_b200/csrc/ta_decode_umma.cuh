@@ -1,6 +1,7 @@
 // Decode attention over the latent KV cache (Eq. 9) on tcgen05 tensor cores.
 //
-// Same job, same tile split and same partial format as dec::k_dec_attn (the mma.sync kernel), but the
+// Streams every sequence's latent K / V cache exactly once.  All n_H (<= 32) heads share each K / V byte, so the
+// arithmetic is 2 n_H flop per cached element: beyond plain FMA throughput at HBM speed, hence tensor cores.  The
 // two products of a 128-key tile run as UMMA instructions with the KEYS on the M dimension, so that
 // no tensor work is spent on padding the (at most 32) heads up to a 128-row tile:
 //   S^T [128 keys x 32 heads] = K_tile [128 x r3] * Qhat^T          A = K tile as loaded (K-major), B = Qhat (K-major)
@@ -14,8 +15,7 @@
 // P goes back through shared memory (B operands are read from there); the row sums stay in registers
 // per thread and are reduced once per segment.  Score and P buffers are double-buffered, the output
 // accumulator is single: tile t + 1 is scored and exponentiated while P V of tile t runs, and a segment
-// ends with each warpgroup writing its heads of the partial -- the same partial per (CTA, sequence)
-// that the mma.sync kernel writes.
+// ends with each warpgroup writing its heads of the partial (max, sum, unnormalised O) of (CTA, sequence).
 //
 //   warp 0       TMA producer: Qhat of the segment's sequence, K / V ring
 //   warp 1       TMEM allocation, MMA issue
@@ -184,7 +184,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t tmem = tmem_slot;
   const uint32_t tm_o = tmem + 64;
 
-  // ---- this CTA's range of the flat tile list (same split as the mma.sync kernel) ----
+  // ---- this CTA's range of the flat tile list ----
   int lo, hi;
   long excl;
   const long total = dec::block_tile_scan(p.cache_len, p.B, p.Lmax, lo, hi, excl, wtot_s);
@@ -489,12 +489,14 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         if (!(ok = wg_sync())) break;
         const long slot = (long)blockIdx.x + w.b;
-        if (q == 0 && lane < HPW) {
+        // one partial slot per (CTA, sequence) pair that can occur: gridDim.x + B of them
+        const bool slot_ok = TA_IDX_OK(p.err, slot, 1, (long)gridDim.x + p.B);
+        if (slot_ok && q == 0 && lane < HPW) {
           float* ml = p.part_ml + slot * 64 + (wg * HPW + lane) * 2;
           ml[0] = m_lane;
           ml[1] = sum_s[wg][0][lane] + sum_s[wg][1][lane] + sum_s[wg][2][lane] + sum_s[wg][3][lane];
         }
-        if (tid < p.t3) {
+        if (slot_ok && tid < p.t3) {
           float* dst = p.part_o + slot * 32 * p.t3 + (long)(wg * HPW) * p.t3 + tid;
 #pragma unroll
           for (int h = 0; h < HPW; ++h) dst[h * p.t3] = __uint_as_float(o[h]);

@@ -74,6 +74,7 @@ struct PrepParams {
   float mult;
   dec::RopeFreqs freqs;
   int g1, g2, g3;
+  unsigned int* err;
 };
 
 constexpr int PREP_THREADS = 128;
@@ -134,8 +135,9 @@ __global__ void __launch_bounds__(PREP_THREADS) k_prefill_prep(const PrepParams 
     __syncthreads();
     {
       const int cl = t / 4, bb = (t % 4) * 8;
-      *reinterpret_cast<uint4*>(p.GcatT + ((long)h * p.r3 + c0 + cl) * p.r2 + b0 + bb) =
-          *reinterpret_cast<const uint4*>(&tile[cl][bb]);
+      if (TA_IDX_OK(p.err, ((long)h * p.r3 + c0 + cl) * p.r2 + b0 + bb, 8, (long)p.nH * p.r3 * p.r2))
+        *reinterpret_cast<uint4*>(p.GcatT + ((long)h * p.r3 + c0 + cl) * p.r2 + b0 + bb) =
+            *reinterpret_cast<const uint4*>(&tile[cl][bb]);
     }
   } else if (blk < p.g1 + p.g2) {
     // GtP[j, h, c .. c + 8): the value coordinate c is contiguous in the core and in the output
@@ -146,7 +148,8 @@ __global__ void __launch_bounds__(PREP_THREADS) k_prefill_prep(const PrepParams 
       const int c8 = (int)(i % cch) * 8, h = (int)((i / cch) % p.nH), j = (int)(i / ((long)cch * p.nH));
       float acc[8];
       head_core_8(p.Ct + ((long)j * p.t3 + c8), (long)p.t2 * p.t3, p.Ut1 + (long)h * p.t1, p.t1, acc);
-      *reinterpret_cast<uint4*>(p.GtP + ((long)j * p.nH + h) * p.t3 + c8) = pack8(acc);
+      if (TA_IDX_OK(p.err, ((long)j * p.nH + h) * p.t3 + c8, 8, (long)p.t2 * p.nH * p.t3))
+        *reinterpret_cast<uint4*>(p.GtP + ((long)j * p.nH + h) * p.t3 + c8) = pack8(acc);
     }
   } else {
     // (cos, sin) table: four consecutive pairs of one position per thread, two 16-byte stores
@@ -158,8 +161,10 @@ __global__ void __launch_bounds__(PREP_THREADS) k_prefill_prep(const PrepParams 
 #pragma unroll
       for (int e = 0; e < 4; ++e) cs[e] = dec::rope_cos_sin_theta(pos, p.freqs.theta[i0 + e]);
       float4* dst = reinterpret_cast<float4*>(p.rope + i4);
+      if (TA_IDX_OK(p.err, i4, 4, (long)p.n_pos * half)) {
       dst[0] = make_float4(cs[0].x, cs[0].y, cs[1].x, cs[1].y);
       dst[1] = make_float4(cs[2].x, cs[2].y, cs[3].x, cs[3].y);
+      }
     }
   }
 }
@@ -247,11 +252,8 @@ int launch_gemm(Problem& p, const bf16* A, long lda, int M, int K, const BOperan
   while (gp.stages > 1 && umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major, gp.ncb) > kMaxSmem) --gp.stages;
   if (umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major, gp.ncb) > kMaxSmem || Ntot % (BN * gp.ncb) != 0)
     return TA_ERR_UNSUPPORTED_SHAPE;
-  static bool attr_set = false;
-  if (!attr_set) {
-    TA_CUDA_TRY(cudaFuncSetAttribute(umma_gemm::k_umma_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmem));
-    attr_set = true;
-  }
+  static PerDeviceFlag attr;
+  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)umma_gemm::k_umma_gemm, (int)kMaxSmem));
   dim3 grid(Ntot / (BN * gp.ncb), (M + 127) / 128, splits);
   (void)launch_pdl(umma_gemm::k_umma_gemm, grid, dim3(umma_gemm::THREADS),
                    umma_gemm::smem_bytes(gp.stages, BN, gp.b_mn_major, gp.ncb), p.stream, tmA, tmB[0], tmB[1], tmB[2], gp);
@@ -324,12 +326,8 @@ int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const f
   ap.fused = fused ? 1 : 0;
   ap.rope = (fused && d.rope) ? rope : nullptr;
   ap.O = O; ap.err = p.dev_err;
-  static bool attr_set = false;
-  if (!attr_set) {
-    TA_CUDA_TRY(cudaFuncSetAttribute(attn::k_attn_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)attn::SMEM_BYTES));
-    attr_set = true;
-  }
+  static PerDeviceFlag attr;
+  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)attn::k_attn_prefill, (int)attn::SMEM_BYTES));
   const long items = (long)ap.n_qt * d.B * ap.n_hg;
   prof_begin(p);
   (void)launch_pdl(attn::k_attn_prefill, dim3((unsigned)items), dim3(attn::THREADS), attn::SMEM_BYTES, p.stream, tmQ, tmG,
@@ -373,7 +371,7 @@ int fast_fwd(Problem& p) {
     pp.C = (const bf16*)p.C; pp.U1 = (const bf16*)p.U1; pp.Ct = (const bf16*)p.Ct; pp.Ut1 = (const bf16*)p.Ut1;
     pp.GcatT = w.GcatT; pp.GtP = w.GtP; pp.rope = w.rope;
     pp.nH = d.n_H; pp.r1 = d.r1; pp.r2 = d.r2; pp.r3 = d.r3; pp.t1 = d.t1; pp.t2 = d.t2; pp.t3 = d.t3;
-    pp.n_pos = d.N; pp.pos0 = d.pos0;
+    pp.n_pos = d.N; pp.pos0 = d.pos0; pp.err = p.dev_err;
     pp.mult = tc_attn ? p.scale * LOG2E : p.scale;
     pp.freqs = rope_freqs(d);
     // one block per 32 x 32 tile of every G_h^T, one thread per 8 outputs of Gt / 4 entries of the table
@@ -443,12 +441,8 @@ int fast_fwd(Problem& p) {
     zy::Params zp;
     zp.M = T; zp.K1 = K1; zp.t2 = d.t2; zp.d = d.d_model; zp.stages = zy::MAX_STAGES;
     zp.Y = (bf16*)p.Y; zp.err = p.dev_err;
-    static bool attr_set = false;
-    if (!attr_set) {
-      TA_CUDA_TRY(cudaFuncSetAttribute(zy::k_zy_fused, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)zy::smem_bytes(zy::MAX_STAGES)));
-      attr_set = true;
-    }
+    static PerDeviceFlag attr;
+    TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)zy::k_zy_fused, (int)zy::smem_bytes(zy::MAX_STAGES)));
     (void)launch_pdl(zy::k_zy_fused, dim3((T + 127) / 128), dim3(zy::THREADS), zy::smem_bytes(zp.stages), p.stream, tmO, tmG,
                      tmU, zp);
     TA_LAUNCH_CHECK(p);
@@ -482,26 +476,40 @@ namespace {
 
 constexpr int kProjSplits = 16;
 
+// Device properties, looked up once per device ordinal (a process may drive several GPUs).
+struct DeviceProps {
+  std::mutex m;
+  int sms[kMaxDevices] = {};
+  size_t l2[kMaxDevices] = {};
+};
+DeviceProps g_props;
+
+int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  return dev;
+}
+
 int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
+  const int dev = current_device_slot();
+  std::lock_guard<std::mutex> lock(g_props.m);
+  if (!g_props.sms[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    g_props.sms[dev] = n;
   }
-  return n;
+  return g_props.sms[dev];
 }
 
 size_t l2_bytes() {
-  static size_t n = 0;
-  if (!n) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) != cudaSuccess || v <= 0)
-      v = 126 << 20;
-    n = (size_t)v;
+  const int dev = current_device_slot();
+  std::lock_guard<std::mutex> lock(g_props.m);
+  if (!g_props.l2[dev]) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) != cudaSuccess || v <= 0) v = 126 << 20;
+    g_props.l2[dev] = (size_t)v;
   }
-  return n;
+  return g_props.l2[dev];
 }
 
 // number of K splits of the decode projection GEMM: the largest divisor of the K-block count <= kProjSplits
@@ -539,22 +547,7 @@ size_t carve_fast_dec(const tucker_attn_desc& d, char* base, FastDecWs* w) {
   return c.off;
 }
 
-template <int R3, int T3>
-int launch_dec_attn(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const dec::Params& dp) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    TA_CUDA_TRY(cudaFuncSetAttribute(dec::k_dec_attn<R3, T3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)dec::SMEM_BYTES));
-    attr_set = true;
-  }
-  prof_begin(p);
-  (void)launch_pdl(dec::k_dec_attn<R3, T3>, dim3(dp.grid), dim3(dec::THREADS), dec::SMEM_BYTES, p.stream, tmK, tmV, dp);
-  prof_end(p);
-  TA_LAUNCH_CHECK(p);
-  return TA_OK;
-}
-
-// The tcgen05 form of the cache-streaming kernel (keys on the M dimension, ranks at run time).
+// The cache-streaming kernel (tcgen05, keys on the M dimension, ranks at run time).
 int launch_dec_attn_umma(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const dec::Params& dp, int grid) {
   const tucker_attn_desc& d = p.d;
   CUtensorMap tmQ;   // Qhat [B * n_H rows, r3]: one box = 32 rows (all heads of a sequence) x 64 columns
@@ -563,12 +556,8 @@ int launch_dec_attn_umma(Problem& p, const CUtensorMap& tmK, const CUtensorMap& 
   up.B = dp.B; up.nH = dp.nH; up.Lmax = dp.Lmax; up.r3 = d.r3; up.t3 = d.t3; up.shared_kv = dp.shared_kv;
   up.cache_len = dp.cache_len; up.knew = dp.knew; up.vnew = dp.vnew;
   up.part_o = dp.part_o; up.part_ml = dp.part_ml; up.err = dp.err;
-  static bool attr_set = false;
-  if (!attr_set) {
-    TA_CUDA_TRY(cudaFuncSetAttribute(decu::k_dec_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)decu::SMEM_BYTES));
-    attr_set = true;
-  }
+  static PerDeviceFlag attr;
+  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)decu::k_dec_attn_umma, (int)decu::SMEM_BYTES));
   prof_begin(p);
   (void)launch_pdl(decu::k_dec_attn_umma, dim3(grid), dim3(decu::THREADS), decu::SMEM_BYTES, p.stream, tmK, tmV, tmQ, up);
   prof_end(p);
@@ -598,7 +587,7 @@ size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t) { return carve_
 //   1  split-K GEMM   partial [qt | k | v] = x [U2 | U3 | Ut3]           (factors read in place)
 //   2  k_dec_qhat     finish the projections, latent RoPE, cache append, per-head queries (core
 //                     contracted with the query first; no per-head G_h)
-//   3  k_dec_attn_umma  stream the latent caches once, all heads per tile (tcgen05; k_dec_attn is the mma.sync form)
+//   3  k_dec_attn_umma  stream the latent caches once, all heads per tile (tcgen05)
 //   4  k_dec_out      merge the partials, output-side core -> z
 //   5  GEMM           y = z Ut2^T
 int fast_decode(Problem& p) {
@@ -652,23 +641,14 @@ int fast_decode(Problem& p) {
     dp.shared_kv = p.shared_kv;
     dp.cache_len = p.cache_len; dp.qhat = w.qhat; dp.knew = w.knew; dp.vnew = w.vnew;
     dp.part_o = w.part_o; dp.part_ml = w.part_ml; dp.err = p.dev_err;
-    if (!(d.flags & TA_FLAG_MMA_SYNC_DECODE)) rc = launch_dec_attn_umma(p, tmK, tmV, dp, dp.grid);
-    else if (d.r3 == 128 && d.t3 == 128) rc = launch_dec_attn<128, 128>(p, tmK, tmV, dp);
-    else if (d.r3 == 64 && d.t3 == 64) rc = launch_dec_attn<64, 64>(p, tmK, tmV, dp);
-    else if (d.r3 == 96 && d.t3 == 96) rc = launch_dec_attn<96, 96>(p, tmK, tmV, dp);
-    else if (d.r3 == 128 && d.t3 == 64) rc = launch_dec_attn<128, 64>(p, tmK, tmV, dp);
-    else rc = launch_dec_attn<64, 128>(p, tmK, tmV, dp);
+    rc = launch_dec_attn_umma(p, tmK, tmV, dp, dp.grid);
     if (rc) return rc;
     // ---- 4: merge the partials, output-side core ----
-    static bool out_attr_set = false;
-    if (!out_attr_set) {
-      TA_CUDA_TRY(cudaFuncSetAttribute(dec::k_dec_out, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)dec::dec_out_smem(32, 32, 128)));
-      out_attr_set = true;
-    }
+    static PerDeviceFlag out_attr;
+    TA_CUDA_TRY(ensure_dynamic_smem(out_attr, (const void*)dec::k_dec_out, (int)dec::dec_out_smem(32, 32, 128)));
     (void)launch_pdl(dec::k_dec_out, dim3(d.B, dec::DO_JS), dim3(256), dec::dec_out_smem(d.n_H, d.t1, d.t3), p.stream,
                      w.part_o, w.part_ml, p.cache_len, d.B, p.Lmax, d.n_H, d.t1, d.t2, d.t3, dp.grid, (const bf16*)p.Ct,
-                     (const bf16*)p.Ut1, w.z);
+                     (const bf16*)p.Ut1, w.z, p.dev_err);
     TA_LAUNCH_CHECK(p);
   }
   // ---- 5: y = z Ut2^T ----

@@ -50,10 +50,11 @@ extern "C" int tucker_attn_decode_static(const tucker_attn_desc* desc, const voi
                                          const void* Ut2, const void* Ut3, void* Kcache, void* Vcache, int32_t Lmax,
                                          const int32_t* cache_len, int32_t append, void* y, void* cuda_stream) {
   const size_t need = tucker_attn_decode_workspace_bytes(desc, Lmax);
-  if (need == 0) return TA_ERR_INVALID_ARG;                                   // bad descriptor or Lmax
   if (need > (size_t)TA_STATIC_SCRATCH_BYTES) return TA_ERR_WORKSPACE_TOO_SMALL;   // problem too large for the array
   void* scratch = ta::static_scratch_for_current_device();
   if (!scratch) return TA_ERR_CUDA;
+  // need == 0 (invalid descriptor or Lmax, or a shape no kernel covers): nothing will be launched; the decode
+  // call's own validation below names the reason with the status a caller-supplied workspace would get.
   // Nothing in the decode scratch has to start at zero: every region is written by an
   // earlier kernel of the same call before a later one reads it, so stale contents of the
   // previous call are harmless.

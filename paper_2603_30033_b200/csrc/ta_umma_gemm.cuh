@@ -4,7 +4,7 @@
 // most 256; ncb accumulators side by side in TMEM), so that the A tile is loaded once for all of them:
 //   warp 0      TMA producer (one elected lane)
 //   warp 1      TMEM allocation + MMA issue (one elected lane)
-//   warps 2..5  epilogue: TMEM -> registers -> global, one TMEM lane quadrant each
+//   warps 2..9  epilogue: TMEM -> registers -> global, two warps per TMEM lane quadrant
 // The N range is a concatenation of up to three segments (e.g. [Qt | K | V] of the latent
 // projections), each with its own destination and epilogue (plain, latent RoPE on column
 // pairs, fp32), so that one launch serves several logical outputs.
@@ -222,8 +222,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tmem_ld32(acc + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
           if (row >= p.M) continue;
-          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + (long)blockIdx.z * p.split_stride +
-                                                  (long)row * sg.ld + c0 + ch * 32);
+          const long off = (long)blockIdx.z * p.split_stride + (long)row * sg.ld + c0 + ch * 32;
+          // extent of the partial-sum tensor as seen from this segment's base: splits x [M rows of ld]
+          if (!TA_IDX_OK(p.err, off, 32, (long)(gridDim.z - 1) * p.split_stride + (long)(p.M - 1) * sg.ld + sg.width)) continue;
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(sg.out) + off);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
@@ -270,10 +272,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (grow >= p.M) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)rr * pitch + ch * 64 + cc * 16);
             const int col = c0 + ch * 32 + cc * 8;
-            *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + col) = v;
+            if (TA_IDX_OK(p.err, (long)grow * sg.ld + col, 8, (long)(p.M - 1) * sg.ld + sg.width))
+              *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + col) = v;
             if (sg.out2) {
               const int gb = p.n_pos > 0 ? grow / p.n_pos : 0, gn = p.n_pos > 0 ? grow % p.n_pos : grow;
-              *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + (long)gb * sg.batch2 + (long)gn * sg.ld2 + col) = v;
+              const long off2 = (long)gb * sg.batch2 + (long)gn * sg.ld2 + col;
+              // the second copy is [sequences][batch2]: rows n < n_pos of each sequence, `width` columns
+              const long nb2 = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
+              if (TA_IDX_OK(p.err, off2, 8, (nb2 - 1) * sg.batch2 + (long)((p.n_pos > 0 ? p.n_pos : p.M) - 1) * sg.ld2 + sg.width))
+                *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + off2) = v;
             }
           }
         }

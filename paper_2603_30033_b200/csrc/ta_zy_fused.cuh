@@ -206,7 +206,8 @@ k_zy_fused(const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUte
           const int grow = m0 + rr;
           if (grow < p.M) {
             const uint4 v = *reinterpret_cast<const uint4*>(staging + (size_t)rr * STAGING_PITCH + cc * 16);
-            *reinterpret_cast<uint4*>(p.Y + (long)grow * p.d + n * BN2 + cc * 8) = v;
+            if (TA_IDX_OK(p.err, (long)grow * p.d + n * BN2 + cc * 8, 8, (long)p.M * p.d))
+              *reinterpret_cast<uint4*>(p.Y + (long)grow * p.d + n * BN2 + cc * 8) = v;
           }
         }
         __syncwarp();   // the warp's staging rows are free again before its next chunk is converted

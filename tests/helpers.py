@@ -58,5 +58,26 @@ def tolerances(dtype: str, ref=None):
     return (2e-2 * s, 2e-3 * s)
 
 
+def check(got, ref, dtype, what="", scaled=False):
+    """Element-wise comparison of a result with the oracle's.  scaled=False: the absolute bounds of the
+    benchmark workloads; scaled=True (stress shapes with large outputs): bounds grow with the output rms,
+    see tolerances().  With TA_PARITY_LOG=<file> in the environment every comparison appends its raw
+    figures (max-abs, mean-abs, rms of the reference, whether the unscaled bounds would have held)."""
+    import os
+    got, ref = np.asarray(got, np.float64), np.asarray(ref, np.float64)
+    mx, mean = err_stats(got, ref)
+    tmax, tmean = tolerances(dtype, ref if scaled else None)
+    log = os.environ.get("TA_PARITY_LOG")
+    if log:
+        amax, amean = tolerances(dtype)
+        rms = float(np.sqrt(np.mean(ref ** 2)))
+        with open(log, "a") as f:
+            f.write(f"{dtype} | {what} | max-abs {mx:.3e} | mean-abs {mean:.3e} | rms(ref) {rms:.3f} | "
+                    f"{'scaled' if scaled else 'absolute'} | meets absolute: {mx <= amax and mean <= amean}\n")
+    assert np.isfinite(got).all(), what
+    assert mx <= tmax and mean <= tmean, f"{what}: max-abs {mx:.3e} (<= {tmax}), mean-abs {mean:.3e} (<= {tmean})"
+    return mx, mean
+
+
 def with_(w: W.Workload, **kw) -> W.Workload:
     return dataclasses.replace(w, **kw)

@@ -30,14 +30,7 @@ def gpu_fwd(X, wt, w, flags=0, pos0=0, caches=None, scale=0.0):
     return Y.float().cpu().numpy().astype(np.float64)
 
 
-def check(got, ref, dtype, what="", scaled=False):
-    """scaled=False: the absolute bounds of the benchmark workloads; scaled=True (stress shapes
-    with large outputs): bounds grow with the output rms, see helpers.tolerances."""
-    mx, mean = H.err_stats(got, ref)
-    tmax, tmean = H.tolerances(dtype, ref if scaled else None)
-    assert np.isfinite(got).all(), what
-    assert mx <= tmax and mean <= tmean, f"{what}: max-abs {mx:.3e} (<= {tmax}), mean-abs {mean:.3e} (<= {tmean})"
-    return mx, mean
+check = H.check
 
 
 # --------------------------------------------------------------------------------------
@@ -86,15 +79,18 @@ def test_small_shapes_generic(shape, dtype):
     w = H.custom_workload(dtype=dtype, rope_base=10000.0, seed=31, **shape)
     X, wt = H.host_inputs(w)
     got = gpu_fwd(X, wt, w, flags=Bd.TA_FLAG_FORCE_GENERIC, pos0=5)
-    check(got, oracle_fwd(X, wt, w, pos0=5), dtype, str(shape), scaled=True)
+    check(got, oracle_fwd(X, wt, w, pos0=5), dtype, str(shape))
 
 
+# `scaled=True` marks the stress shapes whose outputs are several times larger than the benchmark workloads'
+# (rms 0.45 .. 1.5 against <= 0.16) and whose raw bf16 errors exceed the absolute 2e-2 / 2e-3; every other shape is
+# held to the absolute bounds.
 FAST = [
-    dict(B=2, N=200, d_model=128, n_H=4, r=(4, 64, 64), t=(4, 64, 64), causal=True, rope=True),
+    dict(B=2, N=200, d_model=128, n_H=4, r=(4, 64, 64), t=(4, 64, 64), causal=True, rope=True, scaled=True),
     dict(B=1, N=333, d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 128), causal=False, rope=False),
-    dict(B=3, N=128, d_model=256, n_H=8, r=(8, 128, 128), t=(8, 128, 128), causal=True, rope=True),
-    dict(B=2, N=77, d_model=64, n_H=2, r=(2, 32, 32), t=(2, 96, 96), causal=True, rope=False),
-    dict(B=1, N=1, d_model=64, n_H=2, r=(2, 64, 64), t=(2, 64, 64), causal=True, rope=True),
+    dict(B=3, N=128, d_model=256, n_H=8, r=(8, 128, 128), t=(8, 128, 128), causal=True, rope=True, scaled=True),
+    dict(B=2, N=77, d_model=64, n_H=2, r=(2, 32, 32), t=(2, 96, 96), causal=True, rope=False, scaled=True),
+    dict(B=1, N=1, d_model=64, n_H=2, r=(2, 64, 64), t=(2, 64, 64), causal=True, rope=True, scaled=True),
     # query rank above 128: per-head queries come from the separate GEMM, not the attention prologue
     dict(B=2, N=150, d_model=256, n_H=4, r=(4, 256, 64), t=(4, 64, 64), causal=True, rope=True),
     # no mask: one CTA walks several head pairs; odd head count ends on a single head
@@ -109,11 +105,13 @@ FAST = [
 
 @pytest.mark.parametrize("shape", FAST)
 def test_small_shapes_tensor_core_path(shape):
+    shape = dict(shape)
+    scaled = shape.pop("scaled", False)
     w = H.custom_workload(dtype="bf16", rope_base=10000.0, seed=77, **shape)
     X, wt = H.host_inputs(w)
     got = gpu_fwd(X, wt, w, pos0=3)
     assert Bd.last_path() == 2
-    check(got, oracle_fwd(X, wt, w, pos0=3), "bf16", str(shape), scaled=True)
+    check(got, oracle_fwd(X, wt, w, pos0=3), "bf16", str(shape), scaled=scaled)
 
 
 def test_fused_and_unfused_query_paths_agree():
@@ -125,7 +123,7 @@ def test_fused_and_unfused_query_paths_agree():
     for flags in (0, Bd.TA_FLAG_SEPARATE_QUERIES, Bd.TA_FLAG_FMA_ATTENTION, Bd.TA_FLAG_SEPARATE_OUTPUT_GEMMS):
         got = gpu_fwd(X, wt, w, flags=flags, pos0=1000)
         assert Bd.last_path() == 2
-        check(got, ref, "bf16", f"flags={flags}", scaled=True)
+        check(got, ref, "bf16", f"flags={flags}")
 
 
 def test_results_are_bit_repeatable():
@@ -226,7 +224,7 @@ def test_decode_small_generic(dtype):
     w = H.custom_workload(kind="decode", dtype=dtype, d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 20), rope=True, seed=17)
     lens = [0, 1, 31, 32, 33, 100]
     y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, 6, lens, 128, flags=Bd.TA_FLAG_FORCE_GENERIC)
-    check(y, ref, dtype, "decode small", scaled=True)
+    check(y, ref, dtype, "decode small")
     tol = 1e-5 if dtype == "fp32" else 2e-2
     Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
     for b, L in enumerate(lens):
@@ -239,21 +237,20 @@ DEC_FAST = [
     dict(d_model=256, n_H=4, r=(2, 64, 64), t=(2, 64, 64), lens=[0, 1, 127, 128, 129, 300, 1000], Lmax=1024),
     dict(d_model=256, n_H=32, r=(8, 128, 128), t=(8, 128, 128), lens=[511, 5, 2047, 256, 255], Lmax=2048),
     dict(d_model=192, n_H=12, r=(4, 96, 96), t=(4, 32, 96), lens=[700, 33], Lmax=777),
-    dict(d_model=128, n_H=2, r=(2, 32, 128), t=(2, 64, 64), lens=[100] * 3 + [4000] + [0] * 200, Lmax=4001),
+    dict(d_model=128, n_H=2, r=(2, 32, 128), t=(2, 64, 64), lens=[100] * 3 + [4000] + [0] * 200, Lmax=4001, scaled=True),
     dict(d_model=128, n_H=8, r=(2, 64, 64), t=(2, 32, 128), lens=[50000], Lmax=50001),
 ]
 
 
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
 @pytest.mark.parametrize("append", [True, False])
 @pytest.mark.parametrize("case", DEC_FAST)
-def test_decode_tensor_core_path(case, append, flags):
+def test_decode_tensor_core_path(case, append):
     case = dict(case)
-    lens, Lmax = case.pop("lens"), case.pop("Lmax")
+    lens, Lmax, scaled = case.pop("lens"), case.pop("Lmax"), case.pop("scaled", False)
     w = H.custom_workload(kind="decode", dtype="bf16", rope=True, rope_base=500000.0, seed=23, **case)
-    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, len(lens), lens, Lmax, append=append, flags=flags)
+    y, ref, (Kd, Vd, Kc, Vc, ref_k, ref_v, cl) = run_decode(w, len(lens), lens, Lmax, append=append)
     assert Bd.last_path() == 2
-    check(y, ref, "bf16", f"decode {case}", scaled=True)
+    check(y, ref, "bf16", f"decode {case}", scaled=scaled)
     Kh, Vh = Kd.float().cpu().numpy(), Vd.float().cpu().numpy()
     for b, L in enumerate(lens[:8]):
         if append:
@@ -262,8 +259,7 @@ def test_decode_tensor_core_path(case, append, flags):
         assert np.array_equal(Kh[b], Kc[b].astype(np.float32)) and np.array_equal(Vh[b], Vc[b].astype(np.float32))
 
 
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
-def test_decode_growing_scores_exercise_the_rescaling(flags):
+def test_decode_growing_scores_exercise_the_rescaling():
     # Cached keys whose norm grows along the sequence and a pre-softmax core scaled by 8: the running maximum
     # of most heads rises by far more than the lazy-rescale threshold from tile to tile, so the accumulated
     # outputs and row sums are rescaled again and again (the random caches of the other tests almost never
@@ -281,7 +277,7 @@ def test_decode_growing_scores_exercise_the_rescaling(flags):
                                      rope_base=w.rope_base)
     y = Bd.tucker_attn_decode(H.to_device(x, w.dtype), *H.weights_to_device(wt, w.dtype), H.to_device(Kc, w.dtype),
                               H.to_device(Vc, w.dtype), torch.from_numpy(cache_len).cuda(), n_H=w.n_H, rope=True,
-                              rope_base=w.rope_base, append=True, flags=flags)
+                              rope_base=w.rope_base, append=True)
     assert Bd.last_device_error() == 0 and Bd.last_path() == 2
     check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "decode, growing scores", scaled=True)
 
@@ -301,8 +297,7 @@ def _shared_weights(w):
     ("bf16", dict(d_model=192, n_H=6, r=(3, 96, 64), t=(2, 32, 64)), 2),
     ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
 ])
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
-def test_decode_shared_latent_cache(dtype, shape, path, flags):
+def test_decode_shared_latent_cache(dtype, shape, path):
     import torch
     w = H.custom_workload(kind="decode", dtype=dtype, rope=False, seed=61, **shape)
     wt = _shared_weights(w)
@@ -316,9 +311,9 @@ def test_decode_shared_latent_cache(dtype, shape, path, flags):
     dw[7] = dw[3]                                        # the same device tensor for U3 and Ut3
     Kd = H.to_device(Kc, dtype)
     y = Bd.tucker_attn_decode(H.to_device(x, dtype), *dw, Kd, Kd, torch.from_numpy(cache_len).cuda(), n_H=w.n_H,
-                              rope=False, append=True, flags=flags)
+                              rope=False, append=True)
     assert Bd.last_device_error() == 0 and Bd.last_path() == path
-    check(y.float().cpu().numpy().astype(np.float64), ref, dtype, f"shared decode {shape}", scaled=True)
+    check(y.float().cpu().numpy().astype(np.float64), ref, dtype, f"shared decode {shape}")
     Kh = Kd.float().cpu().numpy()
     tol = 1e-5 if dtype == "fp32" else 3e-2
     for b, L in enumerate(lens):
@@ -338,7 +333,7 @@ def test_prefill_shared_projection_and_cache():
     cache = torch.full((2, 210, 128), 7.0, device="cuda", dtype=torch.bfloat16)
     Y = Bd.tucker_attn_fwd(H.to_device(X, w.dtype), *dw, n_H=w.n_H, causal=True, rope=False, Kcache=cache, Vcache=cache)
     assert Bd.last_device_error() == 0 and Bd.last_path() == 2
-    check(Y.float().cpu().numpy().astype(np.float64), ref, "bf16", "shared prefill", scaled=True)
+    check(Y.float().cpu().numpy().astype(np.float64), ref, "bf16", "shared prefill")
     for b in range(2):
         assert np.abs(cache[b, :200].float().cpu().numpy() - parts[b]["K"]).max() < 3e-2
     assert (cache[:, 200:] == 7.0).all()
@@ -378,7 +373,7 @@ def test_decode_garbage_beyond_cache_len_is_ignored():
     y = Bd.tucker_attn_decode(H.to_device(x, "bf16"), *H.weights_to_device(wt, "bf16"), Kd, Vd,
                               torch.from_numpy(cache_len).cuda(), n_H=4, rope=True, rope_base=w.rope_base, append=False)
     assert Bd.last_device_error() == 0 and Bd.last_path() == 2
-    check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "garbage tail", scaled=True)
+    check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "garbage tail")
 
 
 def test_decode_no_append_leaves_cache():
@@ -412,6 +407,9 @@ def test_a_wait_that_nothing_ends_gives_up_and_is_reported():
     out = Bd.selftest_wait_timeout(2000)
     err = Bd.last_device_error()                       # synchronises the stream
     assert err == Bd.TA_DEVERR_WAIT_TIMEOUT
+    Bd.selftest_wait_timeout(1000)                     # once more: the status-code form of the same read
+    assert Bd.sync_status() == -5 and Bd.status_string(-5) == "device-side wait timed out"
+    assert Bd.sync_status() == 0
     first, second, cycles_k = out.cpu().tolist()
     assert first == 0 and second == 0                  # both waits gave up ...
     assert cycles_k < (50_000_000 >> 10)               # ... the second long before its own two-second budget
@@ -452,10 +450,9 @@ def test_sharp_softmax_variant():
     check(got[:, rows], oracle_fwd(X, wt, w, rows=rows), w.dtype, "sharp c2", scaled=True)
 
 
-@pytest.mark.parametrize("flags", [0, Bd.TA_FLAG_MMA_SYNC_DECODE])
-def test_full_size_decode_sampled(flags):
+def test_full_size_decode_sampled():
     # benchmark decode workload: 64 sequences, 32768 cached latent rows each, RoPE at position 32768
-    # (with both forms of the cache-streaming kernel, each in the launch configuration bench.py times)
+    # (in the launch configuration bench.py times)
     import torch
     w = W.get_workload("c5")
     L, Lmax, B = w.N, w.N + 1, w.B
@@ -471,7 +468,7 @@ def test_full_size_decode_sampled(flags):
         Kd[b, :lens[b]] = torch.from_numpy(k).to(torch.bfloat16).cuda()
         Vd[b, :lens[b]] = torch.from_numpy(v).to(torch.bfloat16).cuda()
     y = Bd.tucker_attn_decode(H.to_device(x, w.dtype), *dw, Kd, Vd, torch.from_numpy(lens).cuda(), n_H=w.n_H,
-                              rope=True, rope_base=w.rope_base, append=True, flags=flags)
+                              rope=True, rope_base=w.rope_base, append=True)
     assert Bd.last_device_error() == 0
     y = y.float().cpu().numpy().astype(np.float64)
     sample = [0, 5, 40, 63]
