@@ -171,7 +171,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
   // split-K sums: all of qt, this CTA's 32 key coordinates, and the value coordinates c with
   // (c / 32) % gridDim.y == blockIdx.y
   const float* prow = part + (long)b * ncol;
-  const int nB = gridDim.x;                          // sequences
+  [[maybe_unused]] const int nB = gridDim.x;         // sequences
   // the split-K partials are [splits][rows padded to 128][ncol]: this sequence's row must lie in every split
   const bool prow_ok = TA_IDX_OK(err, (long)b * ncol, ncol, split_stride) &&
                        TA_IDX_OK(err, (long)(splits - 1) * split_stride + (long)b * ncol, ncol, (long)splits * split_stride);

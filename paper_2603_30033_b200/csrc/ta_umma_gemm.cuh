@@ -278,7 +278,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const int gb = p.n_pos > 0 ? grow / p.n_pos : 0, gn = p.n_pos > 0 ? grow % p.n_pos : grow;
               const long off2 = (long)gb * sg.batch2 + (long)gn * sg.ld2 + col;
               // the second copy is [sequences][batch2]: rows n < n_pos of each sequence, `width` columns
-              const long nb2 = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
+              [[maybe_unused]] const long nb2 = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
               if (TA_IDX_OK(p.err, off2, 8, (nb2 - 1) * sg.batch2 + (long)((p.n_pos > 0 ? p.n_pos : p.M) - 1) * sg.ld2 + sg.width))
                 *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out2) + off2) = v;
             }
