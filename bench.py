@@ -337,6 +337,8 @@ def oracle_sample(w, budget="default"):
     by = W.decode_bytes(w, B=nseq)
 
     def run():
+        if getattr(w, "shared_kv", False) and w.rope:      # one cache of un-rotated rows, keys rotated when used
+            return O.tucker_attn_decode_shared_rope(x, *args[:7], Kc, lens, rope_base=w.rope_base)
         return O.tucker_attn_decode(x, *args, Kc, Vc, lens, rope=w.rope, rope_base=w.rope_base)
     return run, by["total"] / 1e9, f"{nseq} of {w.B} sequences with the full {L}-entry cache", "GB/s"
 
@@ -487,7 +489,7 @@ def main():
 
     others = []
     if not args.no_others and world == 1:
-        for name in ("c2", "c3", "c4", "c5", "f1"):
+        for name in ("c2", "c3", "c4", "c5", "f1", "f1r"):
             ow = W.get_workload(name)
             if ow.name == w.name:
                 continue

@@ -106,10 +106,12 @@ TA_API size_t tucker_attn_decode_workspace_bytes(const tucker_attn_desc* desc, i
  * All steps, including the weight-only core contraction, run inside the call.
  *
  * Shared key / value projection (Sec. 3.1, "L^KV = X U3"): pass the SAME pointer for U3 and Ut3
- * (then r3 == t3) with rope == 0.  The latent keys are then the latent values; they are projected
- * once, and Kcache_out may equal Vcache_out (one cache of N r3 entries instead of 2 N r3).  With
- * latent RoPE the cached keys are rotated and cannot double as values: Kcache_out == Vcache_out is
- * TA_ERR_INVALID_ARG unless U3 == Ut3, r3 == t3 and rope == 0.
+ * (then r3 == t3).  Kcache_out may then equal Vcache_out: ONE cache of N r3 entries instead of 2 N r3.
+ * Without RoPE the latent keys are the latent values and are projected once.  With latent RoPE
+ * (Definition 2) the keys are the rotated latent rows and the values the un-rotated ones; the one cache
+ * receives the UN-rotated rows (the paper does not say what the single cache holds in this case: the
+ * un-rotated row serves as the value as it is, and its key is re-formed by rotating it when it is read).
+ * Kcache_out == Vcache_out with distinct U3 / Ut3 pointers or r3 != t3 is TA_ERR_INVALID_ARG.
  */
 TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
                     const void* C, const void* U1, const void* U2, const void* U3,
@@ -129,9 +131,11 @@ TA_API int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X,
  *   y         [B, d_model]                     out
  *   desc->N, desc->pos0, desc->causal are ignored.
  *
- * Shared latent cache (Sec. 3.1): Kcache == Vcache is accepted when U3 == Ut3 (same pointer),
- * r3 == t3 and rope == 0; the step then reads every cached row once (half the bytes) and appends
- * one row.  Any other call with Kcache == Vcache is TA_ERR_INVALID_ARG.
+ * Shared latent cache (Sec. 3.1): Kcache == Vcache is accepted when U3 == Ut3 (same pointer) and
+ * r3 == t3; the step then reads every cached row once (half the bytes) and appends one row.  With
+ * rope == 1 that cache holds UN-rotated latent rows (see tucker_attn_fwd): every key tile is rotated
+ * by R(n, r3) on chip after it has been loaded, the values are the rows as stored, and the appended
+ * row is the un-rotated one.  Any other call with Kcache == Vcache is TA_ERR_INVALID_ARG.
  */
 TA_API int tucker_attn_decode(const tucker_attn_desc* desc, const void* x,
                        const void* C, const void* U1, const void* U2, const void* U3,

@@ -52,9 +52,9 @@ static bool use_fast_decode(const tucker_attn_desc& d, int32_t Lmax) {
 
 // Shared key / value projection (Sec. 3.1, L^KV = X U3): the caller passes the SAME factor for U3 and Ut3.
 // Without RoPE the latent keys are then the latent values, so one projection and one cache serve both.
-// (With latent RoPE the cached keys are rotated and cannot double as values.)
+// With latent RoPE the one cache holds the un-rotated latent rows (the values); keys are rotated when used.
 static bool shared_kv_weights(const tucker_attn_desc& d, const void* U3, const void* Ut3) {
-  return U3 == Ut3 && d.r3 == d.t3 && !d.rope;
+  return U3 == Ut3 && d.r3 == d.t3;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -99,7 +99,9 @@ int tucker_attn_fwd(const tucker_attn_desc* desc, const void* X, const void* C, 
   p.X = X; p.C = C; p.U1 = U1; p.U2 = U2; p.U3 = U3; p.Ct = Ct; p.Ut1 = Ut1; p.Ut2 = Ut2; p.Ut3 = Ut3;
   p.Y = Y; p.Kc = Kcache_out; p.Vc = Vcache_out; p.Lmax = Lmax;
   p.cache_len = nullptr; p.append = 0;
-  p.shared_kv = (shared_kv_weights(*desc, U3, Ut3) && Kcache_out == Vcache_out) ? 1 : 0;
+  const bool one_cache = shared_kv_weights(*desc, U3, Ut3) && Kcache_out == Vcache_out;
+  p.shared_kv = (one_cache && !desc->rope) ? 1 : 0;                   // one projection serves keys and values
+  p.shared_rope = (one_cache && desc->rope && Kcache_out) ? 1 : 0;    // rotated keys computed, un-rotated rows cached
   p.ws = static_cast<char*>(workspace); p.ws_bytes = workspace_bytes;
   p.stream = static_cast<cudaStream_t>(cuda_stream);
   p.dev_err = device_error_ptr();
@@ -135,6 +137,7 @@ int tucker_attn_decode(const tucker_attn_desc* desc, const void* x, const void* 
   p.Y = y; p.Kc = Kcache; p.Vc = Vcache; p.Lmax = Lmax;
   p.cache_len = cache_len; p.append = append ? 1 : 0;
   p.shared_kv = (Kcache == Vcache) ? 1 : 0;
+  p.shared_rope = (p.shared_kv && desc->rope) ? 1 : 0;
   p.ws = static_cast<char*>(workspace); p.ws_bytes = workspace_bytes;
   p.stream = static_cast<cudaStream_t>(cuda_stream);
   p.dev_err = device_error_ptr();

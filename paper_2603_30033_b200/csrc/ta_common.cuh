@@ -25,7 +25,8 @@ struct Problem {
   int32_t Lmax;
   const int32_t* cache_len; // decode only (device)
   int32_t append;           // decode only
-  int shared_kv;            // one latent cache / one projection serves keys and values (U3 == Ut3, no RoPE)
+  int shared_kv;            // one latent cache / one projection serves keys and values (U3 == Ut3)
+  int shared_rope;          // ... together with latent RoPE: the one cache holds UN-rotated latent rows
   char* ws;                 // workspace base (256-byte aligned)
   size_t ws_bytes;
   cudaStream_t stream;

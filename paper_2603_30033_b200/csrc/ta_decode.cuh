@@ -187,7 +187,9 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     if (prow_ok) for (int s = 0; s < splits; ++s) acc += prow[s * split_stride + r2 + r3 + c];
     const bf16 vv = __float2bfloat16_rn(acc);
     if (TA_IDX_OK(err, (long)b * t3 + c, 1, (long)nB * t3)) vnew[(long)b * t3 + c] = vv;
-    if (append && !shared_kv && TA_IDX_OK(err, ((long)b * Lmax + L) * t3 + c, 1, (long)nB * Lmax * t3))
+    // shared_kv == 1 (one cache, no RoPE): the key row written below is the value row; == 2 (one cache with
+    // latent RoPE): the cache holds un-rotated rows, i.e. this value row, and the rotated key is not stored
+    if (append && shared_kv != 1 && TA_IDX_OK(err, ((long)b * Lmax + L) * t3 + c, 1, (long)nB * Lmax * t3))
       Vc[((long)b * Lmax + L) * t3 + c] = vv;   // shared cache: the key row written below is the value row
   }
   __syncthreads();
@@ -198,7 +200,7 @@ k_dec_qhat(const float* __restrict__ part, int splits, long split_stride, int nH
     const __nv_bfloat162 kv = __floats2bfloat162_rn(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
     if (TA_IDX_OK(err, (long)b * r3 + c0 + 2 * i, 2, (long)nB * r3))
       *reinterpret_cast<__nv_bfloat162*>(knew + (long)b * r3 + c0 + 2 * i) = kv;
-    if (append && TA_IDX_OK(err, ((long)b * Lmax + L) * r3 + c0 + 2 * i, 2, (long)nB * Lmax * r3))
+    if (append && shared_kv != 2 && TA_IDX_OK(err, ((long)b * Lmax + L) * r3 + c0 + 2 * i, 2, (long)nB * Lmax * r3))
       *reinterpret_cast<__nv_bfloat162*>(Kc + ((long)b * Lmax + L) * r3 + c0 + 2 * i) = kv;
   }
   // ---- w[a, c0 + .] for batches of AB slices ----

@@ -22,6 +22,14 @@
 //   warps 4 + 4 g .. 7 + 4 g   softmax warpgroup g (heads HPW g .. HPW g + HPW - 1)
 // TMEM columns: S_0 [0,32) S_1 [32,64) O [64,96).
 // Every wait is bounded (Abort): on a timeout the CTA raises the device error word and leaves.
+//
+// ROT = true: one shared latent cache L^KV (Sec. 3.1) together with latent RoPE (Definition 2).  The cache then
+// holds UN-rotated rows: the value side uses a tile as it was loaded, and a fourth warpgroup (thread = key
+// row = TMEM lane) writes the rotated copy K_n R(n, r3) of every tile into TMEM (bf16 pairs, columns
+// [128, 256), two buffers), from where it feeds the score product as the A operand.
+// cos / sin of n theta_i = (k0 + row) theta_i come by angle addition from the thread's own constants for `row`
+// (registers) and the tile's 64 base values for k0 (formed per tile with the angle reduced in double precision).
+//   warps 12..15  rotation warpgroup (ROT only)
 #pragma once
 
 #include "ta_common.cuh"
@@ -39,6 +47,8 @@ constexpr int TK = 128;                  // keys per tile
 constexpr int NWG = 2;                    // softmax warpgroups (4 was measured: slower, 138 us against 118 us with the shared cache)
 constexpr int HPW = 32 / NWG;             // head columns per warpgroup
 constexpr int THREADS = 128 + 128 * NWG;
+constexpr int THREADS_ROT = THREADS + 128;           // plus the rotation warpgroup
+constexpr uint32_t TMEM_KROT = 128;                   // first TMEM column of the two rotated key tiles (64 columns each)
 constexpr int MAX_STAGES = 6;
 constexpr int SUB_BYTES = 128 * 64 * 2;  // [128 keys x 64] bf16
 constexpr int MAX_SUB = 2;               // r3, t3 <= 128
@@ -122,9 +132,10 @@ template <> struct TmemCols<8> {
   static __device__ __forceinline__ void st(uint32_t a, const uint32_t (&r)[8]) { tmem_st8(a, r); }
 };
 
-__global__ void __launch_bounds__(THREADS, 1)
+template <bool ROT, int R3C>
+__global__ void __launch_bounds__(ROT ? THREADS_ROT : THREADS, 1)
 k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                const __grid_constant__ CUtensorMap tmQ, const Params p) {
+                const __grid_constant__ CUtensorMap tmQ, const Params p, const dec::RopeFreqs freqs) {
   // cache_len was final before the preceding kernel (which forms the queries and appends the new row)
   // began: set-up and the tile split run while it finishes, and every role passes pdl_enter() before it
   // touches anything else.  (Requesting the first cache tiles ahead of that wait as well was measured:
@@ -132,6 +143,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[MAX_STAGES], empty_bar[MAX_STAGES], q_full[2], q_empty[2];
   __shared__ uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_read, patched, wg_bar[NWG];
+  __shared__ uint64_t kr_full[2], kr_free[2];        // ROT: rotated key tile written / consumed by the score product
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   // per tile: the four warps' maxima per head of each warpgroup, as bf16 (the reference maximum only has
@@ -139,7 +151,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   // warp may start the next tile while another still reads this one's; per segment: the warps' row sums
   __shared__ __align__(16) __nv_bfloat16 mxh[NWG][2][4][HPW];   // [wg][tile parity][warp][head]
   __shared__ float sum_s[NWG][4][HPW];                          // [wg][warp][head]
-  __shared__ long long wtot_s[THREADS / 32];
+  __shared__ long long wtot_s[THREADS_ROT / 32];
   __shared__ int loc_b;
   __shared__ long long loc_first;
 
@@ -170,12 +182,16 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mbar_init(&p_free[i], 1);         // the P V product that read this P buffer is complete
     }
     for (int i = 0; i < NWG; ++i) mbar_init(&wg_bar[i], 4);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&kr_full[i], 4);        // one arrival per rotation warp
+      mbar_init(&kr_free[i], 1);
+    }
     mbar_init(&o_read, 4 * NWG);
     mbar_init(&patched, 4);
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(&tmem_slot, 128);
+    tmem_alloc(&tmem_slot, ROT ? 256 : 128);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -297,8 +313,12 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           ++seg;
           if (!(ok = mbar_wait(&q_full[seg & 1], (uint32_t)((seg >> 1) & 1), ab))) break;
         }
-        if (!(ok = mbar_wait(&full_bar[st], st_par, ab))) break;
-        if (w.last_tile(t)) {
+        if (ROT) {
+          // the rotation warpgroup has seen the tile arrive, written its rotated copy and (last tile of a
+          // sequence) patched the new token's row into both
+          if (!(ok = mbar_wait(&kr_full[buf], (uint32_t)(j & 1), ab))) break;
+        } else if (!(ok = mbar_wait(&full_bar[st], st_par, ab))) break;
+        if (!ROT && w.last_tile(t)) {
           // Warpgroup 0 patches this tile only after it has flushed the segments before it, and such a
           // flush waits for every P V issued so far: issue the pending ones first.
           while (n_pend > 0 && ok) ok = pop_pv();
@@ -313,12 +333,16 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           const uint64_t dk = dk0 + stage_step * (uint64_t)st;
           const uint64_t dq = dq0 + (uint64_t)((seg & 1) * (QBUF_BYTES >> 4));
           const uint32_t d = tmem + (uint32_t)buf * 32u;
+          const uint32_t akr = tmem + TMEM_KROT + (uint32_t)buf * 64u;    // ROT: the rotated key tile, 8 columns per K step
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            if (ks < ksteps)
-              umma_ss(d, dk + (uint64_t)((ks >> 2) * (SUB_BYTES >> 4) + (ks & 3) * 2),
-                      dq + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2), idesc_qk, ks != 0 ? 1u : 0u);
+            if (ks < ksteps) {
+              const uint64_t dqk = dq + (uint64_t)((ks >> 2) * (QSUB_BYTES >> 4) + (ks & 3) * 2);
+              if (ROT) umma_ts(d, akr + (uint32_t)ks * 8u, dqk, idesc_qk, ks != 0 ? 1u : 0u);
+              else umma_ss(d, dk + (uint64_t)((ks >> 2) * (SUB_BYTES >> 4) + (ks & 3) * 2), dqk, idesc_qk, ks != 0 ? 1u : 0u);
+            }
           umma_commit(&s_full[buf]);
+          if (ROT) umma_commit(&kr_free[buf]);
           if (w.seg_end(t)) umma_commit(&q_empty[seg & 1]);   // the segment's Qhat buffer is free once these complete
         }
         {
@@ -336,9 +360,114 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
    // with (registers at launch x threads) minus what the first warpgroup keeps.  2 warpgroups: 168 x 384
    // = 64512 = 128 x 56 + 256 x 224.  4 warpgroups: 96 x 640 = 61440 >= 128 x 56 + 512 x 104 = 60416.
    static_assert(NWG == 2 || NWG == 4, "register budgets below are written for 2 or 4 softmax warpgroups");
-   if (NWG == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+   // ROT (512 threads, 128 registers at launch): 128 x 56 + 256 x 128 (unchanged) + 128 x 200 = 65536.
+   if (ROT && warp >= 12) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+   else if (ROT) { }
+   else if (NWG == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
    else asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
-   if (have_work) {
+   if (ROT && warp >= 12) {
+    if (have_work) {
+     pdl_enter();
+     // ------------------------------- rotation warpgroup --------------------------
+     constexpr int HALF = R3C / 2;                // coordinate pairs per row
+     const int q = warp - 12;
+     const int tid = q * 32 + lane;              // key row of a tile
+     float ac[HALF > 0 ? HALF : 1], as_[HALF > 0 ? HALF : 1];   // (cos, sin)(tid theta_i)
+#pragma unroll
+     for (int i = 0; i < HALF; ++i) {
+       const float2 cs = dec::rope_cos_sin_theta(tid, freqs.theta[i]);
+       ac[i] = cs.x; as_[i] = cs.y;
+     }
+     auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+       bool good = mbar_wait(bar, parity, ab);
+       return __all_sync(0xffffffffu, good);
+     };
+     const float2 step_lo = dec::rope_cos_sin_theta(TK, freqs.theta[lane]);
+     const float2 step_hi = dec::rope_cos_sin_theta(TK, freqs.theta[32 + (lane & 31)]);
+     float2 base_lo = make_float2(1.f, 0.f), base_hi = make_float2(1.f, 0.f);
+     Walk w;
+     w.init(p, t_begin, t_end, b0, seq_first);
+     int it = 0;
+     bool ok = true;
+     for (long t = t_begin; t < t_end && ok; ++t, ++it) {
+       w.seek(t);
+       const int s = it % STAGES, buf = it & 1, j = it >> 1;
+       if (!(ok = wait_all(&full_bar[s], (uint32_t)((it / STAGES) & 1)))) break;
+       if (j > 0 && !(ok = wait_all(&kr_free[buf], (uint32_t)((j - 1) & 1)))) break;   // score product of tile it - 2 is done
+       tc_fence_after();
+       const int k0 = w.k0(t);
+       // (cos, sin)(k0 theta_i) of this tile: lane l holds the values of pairs l and l + 32; they reach the
+       // other lanes by shuffles (all lanes of a warp work on the same pair index at the same time).  At the
+       // first tile of a segment they are formed with the angle reduced in double precision; from tile to tile
+       // they advance by the rotation through 128 theta_i (at most 256 steps of 1e-7 each: far below bf16).
+       if (w.seg_start(t)) {
+         base_lo = dec::rope_cos_sin_theta(k0, freqs.theta[lane]);
+         base_hi = (HALF > 32) ? dec::rope_cos_sin_theta(k0, freqs.theta[32 + (lane & 31)]) : make_float2(1.f, 0.f);
+       } else {
+         base_lo = make_float2(base_lo.x * step_lo.x - base_lo.y * step_lo.y, base_lo.y * step_lo.x + base_lo.x * step_lo.y);
+         base_hi = make_float2(base_hi.x * step_hi.x - base_hi.y * step_hi.y, base_hi.y * step_hi.x + base_hi.x * step_hi.y);
+       }
+       uint8_t* raw = ring + (size_t)s * stage_bytes;
+       const bool last = w.last_tile(t);
+       const int rnew = w.L - k0;               // row of the new token (last tile of a sequence only)
+       const bool is_new = last && tid == rnew;
+       const uint32_t kaddr = tmem + TMEM_KROT + (uint32_t)buf * 64u + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+       for (int hf = 0; hf < 2; ++hf) {         // 32 TMEM columns = 64 coordinates at a time
+         if (hf * 64 < R3C) {
+           uint32_t o[32];
+#pragma unroll
+           for (int cc = 0; cc < 8; ++cc) {
+             const int c = hf * 8 + cc;         // 16-byte chunk of the row
+             if (c < R3C / 8) {
+               const uint4 v = *reinterpret_cast<const uint4*>(raw + swz(tid, c));
+               const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+               for (int e = 0; e < 4; ++e) {
+                 const int i = 4 * c + e;
+                 const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[e]));
+                 const float2 bs = make_float2(__shfl_sync(0xffffffffu, i < 32 ? base_lo.x : base_hi.x, i & 31),
+                                               __shfl_sync(0xffffffffu, i < 32 ? base_lo.y : base_hi.y, i & 31));
+                 const float cs_c = ac[i] * bs.x - as_[i] * bs.y, cs_s = as_[i] * bs.x + ac[i] * bs.y;   // angle addition
+                 const uint32_t rot = pack_bf16(x.x * cs_c - x.y * cs_s, x.x * cs_s + x.y * cs_c);
+                 o[4 * cc + e] = rot;
+               }
+             } else {
+#pragma unroll
+               for (int e = 0; e < 4; ++e) o[4 * cc + e] = 0u;
+             }
+           }
+           if (is_new) {
+             // the new token's rotated key comes from the workspace
+             const uint4* kn = reinterpret_cast<const uint4*>(p.knew + (long)w.b * p.r3) + hf * 8;
+#pragma unroll
+             for (int cc = 0; cc < 8; ++cc)
+               if (hf * 8 + cc < R3C / 8) {
+                 const uint4 v = kn[cc];
+                 o[4 * cc] = v.x; o[4 * cc + 1] = v.y; o[4 * cc + 2] = v.z; o[4 * cc + 3] = v.w;
+               }
+           }
+           tmem_st32(kaddr + (uint32_t)hf * 32u, o);
+         }
+       }
+       tmem_st_wait();
+       if (last) {
+         // as VALUES the new token's un-rotated latent row comes from the workspace and rows past it must be
+         // zero (their probabilities are zero, but the slots may hold anything)
+         if (tid == rnew) {
+           const uint4* vs = reinterpret_cast<const uint4*>(p.vnew + (long)w.b * p.t3);
+           for (int c = 0; c < R3C / 8; ++c) *reinterpret_cast<uint4*>(raw + swz(tid, c)) = vs[c];
+         } else if (tid > rnew) {
+           for (int c = 0; c < R3C / 8; ++c) *reinterpret_cast<uint4*>(raw + swz(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
+         }
+       }
+       tc_fence_before();
+       fence_proxy_async_smem();
+       __syncwarp();
+       if (lane == 0) mbar_arrive(&kr_full[buf]);
+     }
+    }
+   } else if (have_work) {
     pdl_enter();
     // ------------------------------- softmax warpgroups --------------------------
     const int wg = (warp - 4) / 4;              // heads [HPW wg, HPW wg + HPW)
@@ -381,7 +510,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const int buf = it & 1, j = it >> 1;
       const int k0 = w.k0(t), L = w.L;
       const bool last_tile = w.last_tile(t);
-      if (last_tile && wg == 0) {
+      if (!ROT && last_tile && wg == 0) {
         const int s = it % STAGES;
         // the tile holding the new token: its row comes from the workspace, rows past it are invalid
         if (!(ok = wait_all(&full_bar[s], (uint32_t)((it / STAGES) & 1)))) break;
@@ -508,7 +637,7 @@ k_dec_attn_umma(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 128);
+  if (warp == 1) tmem_dealloc(tmem, ROT ? 256 : 128);
 }
 
 }  // namespace decu

@@ -399,7 +399,8 @@ int fast_fwd(Problem& p) {
     gp.seg[2] = seg(d.r2 + d.r3, d.t3, umma_gemm::EP_BF16, w.V, d.t3);
     for (int i = 0; i < 3; ++i) { gp.seg[i].bmap = i; gp.seg[i].b_n_off = 0; }
     if (p.Kc) {
-      gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3;
+      // one shared cache with latent RoPE holds the un-rotated latent rows: only the value segment is copied out
+      if (!p.shared_rope) { gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3; }
       gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
     }
     const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
@@ -547,7 +548,21 @@ size_t carve_fast_dec(const tucker_attn_desc& d, char* base, FastDecWs* w) {
   return c.off;
 }
 
-// The cache-streaming kernel (tcgen05, keys on the M dimension, ranks at run time).
+// The cache-streaming kernel (tcgen05, keys on the M dimension, ranks at run time).  With one shared cache and
+// latent RoPE (p.shared_rope) the instance with the rotation warpgroup runs: the cache holds un-rotated rows.
+template <bool ROT, int R3C>
+int launch_dec_attn_inst(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                         const decu::Params& up, int grid, const dec::RopeFreqs& freqs) {
+  static PerDeviceFlag attr;
+  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)decu::k_dec_attn_umma<ROT, R3C>, (int)decu::SMEM_BYTES));
+  prof_begin(p);
+  (void)launch_pdl(decu::k_dec_attn_umma<ROT, R3C>, dim3(grid), dim3(ROT ? decu::THREADS_ROT : decu::THREADS),
+                   decu::SMEM_BYTES, p.stream, tmK, tmV, tmQ, up, freqs);
+  prof_end(p);
+  TA_LAUNCH_CHECK(p);
+  return TA_OK;
+}
+
 int launch_dec_attn_umma(Problem& p, const CUtensorMap& tmK, const CUtensorMap& tmV, const dec::Params& dp, int grid) {
   const tucker_attn_desc& d = p.d;
   CUtensorMap tmQ;   // Qhat [B * n_H rows, r3]: one box = 32 rows (all heads of a sequence) x 64 columns
@@ -556,13 +571,17 @@ int launch_dec_attn_umma(Problem& p, const CUtensorMap& tmK, const CUtensorMap& 
   up.B = dp.B; up.nH = dp.nH; up.Lmax = dp.Lmax; up.r3 = d.r3; up.t3 = d.t3; up.shared_kv = dp.shared_kv;
   up.cache_len = dp.cache_len; up.knew = dp.knew; up.vnew = dp.vnew;
   up.part_o = dp.part_o; up.part_ml = dp.part_ml; up.err = dp.err;
-  static PerDeviceFlag attr;
-  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)decu::k_dec_attn_umma, (int)decu::SMEM_BYTES));
-  prof_begin(p);
-  (void)launch_pdl(decu::k_dec_attn_umma, dim3(grid), dim3(decu::THREADS), decu::SMEM_BYTES, p.stream, tmK, tmV, tmQ, up);
-  prof_end(p);
-  TA_LAUNCH_CHECK(p);
-  return TA_OK;
+  if (p.shared_rope) {
+    const dec::RopeFreqs freqs = rope_freqs(d);
+    switch (d.r3) {
+      case 64: return launch_dec_attn_inst<true, 64>(p, tmK, tmV, tmQ, up, grid, freqs);
+      case 96: return launch_dec_attn_inst<true, 96>(p, tmK, tmV, tmQ, up, grid, freqs);
+      case 128: return launch_dec_attn_inst<true, 128>(p, tmK, tmV, tmQ, up, grid, freqs);
+      default: return TA_ERR_UNSUPPORTED_SHAPE;
+    }
+  }
+  dec::RopeFreqs none = {};
+  return launch_dec_attn_inst<false, 0>(p, tmK, tmV, tmQ, up, grid, none);
 }
 
 bool dec_rank_ok(int r3, int t3) {
@@ -621,7 +640,7 @@ int fast_decode(Problem& p) {
     auto launch = [&](auto kernel) {
       (void)launch_pdl(kernel, grid, dim3(256), 0, p.stream, w.proj_part, splits, (long)Mpad * ncol, d.n_H, d.r1, d.r2,
                        d.r3, d.t3, (const bf16*)p.C, (const bf16*)p.U1, p.scale * LOG2E, w.qhat, w.knew, w.vnew,
-                       (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.shared_kv, p.dev_err);
+                       (bf16*)p.Kc, (bf16*)p.Vc, p.Lmax, p.cache_len, d.rope, freqs, p.append, p.shared_rope ? 2 : p.shared_kv, p.dev_err);
     };
     switch ((d.r2 + 63) / 64) {
       case 1: launch(dec::k_dec_qhat<1>); break;

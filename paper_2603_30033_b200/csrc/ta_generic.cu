@@ -162,7 +162,7 @@ template <typename T>
 __global__ void k_decode_rope_append(float* __restrict__ knew, const float* __restrict__ vnew,
                                      float* __restrict__ qhat, T* __restrict__ Kc, T* __restrict__ Vc,
                                      const int32_t* __restrict__ cache_len, int B, int nH, int r3, int t3, int Lmax,
-                                     int rope, double base, int append, unsigned int* err) {
+                                     int rope, double base, int append, int shared_rope, unsigned int* err) {
   const int b = blockIdx.x;
   int L = cache_len[b];
   if (L < 0 || L >= Lmax) {
@@ -184,7 +184,9 @@ __global__ void k_decode_rope_append(float* __restrict__ knew, const float* __re
   }
   if (append) {
     __syncthreads();
-    for (int c = threadIdx.x; c < r3; c += blockDim.x) st(Kc + ((long)b * Lmax + L) * r3 + c, knew[(long)b * r3 + c]);
+    // one shared cache with latent RoPE holds un-rotated rows: the value row only
+    if (!shared_rope)
+      for (int c = threadIdx.x; c < r3; c += blockDim.x) st(Kc + ((long)b * Lmax + L) * r3 + c, knew[(long)b * r3 + c]);
     for (int c = threadIdx.x; c < t3; c += blockDim.x) st(Vc + ((long)b * Lmax + L) * t3 + c, vnew[(long)b * t3 + c]);
   }
 }
@@ -296,7 +298,7 @@ __global__ void __launch_bounds__(256) k_attn_decode_generic(const float* __rest
                                                              const T* __restrict__ Kc, const T* __restrict__ Vc,
                                                              const int32_t* __restrict__ cache_len,
                                                              float* __restrict__ o, int nH, int r3, int t3,
-                                                             int Lmax) {
+                                                             int Lmax, int rotate_keys, double base) {
   extern __shared__ float smem[];
   float* qs = smem;
   float* Ks = qs + 8 * r3;
@@ -322,8 +324,16 @@ __global__ void __launch_bounds__(256) k_attn_decode_generic(const float* __rest
       int j = i / r3, c = i % r3;
       int kj = k0 + j;
       float v = 0.f;
-      if (kj < L) v = ld(Kb + (long)kj * r3 + c);
-      else if (kj == L) v = knew[(long)b * r3 + c];
+      if (kj < L) {
+        v = ld(Kb + (long)kj * r3 + c);
+        if (rotate_keys) {
+          // shared cache with latent RoPE: the cached row is un-rotated; its key is the row times R(kj, r3)
+          const float other = ld(Kb + (long)kj * r3 + (c ^ 1));
+          double sn, co;
+          sincos((double)kj * pow(base, -2.0 * (double)(c >> 1) / (double)r3), &sn, &co);
+          v = (c & 1) ? other * (float)sn + v * (float)co : v * (float)co - other * (float)sn;
+        }
+      } else if (kj == L) v = knew[(long)b * r3 + c];
       Ks[j * (r3 + 1) + c] = v;
     }
     for (int i = threadIdx.x; i < 32 * t3; i += 256) {
@@ -448,8 +458,10 @@ int fwd_typed(Problem& p) {
     TA_LAUNCH_CHECK(p);
   }
   if (p.Kc) {
-    k_write_cache<T><<<grid_for((long)T_ * d.r3), 256, 0, p.stream>>>(w.K, (T*)p.Kc, d.B, d.N, d.r3, p.Lmax);
-    TA_LAUNCH_CHECK(p);
+    if (!p.shared_rope) {     // one shared cache with latent RoPE holds the un-rotated rows, i.e. V below
+      k_write_cache<T><<<grid_for((long)T_ * d.r3), 256, 0, p.stream>>>(w.K, (T*)p.Kc, d.B, d.N, d.r3, p.Lmax);
+      TA_LAUNCH_CHECK(p);
+    }
     k_write_cache<T><<<grid_for((long)T_ * d.t3), 256, 0, p.stream>>>(w.V, (T*)p.Vc, d.B, d.N, d.t3, p.Lmax);
     TA_LAUNCH_CHECK(p);
   }
@@ -497,7 +509,7 @@ int decode_typed(Problem& p) {
   }
   k_decode_rope_append<T><<<d.B, 128, 0, p.stream>>>(w.knew, w.vnew, w.qhat, (T*)p.Kc, (T*)p.Vc, p.cache_len, d.B,
                                                     d.n_H, d.r3, d.t3, p.Lmax, d.rope, (double)d.rope_base,
-                                                    p.append, p.dev_err);
+                                                    p.append, p.shared_rope, p.dev_err);
   TA_LAUNCH_CHECK(p);
   {
     size_t smem = attn_smem(d.r3, d.t3);
@@ -505,7 +517,8 @@ int decode_typed(Problem& p) {
     dim3 grid((d.n_H + 7) / 8, d.B);
     prof_begin(p);
     k_attn_decode_generic<T><<<grid, 256, smem, p.stream>>>(w.qhat, w.knew, w.vnew, (const T*)p.Kc, (const T*)p.Vc,
-                                                            p.cache_len, w.o, d.n_H, d.r3, d.t3, p.Lmax);
+                                                            p.cache_len, w.o, d.n_H, d.r3, d.t3, p.Lmax, p.shared_rope,
+                                                            (double)d.rope_base);
     prof_end(p);
     TA_LAUNCH_CHECK(p);
   }

@@ -43,7 +43,7 @@ class Workload:
     rope_base: float
     dtype: str                # "fp32" | "bf16"  (storage type; accumulation is fp32 on the GPU)
     seed: int
-    shared_kv: bool = False   # one latent cache serves keys and values (Ut3 := U3; needs rope == False)
+    shared_kv: bool = False   # one latent cache serves keys and values (Ut3 := U3); with rope it holds un-rotated rows
 
     def asdict(self):
         return asdict(self)
@@ -64,6 +64,9 @@ WORKLOADS = {
         # the decode shape with the paper's shared key / value down-projection (one latent cache, no RoPE)
         Workload("f1_decode_shared_kv", "decode", 64, 32768, 4096, 32, (8, 128, 128), (8, 128, 128),
                  True, False, 500000.0, "bf16", 1005, True),
+        # the same with latent RoPE at position 32768: the one cache holds un-rotated rows, keys are rotated on chip
+        Workload("f1r_decode_shared_kv_rope", "decode", 64, 32768, 4096, 32, (8, 128, 128), (8, 128, 128),
+                 True, True, 500000.0, "bf16", 1006, True),
     ]
 }
 

@@ -339,21 +339,92 @@ def test_prefill_shared_projection_and_cache():
     assert (cache[:, 200:] == 7.0).all()
 
 
-def test_aliased_caches_need_shared_weights_and_no_rope():
+def test_aliased_caches_need_shared_weights():
     import torch
     w = H.custom_workload(kind="decode", dtype="bf16", d_model=256, n_H=8, r=(4, 64, 64), t=(4, 64, 64), rope=True, seed=65)
     wt = _shared_weights(w)
-    dw = H.weights_to_device(wt, "bf16")
-    dw[7] = dw[3]
     Kd = torch.zeros(2, 16, 64, device="cuda", dtype=torch.bfloat16)
     x = torch.zeros(2, 256, device="cuda", dtype=torch.bfloat16)
     ld = torch.zeros(2, dtype=torch.int32, device="cuda")
-    with pytest.raises(Bd.TuckerAttnError) as e:      # latent RoPE: rotated keys cannot double as values
-        Bd.tucker_attn_decode(x, *dw, Kd, Kd, ld, n_H=8, rope=True)
-    assert e.value.status == -1
     dw2 = H.weights_to_device(wt, "bf16")             # distinct U3 / Ut3 tensors: not a shared projection
-    with pytest.raises(Bd.TuckerAttnError):
-        Bd.tucker_attn_decode(x, *dw2, Kd, Kd, ld, n_H=8, rope=False)
+    for rope in (False, True):
+        with pytest.raises(Bd.TuckerAttnError) as e:
+            Bd.tucker_attn_decode(x, *dw2, Kd, Kd, ld, n_H=8, rope=rope)
+        assert e.value.status == -1
+
+
+# --------------------------------------------------------------------------------------
+# shared latent cache WITH latent RoPE (Sec. 3.1 + Definition 2): the one cache holds un-rotated rows
+# --------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype,shape,path", [
+    ("bf16", dict(d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128)), 2),
+    ("bf16", dict(d_model=256, n_H=32, r=(8, 128, 64), t=(8, 32, 64)), 2),
+    ("bf16", dict(d_model=192, n_H=6, r=(3, 96, 96), t=(2, 32, 96)), 2),
+    ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
+])
+@pytest.mark.parametrize("append", [True, False])
+def test_decode_shared_latent_cache_with_rope(dtype, shape, path, append):
+    import torch
+    w = H.custom_workload(kind="decode", dtype=dtype, rope=True, rope_base=500000.0, seed=67, **shape)
+    wt = _shared_weights(w)
+    lens = [0, 1, 127, 128, 129, 300, 650, 1023]
+    Lmax = 1024
+    x, Lc, _, cache_len = W.make_decode_state(w, B=len(lens), L=max(lens), Lmax=Lmax, cache_len=lens)
+    x, Lc = (W.round_to_storage(a, dtype) for a in (x, Lc))
+    ref, l_new = O.tucker_attn_decode_shared_rope(x, wt["C"], wt["U1"], wt["U2"], wt["U3"], wt["Ct"], wt["Ut1"], wt["Ut2"],
+                                                  Lc, cache_len, rope_base=w.rope_base)
+    dw = H.weights_to_device(wt, dtype)
+    dw[7] = dw[3]                                        # the same device tensor for U3 and Ut3
+    Ld = H.to_device(Lc, dtype)
+    for b, L in enumerate(lens):                         # slots from cache_len on are never trusted
+        Ld[b, L:] = float("nan")
+    y = Bd.tucker_attn_decode(H.to_device(x, dtype), *dw, Ld, Ld, torch.from_numpy(cache_len).cuda(), n_H=w.n_H,
+                              rope=True, rope_base=w.rope_base, append=append)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == path
+    check(y.float().cpu().numpy().astype(np.float64), ref, dtype, f"shared cache + RoPE decode {shape}", scaled=True)
+    Lh = Ld.float().cpu().numpy()
+    tol = 1e-5 if dtype == "fp32" else 3e-2
+    for b, L in enumerate(lens):
+        if append:
+            assert np.abs(Lh[b, L] - l_new[b]).max() < tol          # the UN-rotated latent row was appended
+        else:
+            assert np.isnan(Lh[b, L]).all()
+        assert np.array_equal(Lh[b, :L], Lc[b, :L].astype(np.float32))
+
+
+@pytest.mark.parametrize("dtype,shape,path", [
+    ("bf16", dict(d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128)), 2),
+    ("fp32", dict(d_model=64, n_H=4, r=(2, 16, 12), t=(2, 10, 12)), 1),
+])
+def test_prefill_then_decode_with_one_unrotated_cache(dtype, shape, path):
+    # prefill of N tokens writes ONE cache of un-rotated latent rows; a decode step for token N on that cache
+    # equals row N of the prefill over N + 1 tokens
+    import torch
+    N = 200
+    w = H.custom_workload(dtype=dtype, B=2, N=N + 1, causal=True, rope=True, rope_base=10000.0, seed=69, **shape)
+    wt = _shared_weights(w)
+    X = W.round_to_storage(W.make_X(w), dtype)
+    ref, parts = O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=True, rope=True, rope_base=w.rope_base,
+                                   return_parts=True)
+    dw = H.weights_to_device(wt, dtype)
+    dw[7] = dw[3]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    cache = torch.full((2, N + 9, shape["r"][2]), 7.0, device="cuda", dtype=tdt)
+    Y = Bd.tucker_attn_fwd(H.to_device(X[:, :N], dtype), *dw, n_H=w.n_H, causal=True, rope=True, rope_base=w.rope_base,
+                           Kcache=cache, Vcache=cache)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == path
+    check(Y.float().cpu().numpy().astype(np.float64), ref[:, :N], dtype, f"shared projection + RoPE prefill {shape}",
+          scaled=True)
+    tol = 1e-5 if dtype == "fp32" else 3e-2
+    for b in range(2):
+        assert np.abs(cache[b, :N].float().cpu().numpy() - parts[b]["V"][:N]).max() < tol     # un-rotated rows
+    assert (cache[:, N:] == 7.0).all()
+    lens = torch.full((2,), N, dtype=torch.int32, device="cuda")
+    y = Bd.tucker_attn_decode(H.to_device(X[:, N], dtype), *dw, cache, cache, lens, n_H=w.n_H, rope=True,
+                              rope_base=w.rope_base, append=True)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == path
+    check(y.float().cpu().numpy().astype(np.float64), ref[:, N], dtype, f"decode after that prefill {shape}", scaled=True)
 
 
 def test_decode_garbage_beyond_cache_len_is_ignored():
