@@ -435,6 +435,47 @@ def bench_pack(torch, Bd, peaks, steps=10):
                          "kernel_ms": ms, "whole_step_frac_of_peak": ach / peaks["hbm_gbs"]}}
 
 
+def bench_hosvd(torch, Bd, peaks, steps=3):
+    """Next row f-4: HOSVD initialiser on synthetic low-rank-plus-noise MHA weights of the c2 layer shape
+    (d = 768, 12 heads), ranks (12, 64, 64).  The dominant kernels are the two d x d Gram matrices of the
+    mode unfoldings, one bf16 tensor-core GEMM each with K = 3 n_H d (high / low split of the fp32 tensor)."""
+    d, n_H, ranks = 768, 12, (12, 64, 64)
+    wm = W.make_lowrank_mha(d, n_H, 64, 0.02, 1200)
+    dev = [torch.from_numpy(np.ascontiguousarray(wm[k], dtype=np.float32)).cuda() for k in ("WQ", "WK", "WV", "WO")]
+    Wt, _ = Bd.tucker_mha_weight_tensors(*dev, n_H=n_H)
+    ws = Bd.alloc_workspace(load_hosvd_ws(Bd, d, n_H, ranks), Wt.device)
+    times, ktimes = [], []
+    for i in range(steps + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        k0.record(); k1.record()
+        Bd.set_profile_events(k0, k1)
+        e0.record()
+        Bd.tucker_hosvd_init(Wt, ranks, workspace=ws)
+        e1.record()
+        Bd.set_profile_events()
+        torch.cuda.synchronize()
+        if i >= 1:
+            times.append(e0.elapsed_time(e1))
+            ktimes.append(k0.elapsed_time(k1))
+    assert Bd.last_device_error() == 0
+    launches = Bd.last_launch_count()
+    ms, kms = sum(times) / len(times), sum(ktimes) / len(ktimes)
+    gram_flops_bf16 = 2.0 * d * d * (3 * n_H * d)          # executed on the tensor cores by one Gram GEMM
+    ach = gram_flops_bf16 / (kms * 1e-3) / 1e12
+    return {"workload": "f4_hosvd_init_gpt2_layer", "unit": "ms", "value": ms, "ms_per_step": ms,
+            "gpu_launches_per_step": launches, "l2": "one tensor of 28 MB, resident",
+            "roofline": {"kernel": "Gram matrix of a mode unfolding (k_umma_gemm, bf16 high/low split, split-K fp32 partials)",
+                         "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": ach / peaks["bf16_tflops"], "traffic": None, "kernel_ms": kms,
+                         "flops_per_launch": gram_flops_bf16, "algorithmic_fp32_flops_per_launch": gram_flops_bf16 / 3,
+                         "whole_step_frac_of_peak": None}}
+
+
+def load_hosvd_ws(Bd, d, n_H, ranks):
+    return int(Bd.load_library().tucker_hosvd_workspace_bytes(int(d), int(n_H), int(ranks[1]), int(ranks[2])))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -500,6 +541,8 @@ def main():
             others.append(o)
         torch.cuda.empty_cache()
         others.append(bench_pack(torch, Bd, peaks))
+        torch.cuda.empty_cache()
+        others.append(bench_hosvd(torch, Bd, peaks))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

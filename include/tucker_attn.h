@@ -222,6 +222,37 @@ TA_API int tucker_pack_mla(int32_t d_model, int32_t n_H, int32_t dcq, int32_t dc
                     void* C, void* U1, void* U2, void* U3, void* Ct, void* Ut1, void* Ut2, void* Ut3,
                     void* cuda_stream);
 
+/*
+ * HOSVD initialiser: pretrained MHA weights -> Tucker-attention weights (App. C.1, paragraph "MHA to Tucker
+ * Attention": a higher-order SVD of the n_H x d x d weight tensors), with the singular spectra of the three mode
+ * unfoldings that Sec. 2.1 ("Informed Compression Across All Modes") uses to choose the ranks.  fp32 throughout;
+ * all pointers caller-owned device memory; asynchronous on `cuda_stream`; no host synchronisation.
+ *
+ * tucker_mha_weight_tensors: W[i] = WQ_i WK_i^T and Wt[i] = (WV_i WO_i)^T (Eqs. 2-3: the per-head matrices,
+ * the second stack transposed so that mode 2 is the output and mode 3 the value mode), both [n_H, d, d], from
+ * WQ, WK, WV [d, d] (heads = column blocks of width d / n_H) and WO [d, d] (head i = rows i d_H ..).
+ *
+ * tucker_hosvd_init: for one tensor W [n_H, d, d] and ranks (r1, r2, r3), 1 <= r1 <= n_H <= 64, r2, r3 <= d <= 8192:
+ *   U_j [n_j, r_j]   the r_j leading left singular vectors of the mode-j unfolding (orthonormal columns, each with
+ *                    its largest component positive), from the eigenvectors of the Gram matrix Mat_j Mat_j^T
+ *   C [r1, r2, r3]   the core W x_1 U1^T x_2 U2^T x_3 U3^T
+ *   spectra          optional [n_H + 2 d]: all singular values of the mode-1, mode-2 and mode-3 unfoldings, each
+ *                    block descending (divide by the first entry of a block for the normalised spectrum)
+ * so that W ~ C x_1 U1 x_2 U2 x_3 U3 with squared error <= the sum of the squared truncated singular values.
+ * Call it once for the pre-softmax tensor (-> C, U1, U2, U3) and once for the post-softmax tensor (-> Ct, Ut1,
+ * Ut2, Ut3).  The two d-sized Gram matrices run on the tensor cores when d is a multiple of 64 (bf16 high / low
+ * split, fp32 accumulation, about 2^-16 relative), else on fp32 FMA kernels; eigenvectors by one-sided Jacobi
+ * sweeps in fp32.  Singular values below about 1e-3 of the largest are at the noise level of that arithmetic.
+ * workspace: >= tucker_hosvd_workspace_bytes(d_model, n_H, r2, r3) bytes, 256-byte aligned.
+ * Returns TA_OK, TA_ERR_INVALID_ARG, TA_ERR_WORKSPACE_TOO_SMALL, TA_ERR_UNSUPPORTED_SHAPE or TA_ERR_CUDA.
+ */
+TA_API size_t tucker_hosvd_workspace_bytes(int32_t d_model, int32_t n_H, int32_t r2, int32_t r3);
+TA_API int tucker_hosvd_init(int32_t d_model, int32_t n_H, int32_t r1, int32_t r2, int32_t r3, const float* W,
+                      float* C, float* U1, float* U2, float* U3, float* spectra,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+TA_API int tucker_mha_weight_tensors(int32_t d_model, int32_t n_H, const float* WQ, const float* WK,
+                              const float* WV, const float* WO, float* W, float* Wt, void* cuda_stream);
+
 /* Human-readable name of a status code (static storage). */
 TA_API const char* tucker_attn_status_string(int status);
 

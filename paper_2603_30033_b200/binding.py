@@ -30,6 +30,7 @@ EXPORTS = (
     "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout", "tucker_attn_sync_status",
     "tucker_attn_bounds_checked",
     "tucker_pack_gqa", "tucker_pack_mha", "tucker_pack_mla",
+    "tucker_hosvd_workspace_bytes", "tucker_hosvd_init", "tucker_mha_weight_tensors",
 )
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -96,6 +97,12 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_pack_mha.argtypes = [i32] * 3 + [vp] * 13
     lib.tucker_pack_mla.restype = ctypes.c_int
     lib.tucker_pack_mla.argtypes = [i32] * 5 + [vp] * 16
+    lib.tucker_hosvd_workspace_bytes.restype = sz
+    lib.tucker_hosvd_workspace_bytes.argtypes = [i32] * 4
+    lib.tucker_hosvd_init.restype = ctypes.c_int
+    lib.tucker_hosvd_init.argtypes = [i32] * 5 + [vp] * 7 + [sz, vp]
+    lib.tucker_mha_weight_tensors.restype = ctypes.c_int
+    lib.tucker_mha_weight_tensors.argtypes = [i32] * 2 + [vp] * 7
     _lib = lib
     return lib
 
@@ -366,6 +373,55 @@ def tucker_pack_mla(WDQ, WUQ, WDKV, WUK, WDV, WUV, WO, *, n_H: int, out=None):
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_pack_mla")
     return outs
+
+
+def tucker_mha_weight_tensors(WQ, WK, WV, WO, *, n_H: int):
+    """The two n_H x d x d weight tensors of MHA weights (fp32): W[i] = WQ_i WK_i^T, Wt[i] = (WV_i WO_i)^T."""
+    torch = _torch()
+    d = WQ.shape[0]
+    dev = WQ.device
+    if d % n_H:
+        raise ValueError("d_model must be a multiple of n_H")
+    for name, t in (("WQ", WQ), ("WK", WK), ("WV", WV), ("WO", WO)):
+        _check(t, name, (d, d), torch.float32, dev)
+    W = torch.empty(n_H, d, d, dtype=torch.float32, device=dev)
+    Wt = torch.empty_like(W)
+    with torch.cuda.device(dev):
+        rc = load_library().tucker_mha_weight_tensors(int(d), int(n_H), WQ.data_ptr(), WK.data_ptr(), WV.data_ptr(),
+                                                      WO.data_ptr(), W.data_ptr(), Wt.data_ptr(), _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_mha_weight_tensors")
+    return W, Wt
+
+
+def tucker_hosvd_init(W, ranks, *, workspace=None):
+    """HOSVD of one weight tensor W [n_H, d, d] (fp32): returns (C [r1, r2, r3], U1 [n_H, r1], U2 [d, r2],
+    U3 [d, r3], spectra), spectra = the singular values of the mode-1, mode-2 and mode-3 unfoldings
+    ([n_H], [d], [d], each descending)."""
+    torch = _torch()
+    lib = load_library()
+    if W.dim() != 3 or W.shape[1] != W.shape[2]:
+        raise ValueError("W must be [n_H, d, d]")
+    n_H, d, _ = W.shape
+    dev = W.device
+    _check(W, "W", (n_H, d, d), torch.float32, dev)
+    r1, r2, r3 = (int(r) for r in ranks)
+    f = dict(dtype=torch.float32, device=dev)
+    C, U1 = torch.empty(r1, r2, r3, **f), torch.empty(n_H, r1, **f)
+    U2, U3 = torch.empty(d, r2, **f), torch.empty(d, r3, **f)
+    spectra = torch.empty(n_H + 2 * d, **f)
+    need = int(lib.tucker_hosvd_workspace_bytes(int(d), int(n_H), r2, r3))
+    if need == 0:
+        raise ValueError("invalid sizes for tucker_hosvd_init")
+    if workspace is None:
+        workspace = alloc_workspace(need, dev)
+    with torch.cuda.device(dev):
+        rc = lib.tucker_hosvd_init(int(d), int(n_H), r1, r2, r3, W.data_ptr(), C.data_ptr(), U1.data_ptr(), U2.data_ptr(),
+                                   U3.data_ptr(), spectra.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                   _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_hosvd_init")
+    return C, U1, U2, U3, (spectra[:n_H], spectra[n_H:n_H + d], spectra[n_H + d:])
 
 
 def selftest_wait_timeout(budget_us: int = 2000, device=None):

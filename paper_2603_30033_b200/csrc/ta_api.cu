@@ -173,6 +173,46 @@ int tucker_attn_last_device_error(void* cuda_stream) {
   return (int)host;
 }
 
+static bool hosvd_args_ok(int32_t d, int32_t nH, int32_t r1, int32_t r2, int32_t r3) {
+  return d > 0 && d <= 8192 && nH > 0 && nH <= 64 && r1 >= 1 && r1 <= nH && r2 >= 1 && r2 <= d && r3 >= 1 && r3 <= d;
+}
+
+size_t tucker_hosvd_workspace_bytes(int32_t d_model, int32_t n_H, int32_t r2, int32_t r3) {
+  if (!hosvd_args_ok(d_model, n_H, 1, r2, r3)) return 0;
+  return hosvd_workspace(n_H, d_model, d_model, r2, r3);
+}
+
+int tucker_hosvd_init(int32_t d_model, int32_t n_H, int32_t r1, int32_t r2, int32_t r3, const float* W, float* C,
+                      float* U1, float* U2, float* U3, float* spectra, void* workspace, size_t workspace_bytes,
+                      void* cuda_stream) {
+  if (!hosvd_args_ok(d_model, n_H, r1, r2, r3)) return TA_ERR_INVALID_ARG;
+  if (!W || !C || !U1 || !U2 || !U3 || !workspace) return TA_ERR_INVALID_ARG;
+  if (!aligned16(W) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TA_ERR_INVALID_ARG;
+  if (workspace_bytes < hosvd_workspace(n_H, d_model, d_model, r2, r3)) return TA_ERR_WORKSPACE_TOO_SMALL;
+  Problem p = {};
+  p.ws = static_cast<char*>(workspace); p.ws_bytes = workspace_bytes;
+  p.stream = static_cast<cudaStream_t>(cuda_stream);
+  p.dev_err = device_error_ptr();
+  p.prof_start = tl_prof_start; p.prof_stop = tl_prof_stop;
+  if (!p.dev_err) return TA_ERR_CUDA;
+  const int rc = hosvd_run(p, n_H, d_model, d_model, r1, r2, r3, W, C, U1, U2, U3, spectra);
+  tl_last_path = 2;
+  tl_last_launches = p.launches;
+  return rc;
+}
+
+int tucker_mha_weight_tensors(int32_t d_model, int32_t n_H, const float* WQ, const float* WK, const float* WV,
+                              const float* WO, float* W, float* Wt, void* cuda_stream) {
+  if (d_model <= 0 || n_H <= 0 || d_model % n_H || !WQ || !WK || !WV || !WO || !W || !Wt) return TA_ERR_INVALID_ARG;
+  Problem p = {};
+  p.stream = static_cast<cudaStream_t>(cuda_stream);
+  p.dev_err = device_error_ptr();
+  if (!p.dev_err) return TA_ERR_CUDA;
+  const int rc = mha_weight_tensors_run(p, d_model, n_H, WQ, WK, WV, WO, W, Wt);
+  tl_last_launches = p.launches;
+  return rc;
+}
+
 int tucker_attn_sync_status(void* cuda_stream) {
   const int word = tucker_attn_last_device_error(cuda_stream);
   if (word < 0) return word;

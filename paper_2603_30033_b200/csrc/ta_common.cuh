@@ -73,6 +73,21 @@ size_t fast_decode_workspace(const tucker_attn_desc& d, int32_t Lmax);
 int fast_decode(Problem& p);
 int wait_selftest(unsigned int* dev_err, int budget_us, int* out_dev, cudaStream_t stream);
 
+// Tensor-core GEMM with fp32 split-K partial outputs (ta_fast.cu): for z < splits,
+//   out[z * split_stride + row * N + col] = sum over the z-th share of K of A[row, k] B[col, k],
+// A [M, K] and B [N, K] bf16 with K contiguous (leading dimensions lda, ldb), K a multiple of 64 whose
+// 64-blocks divide evenly by `splits`, N a multiple of 64; rows >= M of a 128-row tile are not written.
+// Uses p.stream, p.dev_err, p.launches only.
+int umma_gemm_f32_partials(Problem& p, const bf16* A, long lda, int M, const bf16* B, long ldb, int N, int K, int splits,
+                           float* out, long split_stride);
+
+// HOSVD initialiser (ta_hosvd.cu)
+size_t hosvd_workspace(int n1, int n2, int n3, int r2, int r3);
+int hosvd_run(Problem& p, int n1, int n2, int n3, int r1, int r2, int r3, const float* T, float* core, float* U1,
+              float* U2, float* U3, float* spectra);
+int mha_weight_tensors_run(Problem& p, int d, int nH, const float* WQ, const float* WK, const float* WV, const float* WO,
+                           float* W, float* Wt);
+
 // Programmatic dependent launch.  Every kernel of the tensor-core paths starts with pdl_enter():
 // it waits until the preceding kernels of the stream have completed and their writes are visible,
 // and only then lets the next kernel of the stream be scheduled.  Launched through launch_pdl, a

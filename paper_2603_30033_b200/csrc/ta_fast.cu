@@ -470,6 +470,18 @@ int fast_fwd(Problem& p) {
   return TA_OK;
 }
 
+int umma_gemm_f32_partials(Problem& p, const bf16* A, long lda, int M, const bf16* B, long ldb, int N, int K, int splits,
+                           float* out, long split_stride) {
+  if (K % 64 || N % 64 || splits < 1 || (K / 64) % splits) return TA_ERR_UNSUPPORTED_SHAPE;
+  umma_gemm::Params gp = {};
+  gp.nseg = 1;
+  gp.seg[0] = seg(0, N, umma_gemm::EP_F32, out, N);
+  gp.kb_per_split = (K / 64) / splits;
+  gp.split_stride = split_stride;
+  const BOperand bop = {B, ldb, N};
+  return launch_gemm(p, A, lda, M, K, &bop, 1, N, pick_bn(N), gp, splits);
+}
+
 // ---------------------------------------------------------------------------------------------
 // decode
 // ---------------------------------------------------------------------------------------------

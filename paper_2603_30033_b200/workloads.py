@@ -244,3 +244,18 @@ def decode_flops(w: Workload, B: int | None = None, L: int | None = None) -> int
     other = 2 * B * d * (r2 + r3 + t3) + 2 * B * nH * (r2 * r3 + t3 * t2) + 2 * B * t2 * d \
         + 2 * nH * (r1 * r2 * r3 + t1 * t2 * t3)
     return attn + other
+
+
+def make_lowrank_mha(d: int, n_H: int, rank: int, noise: float, seed: int) -> dict:
+    """Synthetic MHA weights WQ, WK, WV, WO [d, d] whose per-head products have a dominant shared rank-`rank`
+    structure plus Gaussian noise of relative size `noise` (stand-in for pretrained weights, whose spectra decay;
+    input of the HOSVD initialiser).  Every head's query / key / value columns are mixtures of `rank` common
+    directions, so the three unfoldings of the weight tensors have `rank` (modes 2, 3) large singular values."""
+    out = {}
+    for idx, name in enumerate(("WQ", "WK", "WV", "WO")):
+        rng = _rng(seed, 20 + idx)
+        basis = orthonormal_factor(rng, d, rank)                       # common directions
+        mix = rng.standard_normal((rank, d)) / np.sqrt(rank)
+        Wm = basis @ mix if name != "WO" else (basis @ mix).T
+        out[name] = Wm + noise * rng.standard_normal((d, d)) / np.sqrt(d)
+    return out
