@@ -472,6 +472,23 @@ def bench_hosvd(torch, Bd, peaks, steps=3):
                          "whole_step_frac_of_peak": None}}
 
 
+def bench_plane_mix(torch, Bd):
+    """Row f-2 (core-factorised scores), priced instead of built: the mixing of r1 = 8 score planes into the two
+    score tiles of a head pair, alone, at the tile count of the long causal prefill (66560 [128 x 128] tiles of
+    head pairs over 148 SMs = 450 per SM), against the tensor-core cycles per tile that the form could save."""
+    cyc, ms = Bd.probe_plane_mix(450, 8, 148)
+    # what the form replaces: per head pair and tile 2 score MMAs of 128 x 128 x 128 (about 560 cycles each at the
+    # measured 70 cycles per K = 16 step); with r1 = 8 planes and n_H = 32 heads it would issue 8 / 16 of them
+    saved = 2 * 8 * 70.0 * (1.0 - 8.0 / 32.0)
+    return {"workload": "f2_plane_mix_probe", "unit": "cycles/tile", "value": cyc, "ms_per_step": ms,
+            "gpu_launches_per_step": 1, "l2": "n/a",
+            "note": f"mixing alone: {cyc:.0f} cycles per tile and head pair in the softmax warps; tensor-core cycles "
+                    f"it could save per tile and head pair: at most {saved:.0f}, on a tensor pipe that is half idle",
+            "roofline": {"kernel": "plane mixing S_h = sum_a U1[h,a] P_a (FMA pipe)", "bound": "alu", "achieved": None,
+                         "peak": None, "unit": "cycles/tile", "frac": None, "traffic": None, "kernel_ms": ms,
+                         "whole_step_frac_of_peak": None}}
+
+
 def load_hosvd_ws(Bd, d, n_H, ranks):
     return int(Bd.load_library().tucker_hosvd_workspace_bytes(int(d), int(n_H), int(ranks[1]), int(ranks[2])))
 
@@ -543,6 +560,7 @@ def main():
         others.append(bench_pack(torch, Bd, peaks))
         torch.cuda.empty_cache()
         others.append(bench_hosvd(torch, Bd, peaks))
+        others.append(bench_plane_mix(torch, Bd))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -319,6 +319,18 @@ TA_API int tucker_attn_last_launch_count(void);
  */
 TA_API int tucker_attn_set_profile_events(void* ev_start, void* ev_stop);
 
+/*
+ * Measurement probe (no counterpart in the paper's experiments; it prices the kernel that Sec. 3.3 leaves to
+ * future work, scores formed from the factorised core as S_h = sum_a U1[h, a] (Qt C_a K^T)).  Runs ONLY the
+ * step that form would add to the softmax warps -- mixing r1 plane tiles into the score tiles of a head pair,
+ * r1 multiply-adds per score and head -- for `tiles` [128 x 128] tiles per block on `n_blocks` blocks of 256
+ * threads (one per SM is the attention kernel's occupancy).  u1 [2, r1] fp32 mixing weights; cycles
+ * [n_blocks] receives each block's clock64 count for the loop; sink [n_blocks * 256] receives checksums.
+ * All device memory, caller-owned.  Returns TA_OK, TA_ERR_INVALID_ARG (r1 > 16, null pointers) or TA_ERR_CUDA.
+ */
+TA_API int tucker_probe_plane_mix(int32_t tiles, int32_t r1, int32_t n_blocks, const float* u1, long long* cycles,
+                           float* sink, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

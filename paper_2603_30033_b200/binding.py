@@ -30,7 +30,7 @@ EXPORTS = (
     "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout", "tucker_attn_sync_status",
     "tucker_attn_bounds_checked",
     "tucker_pack_gqa", "tucker_pack_mha", "tucker_pack_mla",
-    "tucker_hosvd_workspace_bytes", "tucker_hosvd_init", "tucker_mha_weight_tensors",
+    "tucker_hosvd_workspace_bytes", "tucker_hosvd_init", "tucker_mha_weight_tensors", "tucker_probe_plane_mix",
 )
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_hosvd_init.argtypes = [i32] * 5 + [vp] * 7 + [sz, vp]
     lib.tucker_mha_weight_tensors.restype = ctypes.c_int
     lib.tucker_mha_weight_tensors.argtypes = [i32] * 2 + [vp] * 7
+    lib.tucker_probe_plane_mix.restype = ctypes.c_int
+    lib.tucker_probe_plane_mix.argtypes = [i32] * 3 + [vp] * 4
     _lib = lib
     return lib
 
@@ -422,6 +424,28 @@ def tucker_hosvd_init(W, ranks, *, workspace=None):
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_hosvd_init")
     return C, U1, U2, U3, (spectra[:n_H], spectra[n_H:n_H + d], spectra[n_H + d:])
+
+
+def probe_plane_mix(tiles: int, r1: int, n_blocks: int = 148):
+    """Runs the plane-mixing probe (see tucker_probe_plane_mix); returns (median cycles per tile over the
+    blocks, kernel milliseconds by CUDA events)."""
+    torch = _torch()
+    dev = torch.device("cuda", torch.cuda.current_device())
+    u1 = torch.randn(2, r1, device=dev, dtype=torch.float32)
+    cycles = torch.zeros(n_blocks, dtype=torch.int64, device=dev)
+    sink = torch.zeros(n_blocks * 256, dtype=torch.float32, device=dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ms = 0.0
+    for _ in range(2):      # the second run is the measured one
+        e0.record()
+        rc = load_library().tucker_probe_plane_mix(int(tiles), int(r1), int(n_blocks), u1.data_ptr(), cycles.data_ptr(),
+                                                   sink.data_ptr(), _stream_ptr(dev))
+        e1.record()
+        if rc != TA_OK:
+            raise TuckerAttnError(rc, "tucker_probe_plane_mix")
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+    return float(cycles.median().item()) / tiles, ms
 
 
 def selftest_wait_timeout(budget_us: int = 2000, device=None):
