@@ -34,18 +34,36 @@ import numpy as np
 from paper_2603_30033_b200 import workloads as W
 
 LIB_FLAGS = 0   # TA_FLAG_* bits for every library call (set from --flags)
+SUSTAINED_SECONDS = 0.0   # length of the sustained leg of the main workload (set from --sustained)
 
 METRIC = "prefill TFLOP/s & decode GB/s vs B200 roofline (fused Tucker attention)"
 KEYS = ("C", "U1", "U2", "U3", "Ct", "Ut1", "Ut2", "Ut3")
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on
-# this workload (profiles/).  A value is only listed while the kernel is unchanged since its capture.
-NCU_TRAFFIC_BYTES = {
-    "c4_long_prefill": 17.99e6 + 77.25e6,     # attn::k_attn_prefill, profiles/k_attn_prefill_c4_long_prefill.md
-    "c3_vit_prefill": 34.02e6 + 64.90e6,      # attn::k_attn_prefill, profiles/k_attn_prefill_c3_vit_prefill.md
-    "c5_decode": 1075.34e6 + 4.56e6,          # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_c5_decode.md
-    "f1_decode_shared_kv": 538.05e6 + 4.87e6,  # decu::k_dec_attn_umma, profiles/k_dec_attn_umma_f1_decode_shared_kv.md
+# DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on this
+# workload: value, the summary under profiles/ it comes from, and the SHA-256 of the kernel's source file at the
+# time of the capture.  A value is only reported while that file is unchanged (see ncu_traffic()).
+NCU_TRAFFIC = {
 }
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # the figures the targets are quoted against
+
+
+def ncu_traffic(workload: str):
+    """(bytes per launch or None, provenance string)."""
+    import hashlib
+    rec = NCU_TRAFFIC.get(workload)
+    if not rec:
+        return None, "no ncu capture for this workload"
+    path = os.path.join(ROOT, "paper_2603_30033_b200", "csrc", rec["source"])
+    try:
+        with open(path, "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None, f"{rec['source']} not found"
+    if digest != rec["sha256"]:
+        return None, f"{rec['source']} changed since the capture in {rec['profile']}"
+    return rec["bytes"], f"{rec['profile']} ({rec['source']} unchanged since)"
+
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -168,6 +186,39 @@ def time_steps(torch, Bd, step_fn, steps, warmup, flush, barrier, profile=False)
     return ms, kms, (t0, t1)
 
 
+def sustained_leg(torch, step_fn, seconds, gpu_index, work, div, peak_sustained):
+    """Repeats the step back to back for at least `seconds` (the burst numbers above last tens of
+    milliseconds, during which the SM clock stays at its maximum; under a seconds-long load the power cap pulls
+    it down).  Reports ms per step, the median SM clock sampled meanwhile and their product."""
+    sampler = ClockSampler(gpu_index)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_fn()
+    torch.cuda.synchronize()
+    sampler.start()
+    time.sleep(0.3)
+    t0 = time.time()
+    n = 0
+    e0.record()
+    while True:
+        for _ in range(50):
+            step_fn()
+        n += 50
+        if n % 200 == 0:
+            torch.cuda.synchronize()
+            if time.time() - t0 >= seconds:
+                break
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0 + 0.5, t1)
+    ms = e0.elapsed_time(e1) / n
+    value = work / (ms * 1e-3) / div
+    return {"seconds": t1 - t0, "steps": n, "ms_per_step": ms, "value": value, "sm_mhz_median": clocks["sm_mhz"],
+            "reasons": clocks["reasons"], "ms_times_mhz": ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+            "peak_sustained": peak_sustained, "frac_of_sustained_peak": (value / peak_sustained) if peak_sustained else None,
+            "note": "inputs stay in L2 between steps where they fit; no flush in this leg"}
+
+
 def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sampler=None):
     wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
     dw = [_dev(wt[k], w.dtype, torch) for k in KEYS]
@@ -212,10 +263,16 @@ def bench_prefill(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sa
     res["roofline"] = {
         "kernel": ("attention (per-head queries + scores + online softmax + PV)" if fused_q
                    else "attention (scores + online softmax + PV)"), "bound": "tensor", "achieved": ach, "peak": peak,
-        "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": NCU_TRAFFIC_BYTES.get(w.name), "kernel_ms": kms_avg,
+        "unit": "TFLOP/s", "frac": (ach / peak) if peak else None, "traffic": ncu_traffic(w.name)[0],
+        "traffic_source": ncu_traffic(w.name)[1], "kernel_ms": kms_avg,
         "flops_per_launch": attn_flops, "whole_step_frac_of_peak": (res["value"] / peak) if peak else None,
+        "frac_of_nominal": ach / NOMINAL_PEAKS["bf16_tflops"],
+        "whole_step_frac_of_nominal": res["value"] / NOMINAL_PEAKS["bf16_tflops"],
     }
     res["clocks"] = clocks
+    if SUSTAINED_SECONDS > 0 and sampler is not None:
+        res["sustained"] = sustained_leg(torch, step, SUSTAINED_SECONDS, sampler.gpu, fl["total"], 1e12,
+                                         peaks.get("bf16_tflops_sustained"))
     if with_e2e:
         def e2e_step():
             X.copy_(X_host, non_blocking=True)
@@ -277,9 +334,11 @@ def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sam
     ach = by["cache"] / (kms_avg * 1e-3) / 1e9
     res["roofline"] = {
         "kernel": "decode attention over the latent KV cache", "bound": "hbm", "achieved": ach,
-        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-        "kernel_ms": kms_avg, "bytes_per_launch": by["cache"],
+        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": ncu_traffic(w.name)[0],
+        "traffic_source": ncu_traffic(w.name)[1], "kernel_ms": kms_avg, "bytes_per_launch": by["cache"],
         "whole_step_frac_of_peak": res["value"] / peaks["hbm_gbs"],
+        "frac_of_nominal": ach / NOMINAL_PEAKS["hbm_gbs"],
+        "whole_step_frac_of_nominal": res["value"] / NOMINAL_PEAKS["hbm_gbs"],
     }
     res["clocks"] = clocks
     if with_e2e:
@@ -503,9 +562,12 @@ def main():
     ap.add_argument("--no-others", action="store_true", help="skip the secondary workloads")
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="TA_FLAG_* bits passed to the library (route selection)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained", type=float, default=2.0,
+                    help="seconds of back-to-back steps for the sustained-clock leg of a prefill workload (0 = skip)")
     args = ap.parse_args()
-    global LIB_FLAGS
+    global LIB_FLAGS, SUSTAINED_SECONDS
     LIB_FLAGS = args.flags
+    SUSTAINED_SECONDS = args.sustained
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -528,6 +590,19 @@ def main():
             dist.barrier()
 
     peaks, peak_kind = load_peaks()
+    if args.workload in ("f2", "f3", "f4"):
+        # the widened rows that are not layer steps: the plane-mixing probe, the weight packers, the HOSVD initialiser
+        o = {"f2": lambda: bench_plane_mix(torch, Bd), "f3": lambda: bench_pack(torch, Bd, peaks),
+             "f4": lambda: bench_hosvd(torch, Bd, peaks)}[args.workload]()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": o["value"], "unit": o["unit"], "n_gpus": world, "steps": args.steps,
+                              "warmup": args.warmup, "ms_per_step": o["ms_per_step"], "higher_is_better": o["unit"] != "ms",
+                              "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                              "config": {"workload": o["workload"]}, "roofline": o["roofline"], "cpu_baseline": None,
+                              "gpu_launches": o["gpu_launches_per_step"], "note": o.get("note")}))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     w = W.get_workload(args.workload)
     fn = bench_prefill if w.kind == "prefill" else bench_decode
     gpu_index = local_rank
@@ -574,7 +649,8 @@ def main():
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, **_cfg(w), "l2": res["l2"],
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "roofline": res["roofline"], "cpu_baseline": cpu_baseline, "clocks": res["clocks"],
+            "roofline": res["roofline"], "sustained": res.get("sustained"), "cpu_baseline": cpu_baseline,
+            "clocks": res["clocks"],
             "e2e": {**res["e2e"], "value": e2e_value, "ms_per_step": e2e_ms},
             "gpu_launches": res["gpu_launches_per_step"] * args.steps, "path": res["path"],
             "ms_best": res["ms_best"], "other_workloads": others,

@@ -100,6 +100,8 @@ FAST = [
     dict(B=2, N=300, d_model=320, n_H=5, r=(5, 64, 64), t=(5, 32, 64), causal=True, rope=True),
     dict(B=2, N=150, d_model=256, n_H=4, r=(2, 128, 64), t=(2, 64, 96), causal=False, rope=True),
     dict(B=1, N=64, d_model=192, n_H=6, r=(3, 96, 96), t=(3, 96, 96), causal=True, rope=True),
+    # wide model: the projection GEMM reads K-major copies of the factors
+    dict(B=1, N=150, d_model=2048, n_H=16, r=(4, 64, 96), t=(4, 64, 32), causal=True, rope=True),
 ]
 
 
@@ -321,9 +323,10 @@ def test_decode_shared_latent_cache(dtype, shape, path):
         assert np.array_equal(Kh[b, :L], Kc[b, :L].astype(np.float32))
 
 
-def test_prefill_shared_projection_and_cache():
+@pytest.mark.parametrize("d_model", [256, 2048])
+def test_prefill_shared_projection_and_cache(d_model):
     import torch
-    w = H.custom_workload(dtype="bf16", B=2, N=200, d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128), causal=True,
+    w = H.custom_workload(dtype="bf16", B=2, N=200, d_model=d_model, n_H=8, r=(4, 64, 128), t=(4, 64, 128), causal=True,
                           rope=False, seed=63)
     wt = _shared_weights(w)
     X = W.round_to_storage(W.make_X(w), w.dtype)
