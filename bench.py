@@ -42,7 +42,16 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on this
 # workload: value, the summary under profiles/ it comes from, and the SHA-256 of the kernel's source file at the
 # time of the capture.  A value is only reported while that file is unchanged (see ncu_traffic()).
+_ATTN = {"source": "ta_attn_prefill.cuh", "sha256": "d6ed99eafcf2f1fa097944519b95002d1e655e58ca03f7790f1fba0f790efc6a"}
+_DEC = {"source": "ta_decode_umma.cuh", "sha256": "b29368639f2d9ea4a252a55117459bd2a1a167eff6dc63668ccc285447534b03"}
 NCU_TRAFFIC = {
+    "c4_long_prefill": {"bytes": 17916160 + 77050880, "profile": "profiles/k_attn_prefill_c4_long_prefill.md", **_ATTN},
+    "c3_vit_prefill": {"bytes": 33788928 + 64443648, "profile": "profiles/k_attn_prefill_c3_vit_prefill.md", **_ATTN},
+    "c2_gpt2_prefill": {"bytes": 3593472 + 0, "profile": "profiles/k_attn_prefill_c2_gpt2_prefill.md", **_ATTN},
+    "c5_decode": {"bytes": 1075363072 + 4196608, "profile": "profiles/k_dec_attn_umma_c5_decode.md", **_DEC},
+    "f1_decode_shared_kv": {"bytes": 537998592 + 4850688, "profile": "profiles/k_dec_attn_umma_f1_decode_shared_kv.md", **_DEC},
+    "f1r_decode_shared_kv_rope": {"bytes": 538054400 + 6371328,
+                                  "profile": "profiles/k_dec_attn_umma_f1r_decode_shared_kv_rope.md", **_DEC},
 }
 NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # the figures the targets are quoted against
 
@@ -548,6 +557,17 @@ def bench_plane_mix(torch, Bd):
                          "whole_step_frac_of_peak": None}}
 
 
+def bench_mma_rates(torch, Bd):
+    """Cycles per tcgen05.mma (128 x N x 16, bf16) by operand source and layout, all SMs busy."""
+    names = {0: "A, B shared memory K-major", 1: "A in TMEM, B K-major", 2: "B MN-major in shared memory"}
+    table = {f"{names[m]}, N={n}": round(Bd.probe_mma_rate(m, n), 1) for m in (0, 1, 2) for n in (64, 128, 256)}
+    assert Bd.last_device_error() == 0
+    return {"workload": "mma_rate_probe", "unit": "cycles per MMA (N=128, smem K-major)", "value": table["A, B shared memory K-major, N=128"],
+            "ms_per_step": 0.0, "gpu_launches_per_step": 9, "l2": "n/a", "note": table,
+            "roofline": {"kernel": "tcgen05.mma issue rate", "bound": "tensor", "achieved": None, "peak": None, "unit": "cycles",
+                         "frac": None, "traffic": None, "kernel_ms": 0.0, "whole_step_frac_of_peak": None}}
+
+
 def load_hosvd_ws(Bd, d, n_H, ranks):
     return int(Bd.load_library().tucker_hosvd_workspace_bytes(int(d), int(n_H), int(ranks[1]), int(ranks[2])))
 
@@ -590,10 +610,10 @@ def main():
             dist.barrier()
 
     peaks, peak_kind = load_peaks()
-    if args.workload in ("f2", "f3", "f4"):
+    if args.workload in ("f2", "f3", "f4", "mma"):
         # the widened rows that are not layer steps: the plane-mixing probe, the weight packers, the HOSVD initialiser
         o = {"f2": lambda: bench_plane_mix(torch, Bd), "f3": lambda: bench_pack(torch, Bd, peaks),
-             "f4": lambda: bench_hosvd(torch, Bd, peaks)}[args.workload]()
+             "f4": lambda: bench_hosvd(torch, Bd, peaks), "mma": lambda: bench_mma_rates(torch, Bd)}[args.workload]()
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": o["value"], "unit": o["unit"], "n_gpus": world, "steps": args.steps,
                               "warmup": args.warmup, "ms_per_step": o["ms_per_step"], "higher_is_better": o["unit"] != "ms",

@@ -331,6 +331,17 @@ TA_API int tucker_attn_set_profile_events(void* ev_start, void* ev_stop);
 TA_API int tucker_probe_plane_mix(int32_t tiles, int32_t r1, int32_t n_blocks, const float* u1, long long* cycles,
                            float* sink, void* cuda_stream);
 
+/*
+ * Measurement probe (no counterpart in the paper): cycles per tcgen05.mma of shape 128 x N x 16 (bf16 in, fp32
+ * accumulate) when one thread issues `iters` x 8 of them back to back, by operand source: mode 0 = A and B in
+ * shared memory, K-major; 1 = A in TMEM; 2 = B MN-major in shared memory (a tile used where it lies, as the value
+ * tiles and the in-place factor matrices are).  N in {64, 128, 256}.  cycles [n_blocks] (device) receives each
+ * block's clock64 count for the whole sequence including the final commit.  Decides, with numbers, which operand
+ * layouts the kernels should prefer.  Returns TA_OK, TA_ERR_INVALID_ARG or TA_ERR_CUDA.
+ */
+TA_API int tucker_probe_mma_rate(int32_t mode, int32_t N, int32_t iters, int32_t n_blocks, long long* cycles,
+                          void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ EXPORTS = (
     "tucker_attn_decode_static", "tucker_attn_selftest_wait_timeout", "tucker_attn_sync_status",
     "tucker_attn_bounds_checked",
     "tucker_pack_gqa", "tucker_pack_mha", "tucker_pack_mla",
-    "tucker_hosvd_workspace_bytes", "tucker_hosvd_init", "tucker_mha_weight_tensors", "tucker_probe_plane_mix",
+    "tucker_hosvd_workspace_bytes", "tucker_hosvd_init", "tucker_mha_weight_tensors", "tucker_probe_plane_mix", "tucker_probe_mma_rate",
 )
 TA_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
     lib.tucker_hosvd_init.argtypes = [i32] * 5 + [vp] * 7 + [sz, vp]
     lib.tucker_mha_weight_tensors.restype = ctypes.c_int
     lib.tucker_mha_weight_tensors.argtypes = [i32] * 2 + [vp] * 7
+    lib.tucker_probe_mma_rate.restype = ctypes.c_int
+    lib.tucker_probe_mma_rate.argtypes = [i32] * 4 + [vp] * 2
     lib.tucker_probe_plane_mix.restype = ctypes.c_int
     lib.tucker_probe_plane_mix.argtypes = [i32] * 3 + [vp] * 4
     _lib = lib
@@ -424,6 +426,20 @@ def tucker_hosvd_init(W, ranks, *, workspace=None):
     if rc != TA_OK:
         raise TuckerAttnError(rc, "tucker_hosvd_init")
     return C, U1, U2, U3, (spectra[:n_H], spectra[n_H:n_H + d], spectra[n_H + d:])
+
+
+def probe_mma_rate(mode: int, N: int, iters: int = 256, n_blocks: int = 148) -> float:
+    """Cycles per tcgen05.mma 128 x N x 16 for an operand source / layout (see tucker_probe_mma_rate): the
+    slowest block's count divided by the number of MMAs."""
+    torch = _torch()
+    dev = torch.device("cuda", torch.cuda.current_device())
+    cycles = torch.zeros(n_blocks, dtype=torch.int64, device=dev)
+    rc = load_library().tucker_probe_mma_rate(int(mode), int(N), int(iters), int(n_blocks), cycles.data_ptr(),
+                                              _stream_ptr(dev))
+    if rc != TA_OK:
+        raise TuckerAttnError(rc, "tucker_probe_mma_rate")
+    torch.cuda.synchronize()
+    return float(cycles.max().item()) / (iters * 8)
 
 
 def probe_plane_mix(tiles: int, r1: int, n_blocks: int = 148):

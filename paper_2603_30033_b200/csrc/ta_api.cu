@@ -27,6 +27,8 @@ static unsigned int* device_error_ptr() {
   return cache[dev];
 }
 
+unsigned int* device_error_word() { return device_error_ptr(); }
+
 static bool desc_ok(const tucker_attn_desc* d, bool decode) {
   if (!d) return false;
   if (d->B <= 0 || d->d_model <= 0 || d->n_H <= 0) return false;

@@ -15,6 +15,9 @@ namespace ta {
 
 typedef __nv_bfloat16 bf16;
 
+// Device address of the current device's error word (nullptr if it cannot be resolved); ta_api.cu.
+unsigned int* device_error_word();
+
 // Everything a path needs to run one call; filled by the API layer after validation.
 struct Problem {
   tucker_attn_desc d;

@@ -77,6 +77,50 @@ __global__ void __launch_bounds__(PM_THREADS, 1) k_probe_plane_mix(int tiles, in
   if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
+// Issue rate of tcgen05.mma (M = 128, K = 16, bf16 -> fp32) by operand source and layout: `iters` groups of
+// eight dependent-accumulator MMAs issued back to back by one thread, one commit at the end.
+//   mode 0  A and B in shared memory, both K-major       mode 1  A in TMEM, B K-major in shared memory
+//   mode 2  A K-major, B MN-major in shared memory (a tile used where it lies with its N index contiguous)
+__global__ void __launch_bounds__(128, 1) k_probe_mma_rate(int mode, int N, int iters, long long* __restrict__ cycles,
+                                                            unsigned int* err) {
+  extern __shared__ uint8_t pm_smem[];
+  __shared__ uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  const uint32_t base = (smem_u32(pm_smem) + 1023u) & ~1023u;
+  uint8_t* tiles = pm_smem + (base - smem_u32(pm_smem));
+  for (int i = threadIdx.x; i < 96 * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(tiles)[i] = 0x3c003c00u;
+  const int warp = threadIdx.x / 32;
+  Abort ab{&abort_flag, err};
+  if (threadIdx.x == 0) { abort_flag = 0; mbar_init(&bar, 1); fence_barrier_init(); }
+  if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;
+  if (warp == 1 && elect_one()) {
+    const uint32_t idesc = umma_idesc_bf16(128, (uint32_t)N);
+    const uint32_t a = smem_u32(tiles), b = smem_u32(tiles + 32 * 1024);
+    const long long t0 = clock64();
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32;
+        if (mode == 0) umma_ss(tmem, umma_desc_kmajor_sw128(a + off), umma_desc_kmajor_sw128(b + off), idesc, 1);
+        else if (mode == 1) umma_ts(tmem, tmem + 256 + ks * 8, umma_desc_kmajor_sw128(b + off), idesc, 1);
+        else umma_ss(tmem, umma_desc_kmajor_sw128(a + off), umma_desc_mnmajor_sw128(b + ks * 2048, 16384), idesc | (1u << 16), 1);
+      }
+    }
+    umma_commit(&bar);
+    (void)mbar_wait(&bar, 0, ab);
+    cycles[blockIdx.x] = clock64() - t0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
 }  // namespace
 }  // namespace ta
 
@@ -85,5 +129,18 @@ extern "C" int tucker_probe_plane_mix(int32_t tiles, int32_t r1, int32_t n_block
   using namespace ta;
   if (tiles <= 0 || r1 <= 0 || r1 > PM_MAX_R1 || n_blocks <= 0 || !u1 || !cycles || !sink) return TA_ERR_INVALID_ARG;
   k_probe_plane_mix<<<n_blocks, PM_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(tiles, r1, u1, cycles, sink);
+  return cudaGetLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
+}
+
+extern "C" int tucker_probe_mma_rate(int32_t mode, int32_t N, int32_t iters, int32_t n_blocks, long long* cycles,
+                                     void* cuda_stream) {
+  using namespace ta;
+  if (mode < 0 || mode > 2 || (N != 64 && N != 128 && N != 256) || iters <= 0 || iters > 4096 || n_blocks <= 0 || !cycles)
+    return TA_ERR_INVALID_ARG;
+  unsigned int* errp = device_error_word();
+  if (!errp) return TA_ERR_CUDA;
+  static PerDeviceFlag attr;
+  TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)k_probe_mma_rate, 100 * 1024));
+  k_probe_mma_rate<<<n_blocks, 128, 100 * 1024, static_cast<cudaStream_t>(cuda_stream)>>>(mode, N, iters, cycles, errp);
   return cudaGetLastError() == cudaSuccess ? TA_OK : TA_ERR_CUDA;
 }
