@@ -421,15 +421,19 @@ def bench_decode(w, steps, warmup, torch, Bd, barrier, peaks, with_e2e=True, sam
 # CPU oracle arm (bounded sample)
 # ----------------------------------------------------------------------------------------
 
-def oracle_sample(w, budget="default"):
+def oracle_sample(w, scale=1.0):
     """Returns (callable running the oracle on a bounded sample, work in the metric's unit
-    numerator, description, unit)."""
+    numerator, description, unit).  `scale` enlarges the default sample: more sequences first (up to the
+    workload's batch), then more query rows per sequence (up to all of them)."""
     from oracle import tucker_oracle as O
     wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
     args = [wt[k] for k in KEYS]
     if w.kind == "prefill":
         nrows = {"c4_long_prefill": 256, "c2_gpt2_prefill": 1024, "c3_vit_prefill": 197}.get(w.name, min(w.N, 256))
         nseq = {"c3_vit_prefill": 8}.get(w.name, 1)
+        nseq2 = int(min(w.B, max(nseq, round(nseq * scale))))
+        nrows = int(min(w.N, max(nrows, round(nrows * scale * nseq / nseq2))))
+        nseq = nseq2
         rows = sorted(set(np.linspace(0, w.N - 1, nrows).astype(int).tolist()))
         X = W.round_to_storage(W.make_X(w, B=nseq), w.dtype)
         r1, r2, r3 = w.r
@@ -444,7 +448,7 @@ def oracle_sample(w, budget="default"):
         desc = (f"{nseq} of {w.B} sequences, projections for all {w.N} tokens, attention and output for "
                 f"{len(rows)} evenly spaced query rows per sequence")
         return run, flops / 1e12, desc, "TFLOP/s"
-    nseq = 4
+    nseq = int(min(w.B, max(4, round(4 * scale))))
     L = w.N
     x = W.round_to_storage(W.make_decode_x(w, B=nseq), w.dtype)
     Kc = np.zeros((nseq, L + 1, w.r[2]))
@@ -473,8 +477,15 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(w, steps=1, warmup=0):
+def time_oracle(w, steps=1, warmup=0, budget_s=10.0):
+    """Times the oracle, as it stands, on a bounded sample of the workload sized to take about `budget_s`
+    seconds per run on this host: the default sample is timed once as a probe and enlarged accordingly."""
     run, work, desc, unit = oracle_sample(w)
+    t = time.perf_counter()
+    run()
+    probe = max(time.perf_counter() - t, 1e-3)
+    if budget_s / probe >= 1.5:
+        run, work, desc, unit = oracle_sample(w, scale=budget_s / probe)
     for _ in range(warmup):
         run()
     ts = []
@@ -491,7 +502,9 @@ def run_reference(args, rank):
     if rank != 0:
         return
     w = W.get_workload(args.workload)
-    cb = time_oracle(w, steps=max(1, args.steps), warmup=min(args.warmup, 1))
+    # every step is one bounded sample; their size is set so that the whole run stays within a few minutes
+    n_runs = max(1, args.steps) + min(args.warmup, 1)
+    cb = time_oracle(w, steps=max(1, args.steps), warmup=min(args.warmup, 1), budget_s=min(10.0, max(0.5, 120.0 / n_runs)))
     line = {
         "impl": "reference", "metric": METRIC, "value": cb["value"], "unit": cb["unit"], "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": cb["seconds_per_sample"] * 1e3,
