@@ -24,7 +24,10 @@
  *     contiguous, 16-byte aligned.  The library never allocates, frees or keeps a pointer
  *     after the call returns.  Scratch space is passed in as `workspace`.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t cast to void*; NULL = default
- *     stream).  No host synchronisation happens inside a call.
+ *     stream).  No host synchronisation happens inside a call, and tucker_attn_fwd /
+ *     tucker_attn_decode read no device memory on the host, so (after one ordinary call per
+ *     device, which sets kernel attributes) they can be captured into a CUDA graph and replayed
+ *     on new contents of the same buffers.
  *   - Storage type (`dtype`): TA_DTYPE_F32 = float everywhere (plain FMA arithmetic, no
  *     tensor cores); TA_DTYPE_BF16 = __nv_bfloat16 for X, weights, caches and Y with fp32
  *     accumulation.

@@ -450,6 +450,49 @@ def test_decode_garbage_beyond_cache_len_is_ignored():
     check(y.float().cpu().numpy().astype(np.float64), ref, "bf16", "garbage tail")
 
 
+def test_calls_replay_from_a_cuda_graph():
+    # Neither entry point synchronises, allocates or reads device memory on the host, so a call can be captured
+    # into a CUDA graph (its launches keep their programmatic-dependent-launch edges) and replayed on new contents
+    # of the same buffers; the replays must give the direct calls' bits.
+    import torch
+    w = H.custom_workload(kind="decode", dtype="bf16", d_model=256, n_H=8, r=(4, 64, 64), t=(4, 64, 64), rope=True,
+                          rope_base=500000.0, seed=43)
+    wt = {k: W.round_to_storage(v, w.dtype) for k, v in W.make_weights(w).items()}
+    dw = H.weights_to_device(wt, "bf16")
+    lens = [100, 300, 7, 511]
+    x, Kc, Vc, cl = W.make_decode_state(w, B=4, L=max(lens), Lmax=1024, cache_len=lens)
+    xd, Kd, Vd = (H.to_device(W.round_to_storage(a, "bf16"), "bf16") for a in (x, Kc, Vc))
+    ld = torch.from_numpy(cl).cuda()
+    desc = Bd.make_desc(B=4, N=1, d_model=256, n_H=8, r=w.r, t=w.t, causal=True, rope=True, rope_base=w.rope_base)
+    ws = Bd.alloc_workspace(Bd.decode_workspace_bytes(desc, 1024), xd.device)
+    y = torch.empty_like(xd)
+    dkw = dict(n_H=8, rope=True, rope_base=w.rope_base, append=False, out=y, workspace=ws)
+    Xp = H.to_device(W.round_to_storage(W.make_X(H.with_(w, kind="prefill"), B=2, N=200), "bf16"), "bf16")
+    pdesc = Bd.make_desc(B=2, N=200, d_model=256, n_H=8, r=w.r, t=w.t, causal=True, rope=True, rope_base=w.rope_base)
+    pws = Bd.alloc_workspace(Bd.fwd_workspace_bytes(pdesc), xd.device)
+    Y = torch.empty_like(Xp)
+    pkw = dict(n_H=8, causal=True, rope=True, rope_base=w.rope_base, out=Y, workspace=pws)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        Bd.tucker_attn_decode(xd, *dw, Kd, Vd, ld, **dkw)          # warm-up outside the capture (kernel attributes)
+        Bd.tucker_attn_fwd(Xp, *dw, **pkw)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            Bd.tucker_attn_decode(xd, *dw, Kd, Vd, ld, **dkw)
+            Bd.tucker_attn_fwd(Xp, *dw, **pkw)
+    for trial in range(2):
+        xd.copy_(torch.randn_like(xd))                               # new contents, same buffers
+        Xp.copy_(torch.randn_like(Xp))
+        want_y = Bd.tucker_attn_decode(xd, *dw, Kd, Vd, ld, **{**dkw, "out": torch.empty_like(xd)})
+        want_Y = Bd.tucker_attn_fwd(Xp, *dw, **{**pkw, "out": torch.empty_like(Xp)})
+        y.zero_(); Y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert Bd.last_device_error() == 0
+        assert torch.equal(y, want_y) and torch.equal(Y, want_Y), f"trial {trial}"
+
+
 def test_decode_no_append_leaves_cache():
     w = H.custom_workload(kind="decode", dtype="fp32", d_model=32, n_H=4, r=(2, 8, 8), t=(2, 8, 8), rope=True, seed=18)
     y, ref, (Kd, Vd, Kc, Vc, *_r) = run_decode(w, 2, [5, 9], 16, append=False)
