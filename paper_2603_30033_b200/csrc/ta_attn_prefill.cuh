@@ -2,8 +2,11 @@
 // paper: online softmax over key chunks, one K/V chunk pair shared by all heads), with the
 // per-head latent queries of Definition 2 formed inside the kernel.
 //
-// One CTA handles one work item = (sequence b, 128 query rows, a run of head pairs).  For every
-// head pair (h, h+1) of its run:
+// A work item = (sequence b, 128 query rows, a run of head pairs).  The grid is persistent: one CTA per SM walks
+// the items blockIdx.x, 2 G - 1 - blockIdx.x, 2 G + blockIdx.x, ... of the list ordered heaviest first (G = grid
+// size; the back-and-forth order evens out the causal items' sizes), so that a CTA's start-up (TMEM allocation,
+// barriers, first loads: about 3 us) is paid once per SM and the next item's tiles are already on their way
+// while the current item finishes.  For every head pair (h, h+1) of an item's run:
 //   prologue   Qhat_i = Qt G_{h+i} on the tensor core (Qt tile loaded once per CTA, G tiles
 //              streamed through the V ring), latent RoPE applied while the result moves
 //              TMEM -> registers -> shared memory (bf16, the swizzled K-major layout UMMA reads)
@@ -60,6 +63,7 @@ struct Params {
   int n_hp;          // head pairs
   int hp_per_item;   // consecutive head pairs handled by one CTA (1 in the unfused mode)
   int n_hg;          // head-pair groups = ceil(n_hp / hp_per_item)
+  int n_items;       // work items = n_qt * B * n_hg
   int fused;         // 1: tmQ is the map of Qt [B, N, r2] and Qhat is formed in the prologue
   const float2* rope;   // [N][r3/2] (cos, sin) for rows of this call, or nullptr (fused mode only)
   bf16* O;           // [B, N, nH, t3] (written through the tensor map tmO)
@@ -100,13 +104,32 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
 __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
 
+// The k-th work item of this CTA (see the header comment); false when the CTA has run out of items.
+struct Item {
+  int b, qt, q0, hp_begin, hp_end, nt;
+};
+__device__ __forceinline__ bool get_item(const Params& p, int k, Item& im) {
+  const int G = (int)gridDim.x;
+  long item = (long)k * G + ((k & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
+  if (item >= p.n_items) return false;
+  const int hg = (int)(item % p.n_hg); item /= p.n_hg;
+  im.b = (int)(item % p.B); item /= p.B;
+  im.qt = p.n_qt - 1 - (int)item;            // heaviest (largest query tile) first
+  im.q0 = im.qt * BQ;
+  im.hp_begin = hg * p.hp_per_item;
+  im.hp_end = min(p.n_hp, im.hp_begin + p.hp_per_item);
+  const int n_kt_all = (p.N + BKV - 1) / BKV;
+  im.nt = p.causal ? min(n_kt_all, im.qt + 1) : n_kt_all;
+  return true;
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmO, const Params p) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t q_full, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
+  __shared__ uint64_t q_full, qt_free, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ uint64_t s_full[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];
   __shared__ uint64_t o_staged[2], stage_free[2];   // output rows are in shared memory / the output store has read them
   __shared__ uint32_t tmem_slot;
@@ -120,22 +143,13 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint8_t* v_ring = k_ring + KV_STAGES * MAX_SUB * SUB_BYTES;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  // work item: heaviest (largest query tile) first
-  int item = blockIdx.x;
-  const int hg = item % p.n_hg; item /= p.n_hg;
-  const int b = item % p.B; item /= p.B;
-  const int qt = p.n_qt - 1 - item;
-  const int q0 = qt * BQ;
-  const int hp_begin = hg * p.hp_per_item;
-  const int hp_end = min(p.n_hp, hp_begin + p.hp_per_item);
-  const int n_kt_all = (p.N + BKV - 1) / BKV;
-  const int nt = p.causal ? min(n_kt_all, qt + 1) : n_kt_all;
   const int qsub = (p.r2 + 63) / 64, ksub = (p.r3 + 63) / 64, vsub = (p.t3 + 63) / 64;
   Abort ab{&abort_flag, p.err};
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(&q_full, 1);
+    mbar_init(&qt_free, 1);       // the item's per-head query MMAs have read the Qt tile
     for (int s = 0; s < KV_STAGES; ++s) {
       mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
@@ -171,11 +185,16 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       if (p.fused) tma_prefetch_desc(&tmG);
       int it_k = 0, it_v = 0;          // ring iterations issued so far
       bool ok = true;
-      for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
+      Item im;
+      for (int k = 0; ok && get_item(p, k, im); ++k) {
+      const int b = im.b, q0 = im.q0, nt = im.nt;
+      for (int hp = im.hp_begin; hp < im.hp_end && ok; ++hp) {
         const int h0 = hp * 2;
         const int nh = (h0 + 1) < p.nH ? 2 : 1;
         if (p.fused) {
-          if (hp == hp_begin) {
+          if (hp == im.hp_begin) {
+            // the previous item's per-head query MMAs must have read the Qt tile
+            if (k > 0 && !(ok = mbar_wait(&qt_free, (uint32_t)((k - 1) & 1), ab))) break;
             mbar_expect_tx(&q_full, (uint32_t)(qsub * SUB_BYTES));
             for (int kk = 0; kk < qsub; ++kk) tma_load_3d(qt_tile + kk * SUB_BYTES, &tmQ, &q_full, kk * 64, q0, b);
           }
@@ -205,6 +224,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             tma_load_3d(v_ring + (sv * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[sv], kk * 64, j * BKV, b);
         }
       }
+      }
     }
    } else if (warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
@@ -213,7 +233,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint32_t idesc_pv = umma_idesc_bf16(BQ, (uint32_t)p.t3) | (1u << 16);   // B = V is MN-major
       const uint32_t idesc_qh = umma_idesc_bf16(BQ, (uint32_t)p.r3);
       const int ksteps = p.r3 / 16;
-      int it_k = 0, it_v = 0, jt = 0;  // ring iterations / tiles consumed so far
+      int it_k = 0, it_v = 0;          // ring iterations consumed so far
+      int jt[2] = {0, 0}, gp[2] = {0, 0};   // per head: key tiles / head pairs handled so far (barrier parities)
       auto issue_qk = [&](int i, int s) {
         const uint32_t qa = smem_u32(q_tile[i]), ka = smem_u32(k_ring + s * MAX_SUB * SUB_BYTES);
         for (int ks = 0; ks < ksteps; ++ks) {
@@ -230,11 +251,14 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         umma_commit(&o_full[i]);
       };
       bool ok = true;
-      for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
-        const int g = hp - hp_begin;
+      Item im;
+      for (int k = 0; ok && get_item(p, k, im); ++k) {
+      const int nt = im.nt;
+      for (int hp = im.hp_begin; hp < im.hp_end && ok; ++hp) {
+        const int g = hp - im.hp_begin;
         const int nh = (hp * 2 + 1) < p.nH ? 2 : 1;
         if (p.fused) {
-          if (g == 0 && !(ok = mbar_wait(&q_full, 0, ab))) break;
+          if (g == 0 && !(ok = mbar_wait(&q_full, (uint32_t)(k & 1), ab))) break;
           for (int i = 0; i < nh && ok; ++i, ++it_v) {
             const int s = it_v % KV_STAGES;
             if (!(ok = mbar_wait(&v_full[s], (it_v / KV_STAGES) & 1, ab))) break;
@@ -248,14 +272,15 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             umma_commit(&v_empty[s]);
           }
           if (!ok) break;
+          if (hp == im.hp_end - 1) umma_commit(&qt_free);   // the item's last use of the Qt tile
         } else {
-          if (!(ok = mbar_wait(&q_full, 0, ab))) break;
+          if (!(ok = mbar_wait(&q_full, 0, ab))) break;     // (one item and one pair per CTA in this mode)
         }
         {
           const int s = it_k % KV_STAGES;
           if (!(ok = mbar_wait(&k_full[s], (it_k / KV_STAGES) & 1, ab))) break;
           for (int i = 0; i < nh && ok; ++i) {
-            if (p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)(g & 1), ab))) break;
+            if (p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)(gp[i] & 1), ab))) break;
             tc_fence_after();
             issue_qk(i, s);
           }
@@ -263,13 +288,14 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           umma_commit(&k_empty[s]);
           ++it_k;
         }
-        for (int j = 0; j < nt && ok; ++j, ++jt, ++it_v) {
+        for (int j = 0; j < nt && ok; ++j, ++it_v) {
           const int sv = it_v % KV_STAGES;
           const bool more = (j + 1) < nt;
           const int sk = it_k % KV_STAGES;
           if (!(ok = mbar_wait(&v_full[sv], (it_v / KV_STAGES) & 1, ab))) break;
           for (int i = 0; i < nh && ok; ++i) {
-            if (!(ok = mbar_wait(&p_full[i], (uint32_t)(jt & 1), ab))) break;
+            if (!(ok = mbar_wait(&p_full[i], (uint32_t)(jt[i] & 1), ab))) break;
+            ++jt[i];
             tc_fence_after();
             issue_pv(i, sv, j);
             if (i == nh - 1) umma_commit(&v_empty[sv]);
@@ -284,6 +310,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           }
           if (more) ++it_k;
         }
+        for (int i = 0; i < nh; ++i) ++gp[i];
+      }
       }
     }
    }
@@ -293,14 +321,17 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int i = (warp - 4) / 4;              // which head of the pair
     const int q = warp % 4;                    // TMEM lane quadrant
     const int rloc = q * 32 + lane;            // row inside the tile
-    const int row = q0 + rloc;                 // query row inside the sequence
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int jt = 0;                                // tiles consumed so far (parity of s_full / p_full / o_full)
+    int g = 0;                                 // head pairs this warpgroup has handled so far (parity of the per-pair barriers)
     bool ok = true;
-    for (int hp = hp_begin; hp < hp_end && ok; ++hp) {
-      const int g = hp - hp_begin;
+    Item im;
+    for (int k = 0; ok && get_item(p, k, im); ++k) {
+    const int b = im.b, q0 = im.q0, nt = im.nt;
+    const int row = q0 + rloc;                 // query row inside the sequence
+    for (int hp = im.hp_begin; hp < im.hp_end && ok; ++hp) {
       const int h0 = hp * 2;
-      if (i == 1 && (h0 + 1) >= p.nH) break;   // odd head count: the last pair has one head
+      if (i == 1 && (h0 + 1) >= p.nH) continue;   // odd head count: the last pair has one head
       if (g > 0) {
         // the previous pair's output store must have finished reading this head's Qhat tile
         if (q == 0 && lane == 0) {
@@ -465,6 +496,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
       }
       tc_fence_before();   // the next head pair's MMAs overwrite S_i / O_i after these reads
+      ++g;
+    }
     }
     if (q == 0 && lane == 0) tma_store_wait_all();   // the stores read shared memory: finish before the CTA may exit
   }

@@ -17,6 +17,8 @@
 
 #include <math.h>
 
+#include <algorithm>
+
 namespace ta {
 namespace {
 
@@ -279,9 +281,10 @@ bool tmap_3d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uin
 int sm_count();
 size_t l2_bytes();
 
-// Consecutive head pairs per CTA.  Causal work items differ in size, so many small items balance
-// best; without a mask all items are equal and a CTA that keeps several head pairs amortises its
-// set-up, as long as the number of waves does not grow.
+// Consecutive head pairs per work item.  Causal items differ in size, so many small items balance best over
+// the persistent grid: one pair per item (two were measured equal on the long causal prefill, 951 us both, three
+// and more worse).  Without a mask all items are equal and an item that keeps several head pairs re-uses its
+// Qt tile, as long as the number of waves does not grow.
 int head_pairs_per_item(const tucker_attn_desc& d, int n_qt, int n_hp) {
   if (d.causal) return 1;
   const long sms = sm_count();
@@ -329,8 +332,12 @@ int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const f
   static PerDeviceFlag attr;
   TA_CUDA_TRY(ensure_dynamic_smem(attr, (const void*)attn::k_attn_prefill, (int)attn::SMEM_BYTES));
   const long items = (long)ap.n_qt * d.B * ap.n_hg;
+  if (items >= (1L << 30)) return TA_ERR_UNSUPPORTED_SHAPE;
+  ap.n_items = (int)items;
+  // persistent grid: one CTA per SM walks the item list (the unfused mode keeps one item per CTA)
+  const long grid = fused ? std::min<long>(items, sm_count()) : items;
   prof_begin(p);
-  (void)launch_pdl(attn::k_attn_prefill, dim3((unsigned)items), dim3(attn::THREADS), attn::SMEM_BYTES, p.stream, tmQ, tmG,
+  (void)launch_pdl(attn::k_attn_prefill, dim3((unsigned)grid), dim3(attn::THREADS), attn::SMEM_BYTES, p.stream, tmQ, tmG,
                    tmK, tmV, tmO, ap);
   prof_end(p);
   TA_LAUNCH_CHECK(p);

@@ -558,6 +558,18 @@ def test_full_size_prefill_sampled(name, nrows):
     check(got[batches][:, rows], ref, w.dtype, name)
 
 
+def test_persistent_grid_walks_many_causal_items():
+    # 1152 causal work items of 1 - 8 key tiles on one CTA per SM (each CTA walks about eight items, back and forth
+    # through the size-ordered list), an odd number of head pairs per row tile and ragged last tiles
+    w = H.custom_workload(dtype="bf16", B=16, N=1000, d_model=576, n_H=18, r=(6, 64, 64), t=(6, 64, 64), causal=True,
+                          rope=True, rope_base=10000.0, seed=88)
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w)
+    assert Bd.last_path() == 2
+    batches, rows = [0, 9, 15], sample_rows(w.N, 24, 3)
+    check(got[batches][:, rows], oracle_fwd(X[batches], wt, w, rows=rows), "bf16", "causal, persistent grid")
+
+
 def test_sharp_softmax_variant():
     # pre-softmax core scaled by 8: peaky rows exercise the online rescaling
     w = H.with_(W.get_workload("c2"), B=2)
