@@ -104,6 +104,43 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
 __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
 
+// Waits until the shared-memory counter *c has reached `target` (bounded like the barrier waits).
+__device__ __forceinline__ bool wait_count(const int* c, int target, const Abort& ab) {
+  const volatile int* vc = c;
+  if (*vc >= target) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (*vc >= target) return true;
+    if (ab.raised()) return false;
+    if (clock64() - t0 > kWaitBudgetCycles) {
+      ab.raise();
+      return false;
+    }
+  }
+}
+
+// Eight-or-fewer K = 16 steps of one 128 x N product over K-major, 128-byte-swizzled shared-memory tiles whose
+// 64-element K blocks are SUB_BYTES apart: the step offsets are immediates added to the descriptors' address field.
+__device__ __forceinline__ void issue_kmajor_ss(uint32_t d_tmem, uint32_t a_saddr, uint32_t b_saddr, uint32_t idesc, int ksteps) {
+  const uint64_t ad = umma_desc_kmajor_sw128(a_saddr), bd = umma_desc_kmajor_sw128(b_saddr);
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    if (ks < ksteps) {
+      const uint64_t o = (uint64_t)(((uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32) >> 4);
+      umma_ss(d_tmem, ad + o, bd + o, idesc, ks != 0);
+    }
+  }
+}
+// O += P V over one 128-key tile: A = P from TMEM (bf16, 8 columns per step), B = the transposed value tile.
+__device__ __forceinline__ void issue_kmajor_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_saddr, uint32_t idesc, bool acc) {
+  const uint64_t bd = umma_desc_kmajor_sw128(b_saddr);
+#pragma unroll
+  for (int ks = 0; ks < BKV / 16; ++ks) {
+    const uint64_t o = (uint64_t)(((uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32) >> 4);
+    umma_ts(d_tmem, a_tmem + (uint32_t)ks * 8, bd + o, idesc, acc || ks != 0);
+  }
+}
+
 // The k-th work item of this CTA (see the header comment); false when the CTA has run out of items.
 struct Item {
   int b, qt, q0, hp_begin, hp_end, nt;
@@ -130,10 +167,11 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t q_full, qt_free, k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
-  __shared__ uint64_t s_full[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];
+  __shared__ uint64_t s_full[2], s_free[2], p_full[2], o_full[2], qh_done[2], qh_ready[2];
   __shared__ uint64_t o_staged[2], stage_free[2];   // output rows are in shared memory / the output store has read them
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ int qk_issued;    // score tiles issued so far by this CTA (written by the score issuer, read by the value issuer)
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
@@ -148,6 +186,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    qk_issued = 0;
     mbar_init(&q_full, 1);
     mbar_init(&qt_free, 1);       // the item's per-head query MMAs have read the Qt tile
     for (int s = 0; s < KV_STAGES; ++s) {
@@ -156,6 +195,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1);
+      mbar_init(&s_free[i], 4);     // one arrival per softmax warp: the score tile is in registers
       mbar_init(&p_full[i], 4);     // one arrival per softmax warp
       mbar_init(&o_full[i], 1);
       mbar_init(&qh_done[i], 1);
@@ -173,8 +213,10 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_slot;
-  const uint32_t tm_s[2] = {tmem, tmem + 128};
+  const uint32_t tm_s = tmem;                               // the one score buffer, used by the two heads in turn
+  const uint32_t tm_p[2] = {tmem + 128, tmem + 192};        // probabilities (bf16, two per column)
   const uint32_t tm_o[2] = {tmem + 256, tmem + 384};
+  const uint32_t tm_qh[2] = {tmem, tmem + 128};             // prologue accumulators: S and the two P blocks
 
   if (warp < 4) {
    regs_dec();
@@ -219,37 +261,71 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           for (int kk = 0; kk < ksub; ++kk)
             tma_load_3d(k_ring + (sk * MAX_SUB + kk) * SUB_BYTES, &tmK, &k_full[sk], kk * 64, j * BKV, b);
           if (!(ok = mbar_wait(&v_empty[sv], ((it_v / KV_STAGES) & 1) ^ 1, ab))) break;
-          mbar_expect_tx(&v_full[sv], (uint32_t)(vsub * SUB_BYTES));
-          for (int kk = 0; kk < vsub; ++kk)
-            tma_load_3d(v_ring + (sv * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[sv], kk * 64, j * BKV, b);
+          // value tile, transposed in global memory: [t3 rows][128 keys] as two 64-key blocks of 128-byte rows
+          mbar_expect_tx(&v_full[sv], (uint32_t)(2 * p.t3 * 128));
+          for (int kk = 0; kk < 2; ++kk)
+            tma_load_3d(v_ring + (sv * MAX_SUB + kk) * SUB_BYTES, &tmV, &v_full[sv], j * BKV + kk * 64, 0, b);
         }
       }
       }
     }
    } else if (warp == 1) {
-    // ------------------------------- MMA issuer ---------------------------------
+    // ------------------------------- score issuer: S = Qhat_i K^T ---------------------------------
     if (elect_one()) {
       const uint32_t idesc_qk = umma_idesc_bf16(BQ, BKV);
-      const uint32_t idesc_pv = umma_idesc_bf16(BQ, (uint32_t)p.t3) | (1u << 16);   // B = V is MN-major
-      const uint32_t idesc_qh = umma_idesc_bf16(BQ, (uint32_t)p.r3);
       const int ksteps = p.r3 / 16;
-      int it_k = 0, it_v = 0;          // ring iterations consumed so far
-      int jt[2] = {0, 0}, gp[2] = {0, 0};   // per head: key tiles / head pairs handled so far (barrier parities)
-      auto issue_qk = [&](int i, int s) {
-        const uint32_t qa = smem_u32(q_tile[i]), ka = smem_u32(k_ring + s * MAX_SUB * SUB_BYTES);
-        for (int ks = 0; ks < ksteps; ++ks) {
-          const uint32_t off = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
-          umma_ss(tm_s[i], umma_desc_kmajor_sw128(qa + off), umma_desc_kmajor_sw128(ka + off), idesc_qk, ks != 0);
+      int it_k = 0;                    // K ring iterations consumed so far
+      int ns0 = 0, ns1 = 0;            // score tiles issued so far for head 0 / head 1 of the pairs (s_free phases)
+      int gp0 = 0, gp1 = 0;            // head pairs handled so far per head (qh_ready phases)
+      int n_issued = 0;
+      bool ok = true;
+      Item im;
+      for (int k = 0; ok && get_item(p, k, im); ++k) {
+      const int nt = im.nt;
+      for (int hp = im.hp_begin; hp < im.hp_end && ok; ++hp) {
+        const int nh = (hp * 2 + 1) < p.nH ? 2 : 1;
+        if (!p.fused && !(ok = mbar_wait(&q_full, 0, ab))) break;     // (one item and one pair per CTA in this mode)
+        // The pair's score tiles in issue order: t = j * nh + i for key tile j and head i.  Tile t is issued as soon
+        // as the warpgroup of tile t - 1 holds that tile in registers, so the next scores are ready whenever a
+        // warpgroup finishes a tile.  (Tile 0 waits for the reads of the previous pair's last tiles instead.)
+        const int n_tiles = nt * nh;
+        uint32_t sk = 0;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int i = (nh == 2) ? (t & 1) : 0;
+          if (t >= 1) {
+            const int ip = (nh == 2) ? (i ^ 1) : 0;
+            if (!(ok = mbar_wait(&s_free[ip], (uint32_t)(((ip ? ns1 : ns0) - 1) & 1), ab))) break;
+          } else {
+            if (ns0 > 0 && !(ok = mbar_wait(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
+            if (ns1 > 0 && !(ok = mbar_wait(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
+          }
+          if (i == 0) {
+            sk = (uint32_t)(it_k % KV_STAGES);
+            if (!(ok = mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab))) break;
+          }
+          if (t < nh && p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)((i ? gp1 : gp0) & 1), ab))) break;
+          tc_fence_after();
+          issue_kmajor_ss(tm_s, smem_u32(tiles) + (uint32_t)(1 + i) * (MAX_SUB * SUB_BYTES),
+                          smem_u32(k_ring) + sk * (MAX_SUB * SUB_BYTES), idesc_qk, ksteps);
+          umma_commit(&s_full[i]);
+          *(volatile int*)&qk_issued = ++n_issued;
+          if (i) ++ns1; else ++ns0;
+          if (i == nh - 1) { umma_commit(&k_empty[sk]); ++it_k; }
         }
-        umma_commit(&s_full[i]);
-      };
-      auto issue_pv = [&](int i, int s, int j) {
-        const uint32_t va = smem_u32(v_ring + s * MAX_SUB * SUB_BYTES);
-        for (int ks = 0; ks < BKV / 16; ++ks)
-          umma_ts(tm_o[i], tm_s[i] + (uint32_t)ks * 8, umma_desc_mnmajor_sw128(va + (uint32_t)ks * 2048, SUB_BYTES),
-                  idesc_pv, (j | ks) != 0);
-        umma_commit(&o_full[i]);
-      };
+        ++gp0;
+        if (nh == 2) ++gp1;
+      }
+      }
+    }
+   } else if (warp == 2) {
+    // ------------------------------- value issuer: Qhat_i = Qt G_i^T, O_i += P_i V ------------------
+    if (elect_one()) {
+      const uint32_t idesc_pv = umma_idesc_bf16(BQ, (uint32_t)p.t3);
+      const uint32_t idesc_qh = umma_idesc_bf16(BQ, (uint32_t)p.r3);
+      int it_v = 0;                    // V ring iterations consumed so far
+      int np0 = 0, np1 = 0;            // P V products issued so far per head (p_full phases)
+      int ns0 = 0, ns1 = 0;            // score tiles of the finished pairs per head (s_free phases)
+      int n_before = 0;                // score tiles of the finished pairs, both heads
       bool ok = true;
       Item im;
       for (int k = 0; ok && get_item(p, k, im); ++k) {
@@ -259,58 +335,46 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int nh = (hp * 2 + 1) < p.nH ? 2 : 1;
         if (p.fused) {
           if (g == 0 && !(ok = mbar_wait(&q_full, (uint32_t)(k & 1), ab))) break;
+          // the prologue accumulates into the score and probability columns: the last score tiles of the previous
+          // pair must have been read (its P V products precede these MMAs in this thread's issue order)
+          if (ns0 > 0 && !(ok = mbar_wait(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
+          if (ns1 > 0 && !(ok = mbar_wait(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
           for (int i = 0; i < nh && ok; ++i, ++it_v) {
-            const int s = it_v % KV_STAGES;
+            const uint32_t s = (uint32_t)(it_v % KV_STAGES);
             if (!(ok = mbar_wait(&v_full[s], (it_v / KV_STAGES) & 1, ab))) break;
             tc_fence_after();
-            const uint32_t qa = smem_u32(qt_tile), ga = smem_u32(v_ring + s * MAX_SUB * SUB_BYTES);
-            for (int ks = 0; ks < p.r2 / 16; ++ks) {
-              const uint32_t off = (uint32_t)(ks >> 2) * SUB_BYTES + (uint32_t)(ks & 3) * 32;
-              umma_ss(tm_s[i], umma_desc_kmajor_sw128(qa + off), umma_desc_kmajor_sw128(ga + off), idesc_qh, ks != 0);
-            }
+            issue_kmajor_ss(tmem + (uint32_t)i * 128u, smem_u32(qt_tile), smem_u32(v_ring) + s * (MAX_SUB * SUB_BYTES), idesc_qh,
+                            p.r2 / 16);
             umma_commit(&qh_done[i]);
             umma_commit(&v_empty[s]);
           }
           if (!ok) break;
           if (hp == im.hp_end - 1) umma_commit(&qt_free);   // the item's last use of the Qt tile
-        } else {
-          if (!(ok = mbar_wait(&q_full, 0, ab))) break;     // (one item and one pair per CTA in this mode)
         }
-        {
-          const int s = it_k % KV_STAGES;
-          if (!(ok = mbar_wait(&k_full[s], (it_k / KV_STAGES) & 1, ab))) break;
-          for (int i = 0; i < nh && ok; ++i) {
-            if (p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)(gp[i] & 1), ab))) break;
-            tc_fence_after();
-            issue_qk(i, s);
+        const int n_tiles = nt * nh;
+        uint32_t sv = 0;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int i = (nh == 2) ? (t & 1) : 0;
+          const int j = (nh == 2) ? (t >> 1) : t;
+          if (i == 0) {
+            sv = (uint32_t)(it_v % KV_STAGES);
+            if (!(ok = mbar_wait(&v_full[sv], (it_v / KV_STAGES) & 1, ab))) break;
           }
-          if (!ok) break;
-          umma_commit(&k_empty[s]);
-          ++it_k;
+          if (!(ok = mbar_wait(&p_full[i], (uint32_t)((i ? np1 : np0) & 1), ab))) break;
+          if (i) ++np1; else ++np0;
+          // The tensor core runs MMAs in issue order, and an idle warpgroup is waiting for score tile t + 2 while
+          // nobody waits for this product: when both are ready at about the same time the scores go first.  (Tile
+          // t + 2 only needs tile t + 1 to have been read, which does not depend on this product.)
+          if (t + 2 < n_tiles && !(ok = wait_count(&qk_issued, n_before + t + 3, ab))) break;
+          tc_fence_after();
+          issue_kmajor_ts(tmem + 256u + (uint32_t)i * 128u, tmem + 128u + (uint32_t)i * 64u,
+                          smem_u32(v_ring) + sv * (MAX_SUB * SUB_BYTES), idesc_pv, j != 0);
+          umma_commit(&o_full[i]);
+          if (i == nh - 1) { umma_commit(&v_empty[sv]); ++it_v; }
         }
-        for (int j = 0; j < nt && ok; ++j, ++it_v) {
-          const int sv = it_v % KV_STAGES;
-          const bool more = (j + 1) < nt;
-          const int sk = it_k % KV_STAGES;
-          if (!(ok = mbar_wait(&v_full[sv], (it_v / KV_STAGES) & 1, ab))) break;
-          for (int i = 0; i < nh && ok; ++i) {
-            if (!(ok = mbar_wait(&p_full[i], (uint32_t)(jt[i] & 1), ab))) break;
-            ++jt[i];
-            tc_fence_after();
-            issue_pv(i, sv, j);
-            if (i == nh - 1) umma_commit(&v_empty[sv]);
-            if (more) {
-              if (i == 0) {
-                if (!(ok = mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab))) break;
-                tc_fence_after();
-              }
-              issue_qk(i, sk);
-              if (i == nh - 1) umma_commit(&k_empty[sk]);
-            }
-          }
-          if (more) ++it_k;
-        }
-        for (int i = 0; i < nh; ++i) ++gp[i];
+        ns0 += nt;
+        if (nh == 2) ns1 += nt;
+        n_before += n_tiles;
       }
       }
     }
@@ -324,6 +388,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int jt = 0;                                // tiles consumed so far (parity of s_full / p_full / o_full)
     int g = 0;                                 // head pairs this warpgroup has handled so far (parity of the per-pair barriers)
+    int g_two = 0;                             // ... of which had two heads (parity of the other head's qh_ready)
     bool ok = true;
     Item im;
     for (int k = 0; ok && get_item(p, k, im); ++k) {
@@ -331,7 +396,8 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int row = q0 + rloc;                 // query row inside the sequence
     for (int hp = im.hp_begin; hp < im.hp_end && ok; ++hp) {
       const int h0 = hp * 2;
-      if (i == 1 && (h0 + 1) >= p.nH) continue;   // odd head count: the last pair has one head
+      const bool two_heads = (h0 + 1) < p.nH;
+      if (i == 1 && !two_heads) continue;         // odd head count: the last pair has one head
       if (g > 0) {
         // the previous pair's output store must have finished reading this head's Qhat tile
         if (q == 0 && lane == 0) {
@@ -351,7 +417,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const float2* tab = (p.rope && row < p.N) ? p.rope + (long)row * (p.r3 / 2) : nullptr;
         for (int ch = 0; ch < p.r3 / 32; ++ch) {
           uint32_t r[32];
-          tmem_ld32(tm_s[i] + lane_addr + ch * 32, r);
+          tmem_ld32(tm_qh[i] + lane_addr + ch * 32, r);
           tmem_ld_wait();
           uint32_t o[16];
           if (tab) {
@@ -390,12 +456,16 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         uint32_t sr[128];
         {
           uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(sr);
-          tmem_ld32(tm_s[i] + lane_addr + 0, c[0]);
-          tmem_ld32(tm_s[i] + lane_addr + 32, c[1]);
-          tmem_ld32(tm_s[i] + lane_addr + 64, c[2]);
-          tmem_ld32(tm_s[i] + lane_addr + 96, c[3]);
+          tmem_ld32(tm_s + lane_addr + 0, c[0]);
+          tmem_ld32(tm_s + lane_addr + 32, c[1]);
+          tmem_ld32(tm_s + lane_addr + 64, c[2]);
+          tmem_ld32(tm_s + lane_addr + 96, c[3]);
           tmem_ld_wait();
         }
+        // the tile is in registers: the tensor core may write the other head's (or the next) scores into the buffer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_free[i]);
         const int k0 = j * BKV;
         const bool need_mask = (p.causal && (k0 + BKV - 1 > q0)) || (k0 + BKV > p.N);
         if (need_mask) {
@@ -452,10 +522,20 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           const float2 r01 = __fadd2_rn(rs[0], rs[1]), r23 = __fadd2_rn(rs[2], rs[3]);
           l += (r01.x + r01.y) + (r23.x + r23.y);
         }
+        // P_i is free once the previous P V product of this head has read it; on a pair's first tile head 0 also
+        // waits until head 1's prologue has taken its Qhat accumulator out of the P columns
+        if (j > 0) {
+          ok = mbar_wait(&o_full[i], (uint32_t)((jt - 1) & 1), ab);
+        } else if (p.fused && i == 0 && two_heads) {
+          ok = mbar_wait(&qh_ready[1], (uint32_t)(g_two & 1), ab);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
         {
           uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(sr);
-          tmem_st32(tm_s[i] + lane_addr + 0, c[0]);
-          tmem_st32(tm_s[i] + lane_addr + 32, c[1]);
+          tmem_st32(tm_p[i] + lane_addr + 0, c[0]);
+          tmem_st32(tm_p[i] + lane_addr + 32, c[1]);
           tmem_st_wait();
         }
         tc_fence_before();
@@ -495,8 +575,9 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           tma_store_commit();
         }
       }
-      tc_fence_before();   // the next head pair's MMAs overwrite S_i / O_i after these reads
+      tc_fence_before();   // the next head pair's MMAs overwrite O_i after these reads
       ++g;
+      if (two_heads) ++g_two;
     }
     }
     if (q == 0 && lane == 0) tma_store_wait_all();   // the stores read shared memory: finish before the CTA may exit

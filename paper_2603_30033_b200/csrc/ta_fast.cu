@@ -188,13 +188,16 @@ bool attention_fuses_qhat(const tucker_attn_desc& d) {
 }
 
 // ---- workspace ----------------------------------------------------------------------------
+// Row pitch (elements) of the transposed value tensor: a TMA global stride is a multiple of 16 bytes.
+long value_ld(int N) { return ((long)N + 7) / 8 * 8; }
 struct FastWs {
   float2* rope;   // [N][r3/2]
   bf16* GcatT;    // [n_H * r3, r2]      B operand of the per-head query GEMM
   bf16* GtP;      // [t2, n_H * t3]      B operand of the Z GEMM
   bf16* Qt;       // [T, r2]
   bf16* K;        // [T, r3]  rotated
-  bf16* V;        // [T, t3]
+  bf16* V;        // [T, t3]                 (the FMA attention reads the values token-major)
+  bf16* Vt;       // [B, t3, value_ld(N)]    transposed values: the K-major B operand of P V in the tensor-core attention
   bf16* Qhat;     // [T, n_H * r3]
   bf16* O;        // [T, n_H * t3]
   bf16* Z;        // [T, t2]
@@ -210,6 +213,7 @@ size_t carve_fast(const tucker_attn_desc& d, char* base, FastWs* w) {
   t.Qt = c.take<bf16>(T * d.r2);
   t.K = c.take<bf16>(T * d.r3);
   t.V = c.take<bf16>(T * d.t3);
+  t.Vt = c.take<bf16>((size_t)d.B * d.t3 * value_ld(d.N));
   t.Qhat = c.take<bf16>(attention_fuses_qhat(d) ? 0 : T * d.n_H * d.r3);
   t.O = c.take<bf16>(T * d.n_H * d.t3);
   t.Z = c.take<bf16>(T * d.t2);
@@ -299,8 +303,9 @@ int head_pairs_per_item(const tucker_attn_desc& d, int n_qt, int n_hp) {
 }
 
 // Q: Qt [T, r2] when the kernel forms Qhat itself (G = GcatT [n_H * r3, r2] then), else Qhat [T, n_H * r3].
+// Vt: the values transposed, [B, t3, value_ld(N)].
 int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const float2* rope, const bf16* K,
-                   const bf16* V, bf16* O) {
+                   const bf16* Vt, bf16* O) {
   const tucker_attn_desc& d = p.d;
   CUtensorMap tmQ, tmG, tmK, tmV, tmO;
   {
@@ -319,7 +324,9 @@ int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const f
     tmG = tmQ;
   }
   if (!tmap_3d(&tmK, K, d.r3, d.N, d.B, d.r3, (uint64_t)d.N * d.r3, 64, 128)) return TA_ERR_CUDA;
-  if (!tmap_3d(&tmV, V, d.t3, d.N, d.B, d.t3, (uint64_t)d.N * d.t3, 64, 128)) return TA_ERR_CUDA;
+  // (keys, value column, sequence): keys beyond N are zero-filled by TMA, the row pitch is padded to 16 bytes
+  if (!tmap_3d(&tmV, Vt, d.N, d.t3, d.B, (uint64_t)value_ld(d.N), (uint64_t)d.t3 * value_ld(d.N), 64, (uint32_t)d.t3))
+    return TA_ERR_CUDA;
   attn::Params ap;
   ap.B = d.B; ap.N = d.N; ap.nH = d.n_H; ap.r2 = d.r2; ap.r3 = d.r3; ap.t3 = d.t3; ap.causal = d.causal;
   ap.n_qt = (d.N + attn::BQ - 1) / attn::BQ;
@@ -348,6 +355,7 @@ umma_gemm::Seg seg(int n_begin, int width, int mode, void* out, long ld) {
   umma_gemm::Seg s;
   s.n_begin = n_begin; s.width = width; s.mode = mode; s.out = out; s.ld = ld;
   s.out2 = nullptr; s.ld2 = 0; s.batch2 = 0;
+  s.outT = nullptr; s.ldT = 0; s.batchT = 0;
   s.bmap = 0; s.b_n_off = n_begin;
   return s;
 }
@@ -410,6 +418,12 @@ int fast_fwd(Problem& p) {
       if (!p.shared_rope) { gp.seg[1].out2 = p.Kc; gp.seg[1].ld2 = d.r3; gp.seg[1].batch2 = (long)p.Lmax * d.r3; }
       gp.seg[2].out2 = p.Vc; gp.seg[2].ld2 = d.t3; gp.seg[2].batch2 = (long)p.Lmax * d.t3;
     }
+    if (tc_attn) {
+      // the tensor-core attention takes the value tile with the key index contiguous (K-major operand of P V)
+      umma_gemm::Seg& vs = gp.seg[nseg - 1];
+      vs.outT = w.Vt; vs.ldT = value_ld(d.N); vs.batchT = (long)d.t3 * value_ld(d.N);
+      if (!p.shared_kv) vs.out = nullptr;   // nobody reads the token-major copy
+    }
     const BOperand bops[3] = {{(const bf16*)p.U2, d.r2, d.r2}, {(const bf16*)p.U3, d.r3, d.r3}, {(const bf16*)p.Ut3, d.t3, d.t3}};
     const int ntot = d.r2 + d.r3 + (p.shared_kv ? 0 : d.t3);
     // When X does not fit the L2 cache, each segment's pass over it would come from HBM again; one
@@ -434,7 +448,7 @@ int fast_fwd(Problem& p) {
   }
   // ---- attention ----
   if (tc_attn) {
-    if ((rc = umma_attention(p, fuse_q, fuse_q ? w.Qt : w.Qhat, w.GcatT, w.rope, w.K, Vlat, w.O))) return rc;
+    if ((rc = umma_attention(p, fuse_q, fuse_q ? w.Qt : w.Qhat, w.GcatT, w.rope, w.K, w.Vt, w.O))) return rc;
   } else {
     if ((rc = simt_attention_bf16(p, w.Qhat, w.K, Vlat, w.O))) return rc;
   }

@@ -41,10 +41,12 @@ struct Seg {
   int n_begin;   // first column of this segment in the concatenated N
   int width;     // columns in this segment (a multiple of the tile width BN)
   int mode;      // EP_*
-  void* out;     // destination, row-major [M, width] with leading dimension ld (elements)
+  void* out;     // destination, row-major [M, width] with leading dimension ld (elements); nullptr = not stored
   long ld;
   void* out2;    // optional second bf16 copy: element (row = b*n_pos + n, c) -> out2[b*batch2 + n*ld2 + c]
   long ld2, batch2;
+  void* outT;    // optional transposed bf16 copy: element (row = b*n_pos + n, c) -> outT[b*batchT + c*ldT + n]
+  long ldT, batchT;
   int bmap;      // which B tensor map (0..2) holds this segment's columns
   int b_n_off;   // N coordinate of the segment's first column inside that map
 };
@@ -259,6 +261,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
             for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
           }
+          if (sg.outT && row < p.M) {
+            // transposed copy: for a fixed column the 32 lanes of the warp write 32 consecutive positions
+            const int gb = p.n_pos > 0 ? row / p.n_pos : 0, gn = p.n_pos > 0 ? row % p.n_pos : row;
+            [[maybe_unused]] const long nbT = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
+            uint16_t* dstT = static_cast<uint16_t*>(sg.outT) + (long)gb * sg.batchT + gn;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const long o0 = (long)(col + 2 * i) * sg.ldT;
+              if (TA_IDX_OK(p.err, (long)gb * sg.batchT + o0 + gn, 1, nbT * sg.batchT)) dstT[o0] = (uint16_t)(o[i] & 0xffffu);
+              if (TA_IDX_OK(p.err, (long)gb * sg.batchT + o0 + sg.ldT + gn, 1, nbT * sg.batchT)) dstT[o0 + sg.ldT] = (uint16_t)(o[i] >> 16);
+            }
+          }
           uint4* sdst = reinterpret_cast<uint4*>(stage + (size_t)rloc * pitch + ch * 64);
 #pragma unroll
           for (int i = 0; i < 4; ++i) sdst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
@@ -272,7 +286,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (grow >= p.M) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(stage + (size_t)rr * pitch + ch * 64 + cc * 16);
             const int col = c0 + ch * 32 + cc * 8;
-            if (TA_IDX_OK(p.err, (long)grow * sg.ld + col, 8, (long)(p.M - 1) * sg.ld + sg.width))
+            if (sg.out && TA_IDX_OK(p.err, (long)grow * sg.ld + col, 8, (long)(p.M - 1) * sg.ld + sg.width))
               *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.out) + (long)grow * sg.ld + col) = v;
             if (sg.out2) {
               const int gb = p.n_pos > 0 ? grow / p.n_pos : 0, gn = p.n_pos > 0 ? grow % p.n_pos : grow;
