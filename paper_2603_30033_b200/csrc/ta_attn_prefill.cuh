@@ -10,23 +10,31 @@
 //   prologue   Qhat_i = Qt G_{h+i} on the tensor core (Qt tile loaded once per CTA, G tiles
 //              streamed through the V ring), latent RoPE applied while the result moves
 //              TMEM -> registers -> shared memory (bf16, the swizzled K-major layout UMMA reads)
-//   main loop  both heads use the same latent K / V tiles, so every tile is loaded once and
-//              serves two score tiles; the two softmax warpgroups ping-pong so that the tensor
-//              core works on one head while the other head's scores are being exponentiated
+//   main loop  both heads use the same latent K / V tiles, so every tile is loaded once and serves two score
+//              tiles.  The score tiles of the pair are produced in the order (key tile j, head i) -> t = 2 j + i
+//              into ONE score buffer: as soon as the softmax warpgroup of tile t holds it in registers, tile
+//              t + 1 (the other head's) is issued, so a warpgroup that finishes a tile finds its next scores
+//              ready, and the two warpgroups' exponentials overlap instead of waiting for each other's MMAs
 //   epilogue   O_i / l as bf16 into the head's idle Qhat tile, then out by a TMA tensor store that
 //              completes in the background while the warpgroup starts on the next head pair
 // In the unfused mode (query rank r2 > 128: the Qt tile would not fit) Qhat is read from
 // global memory instead and a CTA handles a single head pair.
 //
-//   warp 0        TMA producer: Qt (once), G tiles, K ring, V ring
-//   warp 1        MMA issuer:  Qhat_i = Qt G_i^T, S_i = Qhat_i K^T (smem x smem), O_i += P_i V (P from TMEM)
+//   warp 0        TMA producer: Qt (once per item), G tiles, K ring, V ring
+//   warp 1        score issuer: S = Qhat_i K^T (smem x smem)
+//   warp 2        value issuer: Qhat_i = Qt G_i^T, O_i += P_i V (P from TMEM, V^T tile K-major from shared memory)
 //   warps 4..7    softmax for head h   : thread t owns query row t (TMEM lane t)
 //   warps 8..11   softmax for head h+1
+// Two issuing threads, because an issuing thread is held until the tensor core has accepted its MMAs; the value
+// issuer lets a score tile that is ready at the same time go first (the tensor core runs MMAs in issue order, and
+// an idle warpgroup waits for the scores while nobody waits for the P V product).
 //
-// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,256+t3) O_1 [384,384+t3); the prologue
-// result occupies S_i; P_i (bf16, two per column) overwrites the first 64 columns of S_i once
-// the row has been read.  Scores arrive in log2 units (softmax scale * log2 e is folded into
-// G_h), so exp2 is used.  The running maximum is only raised when it grows by more than 8
+// The value tile comes from the transposed latent values V^T [B, t3, N] (written by the projection kernel), so
+// that both MMAs read K-major operands (an MN-major B operand costs about 40 cycles more per instruction).
+//
+// TMEM columns: S [0,128)  P_0 [128,192)  P_1 [192,256) (bf16, two per column)  O_0 [256,256+t3)  O_1 [384,384+t3);
+// the prologue's Qhat_0 / Qhat_1 accumulators occupy S and P_0|P_1.  Scores arrive in log2 units (softmax scale *
+// log2 e is folded into G_h), so exp2 is used.  The running maximum is only raised when it grows by more than 8
 // (factor 256), which keeps the O rescaling off the common path; l and O stay consistent
 // because both use the same stale maximum.
 #pragma once
@@ -121,8 +129,7 @@ __device__ __forceinline__ bool wait_count(const int* c, int target, const Abort
 
 // Eight-or-fewer K = 16 steps of one 128 x N product over K-major, 128-byte-swizzled shared-memory tiles whose
 // 64-element K blocks are SUB_BYTES apart: the step offsets are immediates added to the descriptors' address field.
-__device__ __forceinline__ void issue_kmajor_ss(uint32_t d_tmem, uint32_t a_saddr, uint32_t b_saddr, uint32_t idesc, int ksteps) {
-  const uint64_t ad = umma_desc_kmajor_sw128(a_saddr), bd = umma_desc_kmajor_sw128(b_saddr);
+__device__ __forceinline__ void issue_kmajor_ss(uint32_t d_tmem, uint64_t ad, uint64_t bd, uint32_t idesc, int ksteps) {
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
     if (ks < ksteps) {
@@ -292,21 +299,24 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         uint32_t sk = 0;
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int i = (nh == 2) ? (t & 1) : 0;
-          if (t >= 1) {
-            const int ip = (nh == 2) ? (i ^ 1) : 0;
-            if (!(ok = mbar_wait(&s_free[ip], (uint32_t)(((ip ? ns1 : ns0) - 1) & 1), ab))) break;
-          } else {
-            if (ns0 > 0 && !(ok = mbar_wait(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
-            if (ns1 > 0 && !(ok = mbar_wait(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
-          }
+          // everything that does not depend on the score buffer first: the hand-over of the buffer is the
+          // critical path of the tile sequence
           if (i == 0) {
             sk = (uint32_t)(it_k % KV_STAGES);
             if (!(ok = mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab))) break;
           }
           if (t < nh && p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)((i ? gp1 : gp0) & 1), ab))) break;
+          const uint64_t ad = umma_desc_kmajor_sw128(smem_u32(tiles) + (uint32_t)(1 + i) * (MAX_SUB * SUB_BYTES));
+          const uint64_t bd = umma_desc_kmajor_sw128(smem_u32(k_ring) + sk * (MAX_SUB * SUB_BYTES));
+          if (t >= 1) {
+            const int ip = (nh == 2) ? (i ^ 1) : 0;
+            if (!(ok = mbar_wait_poll(&s_free[ip], (uint32_t)(((ip ? ns1 : ns0) - 1) & 1), ab))) break;
+          } else {
+            if (ns0 > 0 && !(ok = mbar_wait_poll(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
+            if (ns1 > 0 && !(ok = mbar_wait_poll(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
+          }
           tc_fence_after();
-          issue_kmajor_ss(tm_s, smem_u32(tiles) + (uint32_t)(1 + i) * (MAX_SUB * SUB_BYTES),
-                          smem_u32(k_ring) + sk * (MAX_SUB * SUB_BYTES), idesc_qk, ksteps);
+          issue_kmajor_ss(tm_s, ad, bd, idesc_qk, ksteps);
           umma_commit(&s_full[i]);
           *(volatile int*)&qk_issued = ++n_issued;
           if (i) ++ns1; else ++ns0;
@@ -337,14 +347,14 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
           if (g == 0 && !(ok = mbar_wait(&q_full, (uint32_t)(k & 1), ab))) break;
           // the prologue accumulates into the score and probability columns: the last score tiles of the previous
           // pair must have been read (its P V products precede these MMAs in this thread's issue order)
-          if (ns0 > 0 && !(ok = mbar_wait(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
-          if (ns1 > 0 && !(ok = mbar_wait(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
+          if (ns0 > 0 && !(ok = mbar_wait_poll(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
+          if (ns1 > 0 && !(ok = mbar_wait_poll(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
           for (int i = 0; i < nh && ok; ++i, ++it_v) {
             const uint32_t s = (uint32_t)(it_v % KV_STAGES);
             if (!(ok = mbar_wait(&v_full[s], (it_v / KV_STAGES) & 1, ab))) break;
             tc_fence_after();
-            issue_kmajor_ss(tmem + (uint32_t)i * 128u, smem_u32(qt_tile), smem_u32(v_ring) + s * (MAX_SUB * SUB_BYTES), idesc_qh,
-                            p.r2 / 16);
+            issue_kmajor_ss(tmem + (uint32_t)i * 128u, umma_desc_kmajor_sw128(smem_u32(qt_tile)),
+                            umma_desc_kmajor_sw128(smem_u32(v_ring) + s * (MAX_SUB * SUB_BYTES)), idesc_qh, p.r2 / 16);
             umma_commit(&qh_done[i]);
             umma_commit(&v_empty[s]);
           }
@@ -360,7 +370,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             sv = (uint32_t)(it_v % KV_STAGES);
             if (!(ok = mbar_wait(&v_full[sv], (it_v / KV_STAGES) & 1, ab))) break;
           }
-          if (!(ok = mbar_wait(&p_full[i], (uint32_t)((i ? np1 : np0) & 1), ab))) break;
+          if (!(ok = mbar_wait_poll(&p_full[i], (uint32_t)((i ? np1 : np0) & 1), ab))) break;
           if (i) ++np1; else ++np0;
           // The tensor core runs MMAs in issue order, and an idle warpgroup is waiting for score tile t + 2 while
           // nobody waits for this product: when both are ready at about the same time the scores go first.  (Tile

@@ -86,6 +86,39 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
   }
 }
 
+// The same wait as a plain poll of mbarrier.test_wait, which never suspends the thread: for the single-thread MMA
+// issuers, whose reaction to a barrier sits on a kernel's critical path (measured on the long causal prefill: 1 %
+// of the attention kernel against the suspending form; for whole warps the polling costs more issue slots than it gains).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, const Abort& ab,
+                                               long long budget_cycles = kWaitBudgetCycles) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  int n = 0;
+  while (true) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if ((++n & 31) == 0) {           // the abort flag and the clock are looked at every 32nd poll
+      if (ab.raised()) return false;
+      if (clock64() - t0 > budget_cycles) {
+        ab.raise();
+        return false;
+      }
+    }
+  }
+}
+
 // ---- fences -----------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

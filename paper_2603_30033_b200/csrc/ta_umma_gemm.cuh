@@ -240,6 +240,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // segments of its chunks out, eight rows per 16-byte store instruction.
         const int pitch = (p.BN + 8) * 2;
         uint8_t* stage = tiles;
+        // transposed copy in 16-byte pieces (8 consecutive positions of one column) when 8-row groups never
+        // straddle a sequence
+        const bool outT_vec = sg.outT && (p.n_pos > 0 ? p.n_pos % 8 == 0 : p.M % 8 == 0);
         for (int ch = hf; ch < p.BN / 32; ch += 2) {
           uint32_t r[32];
           tmem_ld32(acc + (uint32_t)(ch * 32), r);
@@ -261,8 +264,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
             for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
           }
-          if (sg.outT && row < p.M) {
-            // transposed copy: for a fixed column the 32 lanes of the warp write 32 consecutive positions
+          if (sg.outT && !outT_vec && row < p.M) {
+            // transposed copy, general form: for a fixed column the 32 lanes of the warp write 32 consecutive positions
             const int gb = p.n_pos > 0 ? row / p.n_pos : 0, gn = p.n_pos > 0 ? row % p.n_pos : row;
             [[maybe_unused]] const long nbT = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
             uint16_t* dstT = static_cast<uint16_t*>(sg.outT) + (long)gb * sg.batchT + gn;
@@ -278,6 +281,32 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int i = 0; i < 4; ++i) sdst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
         }
         __syncwarp();
+        if (outT_vec) {
+          // lane -> column (lane / 4) of a group of 8 and 8-row group (lane % 4) of the warp's 32 rows: the four
+          // lanes of a column write 64 contiguous bytes
+          const int r8 = q * 32 + (lane % 4) * 8, grow0 = m0 + r8;
+          if (grow0 < p.M) {
+            const int gb = p.n_pos > 0 ? grow0 / p.n_pos : 0, gn = p.n_pos > 0 ? grow0 % p.n_pos : grow0;
+            [[maybe_unused]] const long nbT = p.n_pos > 0 ? (p.M + p.n_pos - 1) / p.n_pos : 1;
+            for (int ch = hf; ch < p.BN / 32; ch += 2) {
+#pragma unroll
+              for (int cg = 0; cg < 4; ++cg) {
+                const int cl = ch * 32 + cg * 8 + lane / 4;
+                const uint8_t* src = stage + (size_t)r8 * pitch + cl * 2;
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const uint32_t lo = *reinterpret_cast<const uint16_t*>(src + (size_t)(2 * e) * pitch);
+                  const uint32_t hi = *reinterpret_cast<const uint16_t*>(src + (size_t)(2 * e + 1) * pitch);
+                  w[e] = lo | (hi << 16);
+                }
+                const long off = (long)gb * sg.batchT + (long)(c0 + cl) * sg.ldT + gn;
+                if (TA_IDX_OK(p.err, off, 8, nbT * sg.batchT))
+                  *reinterpret_cast<uint4*>(static_cast<bf16*>(sg.outT) + off) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+        }
         const int rsub = lane / 4, cc = lane % 4;
         for (int ch = hf; ch < p.BN / 32; ch += 2) {
           for (int r0 = 0; r0 < 32; r0 += 8) {
