@@ -299,15 +299,18 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         uint32_t sk = 0;
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int i = (nh == 2) ? (t & 1) : 0;
-          // everything that does not depend on the score buffer first: the hand-over of the buffer is the
-          // critical path of the tile sequence
-          if (i == 0) {
-            sk = (uint32_t)(it_k % KV_STAGES);
-            if (!(ok = mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab))) break;
-          }
-          if (t < nh && p.fused && !(ok = mbar_wait(&qh_ready[i], (uint32_t)((i ? gp1 : gp0) & 1), ab))) break;
-          const uint64_t ad = umma_desc_kmajor_sw128(smem_u32(tiles) + (uint32_t)(1 + i) * (MAX_SUB * SUB_BYTES));
-          const uint64_t bd = umma_desc_kmajor_sw128(smem_u32(k_ring) + sk * (MAX_SUB * SUB_BYTES));
+          // Long rows: everything that does not depend on the score buffer first, since the hand-over of the buffer
+          // is the critical path of the tile sequence.  Short rows (a few tiles per pair) measured faster the other
+          // way round: there the K tile of a new pair is what arrives last.
+          auto wait_operands = [&]() -> bool {
+            if (i == 0) {
+              sk = (uint32_t)(it_k % KV_STAGES);
+              if (!mbar_wait(&k_full[sk], (it_k / KV_STAGES) & 1, ab)) return false;
+            }
+            return !(t < nh && p.fused) || mbar_wait(&qh_ready[i], (uint32_t)((i ? gp1 : gp0) & 1), ab);
+          };
+          const bool operands_first = nt >= 8;
+          if (operands_first && !(ok = wait_operands())) break;
           if (t >= 1) {
             const int ip = (nh == 2) ? (i ^ 1) : 0;
             if (!(ok = mbar_wait_poll(&s_free[ip], (uint32_t)(((ip ? ns1 : ns0) - 1) & 1), ab))) break;
@@ -315,6 +318,9 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (ns0 > 0 && !(ok = mbar_wait_poll(&s_free[0], (uint32_t)((ns0 - 1) & 1), ab))) break;
             if (ns1 > 0 && !(ok = mbar_wait_poll(&s_free[1], (uint32_t)((ns1 - 1) & 1), ab))) break;
           }
+          if (!operands_first && !(ok = wait_operands())) break;
+          const uint64_t ad = umma_desc_kmajor_sw128(smem_u32(tiles) + (uint32_t)(1 + i) * (MAX_SUB * SUB_BYTES));
+          const uint64_t bd = umma_desc_kmajor_sw128(smem_u32(k_ring) + sk * (MAX_SUB * SUB_BYTES));
           tc_fence_after();
           issue_kmajor_ss(tm_s, ad, bd, idesc_qk, ksteps);
           umma_commit(&s_full[i]);
