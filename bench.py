@@ -42,12 +42,12 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on this
 # workload: value, the summary under profiles/ it comes from, and the SHA-256 of the kernel's source file at the
 # time of the capture.  A value is only reported while that file is unchanged (see ncu_traffic()).
-_ATTN = {"source": "ta_attn_prefill.cuh", "sha256": "449037c0ea0d7b1971cef575c9b6b91e2348d9033efa446df10a80a62cd9c5d7"}
+_ATTN = {"source": "ta_attn_prefill.cuh", "sha256": "b16932a790c85d8d2267a871d06cadeb6d992d03bf49452c3542b200f75020fc"}
 _DEC = {"source": "ta_decode_umma.cuh", "sha256": "b29368639f2d9ea4a252a55117459bd2a1a167eff6dc63668ccc285447534b03"}
 NCU_TRAFFIC = {
-    "c4_long_prefill": {"bytes": 18273280 + 77136384, "profile": "profiles/k_attn_prefill_c4_long_prefill.md", **_ATTN},
-    "c3_vit_prefill": {"bytes": 32633600 + 65390592, "profile": "profiles/k_attn_prefill_c3_vit_prefill.md", **_ATTN},
-    "c2_gpt2_prefill": {"bytes": 3703040 + 0, "profile": "profiles/k_attn_prefill_c2_gpt2_prefill.md", **_ATTN},
+    "c4_long_prefill": {"bytes": 17910784 + 76981248, "profile": "profiles/k_attn_prefill_c4_long_prefill.md", **_ATTN},
+    "c3_vit_prefill": {"bytes": 33807104 + 64868608, "profile": "profiles/k_attn_prefill_c3_vit_prefill.md", **_ATTN},
+    "c2_gpt2_prefill": {"bytes": 3586816 + 0, "profile": "profiles/k_attn_prefill_c2_gpt2_prefill.md", **_ATTN},
     "c5_decode": {"bytes": 1075363072 + 4196608, "profile": "profiles/k_dec_attn_umma_c5_decode.md", **_DEC},
     "f1_decode_shared_kv": {"bytes": 537998592 + 4850688, "profile": "profiles/k_dec_attn_umma_f1_decode_shared_kv.md", **_DEC},
     "f1r_decode_shared_kv_rope": {"bytes": 538054400 + 6371328,
