@@ -430,6 +430,27 @@ def test_prefill_then_decode_with_one_unrotated_cache(dtype, shape, path):
     check(y.float().cpu().numpy().astype(np.float64), ref[:, N], dtype, f"decode after that prefill {shape}", scaled=True)
 
 
+@pytest.mark.parametrize("N", [200, 197])
+def test_prefill_with_one_shared_cache_without_rope(N):
+    # U3 == Ut3, no RoPE, one cache for keys and values: the projection has two segments, and the key segment is
+    # also the value tile of the attention kernel (written transposed, in 16-byte pieces when N is a multiple of 8)
+    import torch
+    shape = dict(d_model=256, n_H=8, r=(4, 64, 128), t=(4, 64, 128))
+    w = H.custom_workload(dtype="bf16", B=2, N=N, causal=True, rope=False, seed=71, **shape)
+    wt = _shared_weights(w)
+    X = W.round_to_storage(W.make_X(w), "bf16")
+    ref, parts = O.tucker_attn_fwd(X, *[wt[k] for k in H.WEIGHT_KEYS], causal=True, rope=False, return_parts=True)
+    dw = H.weights_to_device(wt, "bf16")
+    dw[7] = dw[3]
+    cache = torch.full((2, N + 5, 128), 7.0, device="cuda", dtype=torch.bfloat16)
+    Y = Bd.tucker_attn_fwd(H.to_device(X, "bf16"), *dw, n_H=w.n_H, causal=True, rope=False, Kcache=cache, Vcache=cache)
+    assert Bd.last_device_error() == 0 and Bd.last_path() == 2
+    check(Y.float().cpu().numpy().astype(np.float64), ref, "bf16", f"shared projection prefill N={N}", scaled=True)
+    for b in range(2):
+        assert np.abs(cache[b, :N].float().cpu().numpy() - parts[b]["V"][:N]).max() < 3e-2
+    assert (cache[:, N:] == 7.0).all()
+
+
 def test_decode_garbage_beyond_cache_len_is_ignored():
     # slots at and after cache_len hold NaN / Inf bit patterns: they must not leak into the result
     import torch
