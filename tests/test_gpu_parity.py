@@ -116,6 +116,32 @@ def test_small_shapes_tensor_core_path(shape):
     check(got, oracle_fwd(X, wt, w, pos0=3), "bf16", str(shape), scaled=scaled)
 
 
+def _random_shapes(seed, count):
+    import random
+    rng = random.Random(seed)
+    out = []
+    for _ in range(count):
+        nH = rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 12])
+        ranks = [rng.choice([32, 64, 96, 128]) for _ in range(4)]
+        out.append(dict(B=rng.choice([1, 2, 3]), N=rng.choice([1, 17, 64, 127, 128, 129, 200, 255, 256, 257, 384, 400, 520, 777]),
+                        d_model=nH * 64, n_H=nH, r=(min(nH, rng.choice([1, 2, 4])), ranks[0], ranks[1]),
+                        t=(min(nH, rng.choice([1, 2, 3])), ranks[2], ranks[3]), causal=rng.choice([True, False]),
+                        rope=rng.choice([True, False])))
+    return out
+
+
+@pytest.mark.parametrize("shape", _random_shapes(5, 32), ids=lambda s: "B%dN%dH%d" % (s["B"], s["N"], s["n_H"]))
+def test_random_shapes_tensor_core_path(shape):
+    # seeded random mixes of head counts (odd ones end on a single head), ranks, lengths around the tile edges,
+    # masks and RoPE: every role of the attention kernel's pipeline has to keep its barrier phases in step
+    w = H.custom_workload(dtype="bf16", rope_base=10000.0, seed=300 + shape["N"] + shape["n_H"], **shape)
+    X, wt = H.host_inputs(w)
+    got = gpu_fwd(X, wt, w)
+    assert Bd.last_path() == 2 and Bd.last_device_error() == 0
+    # a single token has no averaging over keys: its error is judged relative to the output's size
+    check(got, oracle_fwd(X, wt, w), "bf16", str(shape), scaled=shape["N"] == 1)
+
+
 def test_fused_and_unfused_query_paths_agree():
     # the attention kernel forming Qhat in its prologue vs reading it from the query GEMM
     w = H.custom_workload(dtype="bf16", B=2, N=300, d_model=256, n_H=8, r=(3, 128, 128), t=(3, 64, 128), causal=True,
