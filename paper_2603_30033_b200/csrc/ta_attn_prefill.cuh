@@ -73,7 +73,7 @@ struct Params {
   int n_hg;          // head-pair groups = ceil(n_hp / hp_per_item)
   int n_items;       // work items = n_qt * B * n_hg
   int fused;         // 1: tmQ is the map of Qt [B, N, r2] and Qhat is formed in the prologue
-  const float2* rope;   // [N][r3/2] (cos, sin) for rows of this call, or nullptr (fused mode only)
+  const float4* rope;   // (cos, sin) for the rows of this call in the rope_unit_index layout, or nullptr (fused mode only)
   bf16* O;           // [B, N, nH, t3] (written through the tensor map tmO)
   unsigned int* err;
 };
@@ -430,17 +430,17 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const float2* tab = (p.rope && row < p.N) ? p.rope + (long)row * (p.r3 / 2) : nullptr;
+        const float4* tab = (p.rope && row < p.N) ? p.rope + rope_unit_index(row, 0, p.r3 / 4) : nullptr;
         for (int ch = 0; ch < p.r3 / 32; ++ch) {
           uint32_t r[32];
           tmem_ld32(tm_qh[i] + lane_addr + ch * 32, r);
           tmem_ld_wait();
           uint32_t o[16];
           if (tab) {
-            const float4* t4 = reinterpret_cast<const float4*>(tab + ch * 16);
+            const float4* t4 = tab + ch * 8 * 32;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-              const float4 cs = t4[c];      // (cos, sin) of two consecutive pairs
+              const float4 cs = t4[c * 32];      // (cos, sin) of two consecutive pairs
               const float xe0 = __uint_as_float(r[4 * c]), xo0 = __uint_as_float(r[4 * c + 1]);
               const float xe1 = __uint_as_float(r[4 * c + 2]), xo1 = __uint_as_float(r[4 * c + 3]);
               o[2 * c] = pack_bf16(xe0 * cs.x - xo0 * cs.y, xe0 * cs.y + xo0 * cs.x);

@@ -91,6 +91,17 @@ int hosvd_run(Problem& p, int n1, int n2, int n3, int r1, int r2, int r3, const 
 int mha_weight_tensors_run(Problem& p, int d, int nH, const float* WQ, const float* WK, const float* WV, const float* WO,
                            float* W, float* Wt);
 
+// Layout of the prefill path's (cos, sin) table.  Its readers hold one position per thread and 32 consecutive
+// positions per warp, so the table is stored in units of one float4 = two (cos, sin) pairs, with the 32 positions
+// of a block of positions next to each other: unit u (0 .. r3/4 - 1) of position n lies at float4 index
+//   ((n / 32) * units + u) * 32 + n % 32,
+// and a warp's load of one unit for its 32 rows is one 512-byte segment.  (Stored position-major, every such load
+// touched 32 different rows of the table: 2500 cycles per 32 columns in the attention kernel's query conversion.)
+__host__ __device__ __forceinline__ long rope_unit_index(int n, int u, int units) {
+  return ((long)(n >> 5) * units + u) * 32 + (n & 31);
+}
+static inline size_t rope_table_units(int n_pos, int r3) { return (size_t)((n_pos + 31) / 32) * 32 * (size_t)(r3 / 4); }
+
 // Programmatic dependent launch.  Every kernel of the tensor-core paths starts with pdl_enter():
 // it waits until the preceding kernels of the stream have completed and their writes are visible,
 // and only then lets the next kernel of the stream be scheduled.  Launched through launch_pdl, a

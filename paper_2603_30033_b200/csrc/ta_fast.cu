@@ -70,7 +70,7 @@ bool tmap_2d(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uin
 struct PrepParams {
   const bf16 *C, *U1, *Ct, *Ut1;
   bf16 *GcatT, *GtP;
-  float2* rope;
+  float4* rope;     // rope_unit_index layout
   int nH, r1, r2, r3, t1, t2, t3;
   int n_pos, pos0;
   float mult;
@@ -154,19 +154,16 @@ __global__ void __launch_bounds__(PREP_THREADS) k_prefill_prep(const PrepParams 
         *reinterpret_cast<uint4*>(p.GtP + ((long)j * p.nH + h) * p.t3 + c8) = pack8(acc);
     }
   } else {
-    // (cos, sin) table: four consecutive pairs of one position per thread, two 16-byte stores
-    const int half = p.r3 / 2;                      // a multiple of 16
-    const long i4 = ((long)(blk - p.g1 - p.g2) * PREP_THREADS + t) * 4;
-    if (i4 < (long)p.n_pos * half) {
-      const int pos = p.pos0 + (int)(i4 / half), i0 = (int)(i4 % half);
-      float2 cs[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) cs[e] = dec::rope_cos_sin_theta(pos, p.freqs.theta[i0 + e]);
-      float4* dst = reinterpret_cast<float4*>(p.rope + i4);
-      if (TA_IDX_OK(p.err, i4, 4, (long)p.n_pos * half)) {
-      dst[0] = make_float4(cs[0].x, cs[0].y, cs[1].x, cs[1].y);
-      dst[1] = make_float4(cs[2].x, cs[2].y, cs[3].x, cs[3].y);
-      }
+    // (cos, sin) table: one unit (two pairs of one position) per thread, in storage order (see rope_unit_index),
+    // so that the stores of a warp are contiguous; the positions that pad the last block of 32 are filled too
+    const int units = p.r3 / 4;
+    const long o = (long)(blk - p.g1 - p.g2) * PREP_THREADS + t;
+    const long total = (long)((p.n_pos + 31) / 32) * 32 * units;
+    if (o < total) {
+      const int n = (int)(o / (32L * units)) * 32 + (int)(o % 32), u = (int)((o / 32) % units);
+      const float2 c0 = dec::rope_cos_sin_theta(p.pos0 + n, p.freqs.theta[2 * u]);
+      const float2 c1 = dec::rope_cos_sin_theta(p.pos0 + n, p.freqs.theta[2 * u + 1]);
+      if (TA_IDX_OK(p.err, o, 1, total)) p.rope[o] = make_float4(c0.x, c0.y, c1.x, c1.y);
     }
   }
 }
@@ -191,7 +188,7 @@ bool attention_fuses_qhat(const tucker_attn_desc& d) {
 // Row pitch (elements) of the transposed value tensor: a TMA global stride is a multiple of 16 bytes.
 long value_ld(int N) { return ((long)N + 7) / 8 * 8; }
 struct FastWs {
-  float2* rope;   // [N][r3/2]
+  float4* rope;   // (cos, sin) of every position and pair, rope_unit_index layout
   bf16* GcatT;    // [n_H * r3, r2]      B operand of the per-head query GEMM
   bf16* GtP;      // [t2, n_H * t3]      B operand of the Z GEMM
   bf16* Qt;       // [T, r2]
@@ -207,7 +204,7 @@ size_t carve_fast(const tucker_attn_desc& d, char* base, FastWs* w) {
   Carver c(base);
   const size_t T = (size_t)d.B * d.N;
   FastWs t;
-  t.rope = c.take<float2>(d.rope ? (size_t)d.N * (d.r3 / 2) : 0);
+  t.rope = c.take<float4>(d.rope ? rope_table_units(d.N, d.r3) : 0);
   t.GcatT = c.take<bf16>((size_t)d.n_H * d.r3 * d.r2);
   t.GtP = c.take<bf16>((size_t)d.t2 * d.n_H * d.t3);
   t.Qt = c.take<bf16>(T * d.r2);
@@ -304,7 +301,7 @@ int head_pairs_per_item(const tucker_attn_desc& d, int n_qt, int n_hp) {
 
 // Q: Qt [T, r2] when the kernel forms Qhat itself (G = GcatT [n_H * r3, r2] then), else Qhat [T, n_H * r3].
 // Vt: the values transposed, [B, t3, value_ld(N)].
-int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const float2* rope, const bf16* K,
+int umma_attention(Problem& p, bool fused, const bf16* Q, const bf16* G, const float4* rope, const bf16* K,
                    const bf16* Vt, bf16* O) {
   const tucker_attn_desc& d = p.d;
   CUtensorMap tmQ, tmG, tmK, tmV, tmO;
@@ -392,7 +389,7 @@ int fast_fwd(Problem& p) {
     // one block per 32 x 32 tile of every G_h^T, one thread per 8 outputs of Gt / 4 entries of the table
     pp.g1 = d.n_H * (d.r2 / 32) * (d.r3 / 32);
     pp.g2 = (int)(((long)d.n_H * d.t2 * (d.t3 / 8) + PREP_THREADS - 1) / PREP_THREADS);
-    pp.g3 = d.rope ? (int)(((long)d.N * (d.r3 / 2) / 4 + PREP_THREADS - 1) / PREP_THREADS) : 0;
+    pp.g3 = d.rope ? (int)((rope_table_units(d.N, d.r3) + PREP_THREADS - 1) / PREP_THREADS) : 0;
     (void)launch_pdl(k_prefill_prep, dim3(pp.g1 + pp.g2 + pp.g3), dim3(PREP_THREADS), 0, p.stream, pp);
     TA_LAUNCH_CHECK(p);
   }

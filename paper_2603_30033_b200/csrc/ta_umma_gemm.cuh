@@ -57,7 +57,7 @@ struct Params {
   int stages;              // ring depth, 1..MAX_STAGES
   int b_mn_major;          // 1: B is given as [K, N] with N contiguous (no transpose needed)
   Seg seg[3];
-  const float2* rope_tab;  // [n_pos][rope_half] (cos, sin); EP_BF16_ROPE only
+  const float4* rope_tab;  // (cos, sin) pairs of positions 0 .. n_pos - 1 in the rope_unit_index layout; EP_BF16_ROPE only
   int n_pos, rope_half;    // row -> position = row % n_pos; RoPE period in columns = 2*rope_half
   int early;               // 0: everything waits for the preceding kernel; 1: A and B were complete before the
                            // preceding kernel started, only the epilogue (tables, outputs) waits; 2: B only
@@ -251,13 +251,16 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           uint32_t o[16];
           if (sg.mode == EP_BF16_ROPE) {
             const int period = 2 * p.rope_half;
-            const float2* tab = p.rope_tab + (long)npos * p.rope_half + ((col % period) >> 1);
+            // eight units (two pairs each) of this row's position; the 32 rows of the warp read neighbouring entries
+            const float4* tab = p.rope_tab + rope_unit_index(npos, (col % period) >> 2, p.rope_half / 2);
             if (row < p.M) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const float2 cs = tab[i];
-                const float xe = __uint_as_float(r[2 * i]), xo = __uint_as_float(r[2 * i + 1]);
-                o[i] = pack_bf16(xe * cs.x - xo * cs.y, xe * cs.y + xo * cs.x);
+              for (int i = 0; i < 8; ++i) {
+                const float4 cs = tab[i * 32];
+                const float xe0 = __uint_as_float(r[4 * i]), xo0 = __uint_as_float(r[4 * i + 1]);
+                const float xe1 = __uint_as_float(r[4 * i + 2]), xo1 = __uint_as_float(r[4 * i + 3]);
+                o[2 * i] = pack_bf16(xe0 * cs.x - xo0 * cs.y, xe0 * cs.y + xo0 * cs.x);
+                o[2 * i + 1] = pack_bf16(xe1 * cs.z - xo1 * cs.w, xe1 * cs.w + xo1 * cs.z);
               }
             }
           } else {
