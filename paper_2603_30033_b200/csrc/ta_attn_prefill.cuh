@@ -414,16 +414,18 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const int h0 = hp * 2;
       const bool two_heads = (h0 + 1) < p.nH;
       if (i == 1 && !two_heads) continue;         // odd head count: the last pair has one head
-      if (g > 0) {
-        // the previous pair's output store must have finished reading this head's Qhat tile
+      // The previous pair's output store must have finished reading this head's Qhat tile before the tile is written
+      // again: waited for as late as possible (the fused prologue reads and rotates its first chunk before).
+      auto wait_stage_free = [&]() -> bool {
+        if (g == 0) return true;
         if (q == 0 && lane == 0) {
           tma_store_wait_read();
           mbar_arrive(&stage_free[i]);
         }
-        ok = mbar_wait(&stage_free[i], (uint32_t)((g - 1) & 1), ab);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
+        const bool w = mbar_wait(&stage_free[i], (uint32_t)((g - 1) & 1), ab);
+        return __all_sync(0xffffffffu, w);
+      };
+      if (!p.fused && !(ok = wait_stage_free())) break;
       if (p.fused) {
         // ---- prologue: Qhat row from TMEM, latent RoPE, bf16, swizzled K-major store ----
         ok = mbar_wait(&qh_done[i], (uint32_t)(g & 1), ab);
@@ -450,6 +452,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
             for (int c = 0; c < 16; ++c) o[c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
           }
+          if (ch == 0 && !(ok = wait_stage_free())) break;
           uint8_t* dst = q_tile[i] + (ch >> 1) * SUB_BYTES + rloc * 128;
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
@@ -458,6 +461,7 @@ k_attn_prefill(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
           }
         }
+        if (!ok) break;
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
