@@ -154,10 +154,11 @@ struct Item {
 };
 __device__ __forceinline__ bool get_item(const Params& p, int k, Item& im) {
   const int G = (int)gridDim.x;
-  long item = (long)k * G + ((k & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
-  if (item >= p.n_items) return false;
-  const int hg = (int)(item % p.n_hg); item /= p.n_hg;
-  im.b = (int)(item % p.B); item /= p.B;
+  const long item64 = (long)k * G + ((k & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
+  if (item64 >= p.n_items) return false;
+  unsigned item = (unsigned)item64;          // (n_items < 2^30: 32-bit divisions, every role calls this per item)
+  const int hg = (int)(item % (unsigned)p.n_hg); item /= (unsigned)p.n_hg;
+  im.b = (int)(item % (unsigned)p.B); item /= (unsigned)p.B;
   im.qt = p.n_qt - 1 - (int)item;            // heaviest (largest query tile) first
   im.q0 = im.qt * BQ;
   im.hp_begin = hg * p.hp_per_item;
