@@ -42,12 +42,12 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from an ncu capture of that kernel on this
 # workload: value, the summary under profiles/ it comes from, and the SHA-256 of the kernel's source file at the
 # time of the capture.  A value is only reported while that file is unchanged (see ncu_traffic()).
-_ATTN = {"source": "ta_attn_prefill.cuh", "sha256": "a470d056b7728ae35522d0cb674f7cbb078b160da3d502fec768719bfffc67ce"}
+_ATTN = {"source": "ta_attn_prefill.cuh", "sha256": "83abe4f00b82ea24232967bb6792cee9c2eed58417272c517f4f348ff22e88c6"}
 _DEC = {"source": "ta_decode_umma.cuh", "sha256": "b29368639f2d9ea4a252a55117459bd2a1a167eff6dc63668ccc285447534b03"}
 NCU_TRAFFIC = {
-    "c4_long_prefill": {"bytes": 17910272 + 77007872, "profile": "profiles/k_attn_prefill_c4_long_prefill.md", **_ATTN},
-    "c3_vit_prefill": {"bytes": 33903360 + 64315904, "profile": "profiles/k_attn_prefill_c3_vit_prefill.md", **_ATTN},
-    "c2_gpt2_prefill": {"bytes": 3586560 + 0, "profile": "profiles/k_attn_prefill_c2_gpt2_prefill.md", **_ATTN},
+    "c4_long_prefill": {"bytes": 17971968 + 77637120, "profile": "profiles/k_attn_prefill_c4_long_prefill.md", **_ATTN},
+    "c3_vit_prefill": {"bytes": 33884416 + 64199424, "profile": "profiles/k_attn_prefill_c3_vit_prefill.md", **_ATTN},
+    "c2_gpt2_prefill": {"bytes": 3584256 + 0, "profile": "profiles/k_attn_prefill_c2_gpt2_prefill.md", **_ATTN},
     "c5_decode": {"bytes": 1075363072 + 4196608, "profile": "profiles/k_dec_attn_umma_c5_decode.md", **_DEC},
     "f1_decode_shared_kv": {"bytes": 537998592 + 4850688, "profile": "profiles/k_dec_attn_umma_f1_decode_shared_kv.md", **_DEC},
     "f1r_decode_shared_kv_rope": {"bytes": 538054400 + 6371328,

@@ -43,10 +43,14 @@
 #include "ta_sm100.cuh"
 
 // Which of every eight consecutive score pairs of a row take their exponential on the FMA pipe instead of the
-// MUFU unit (bit c & 7).  Measured on the long causal prefill (attention kernel, CUDA events): none 1.000 ms,
-// 2 of 8 0.983 ms, 3 of 8 1.014 ms, 4 of 8 1.022 ms.
+// MUFU unit (bit c & 7); a build-time option, none by default.  Measured on the long causal prefill (attention
+// kernel, CUDA events).  With one score buffer per head, where one warp per scheduler exponentiated at a time:
+// none 1.000 ms, 2 of 8 0.983 ms, 3 of 8 1.014 ms.  With the one shared score buffer, where both warpgroups
+// exponentiate at once and the hand-over chain of the buffer sets the pace: none 0.819 - 0.824 ms, 1 of 8 0.825,
+// 2 of 8 0.836 - 0.845, 3 of 8 0.913 - 0.915 (the polynomial's instructions lengthen each warp's tile; the MUFU
+// unit, 49 % busy, is not what the warps wait for).
 #ifndef TA_FMA_EXP_MASK
-#define TA_FMA_EXP_MASK 0x88u
+#define TA_FMA_EXP_MASK 0x00u
 #endif
 
 namespace ta {
